@@ -1,0 +1,188 @@
+"""CPU oracle for the CDL quantized layer: thin numpy/ctypes face of cdl_oracle.c.
+
+TEST INFRASTRUCTURE ONLY.  The arithmetic lives in ``cdl_oracle.c`` (plain C,
+double precision, one function per definition of the paper); this module only
+compiles it with gcc, loads it and marshals numpy arrays.  It imports nothing
+from the CUDA package, and the CUDA package imports nothing from here.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "cdl_oracle.c"
+_SO = _HERE / "libcdl_oracle.so"
+
+MAX_LEVELS = 256
+
+
+def build(force: bool = False) -> Path:
+    """Compile cdl_oracle.c into libcdl_oracle.so (no-op when up to date)."""
+    if force or not _SO.exists() or _SO.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _SO.with_suffix(f".so.tmp{os.getpid()}")
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+               "-o", str(tmp), str(_SRC), "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _SO)
+    return _SO
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_SO))
+        c = ctypes
+        P = c.c_void_p
+        lib.cdl_oracle_threads.restype = c.c_int
+        lib.cdl_oracle_cpmf.argtypes = [c.c_double, c.c_double, c.c_int, c.c_int, c.c_double, c.c_int, P]
+        lib.cdl_oracle_soft.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, P]
+        lib.cdl_oracle_partials.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int,
+                                            P, P, P, P]
+        lib.cdl_oracle_hard.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, P, P]
+        lib.cdl_oracle_entropy.argtypes = [P, c.c_int, P, P, P]
+        lib.cdl_oracle_backward.argtypes = [P, P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int,
+                                            c.c_float, P, P, P, P, P, P]
+        lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        for f in ("cpmf", "soft", "partials", "hard", "entropy", "backward", "gemm_fwd", "gemm_dx", "gemm_dw"):
+            getattr(lib, "cdl_oracle_" + f).restype = None
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+def _check_levels(lo, hi):
+    if not (1 <= hi - lo + 1 <= MAX_LEVELS):
+        raise ValueError("index set must have 1..256 levels")
+
+
+def threads() -> int:
+    """Host threads the oracle's parallel loops use."""
+    return int(_load().cdl_oracle_threads())
+
+
+def cpmf(theta, q, lo, hi, alpha, window=0):
+    """P_alpha(. | theta) over the levels lo..hi (Sec. IV-A, Eq. (4)); float64[nlev]."""
+    _check_levels(lo, hi)
+    P = np.empty(hi - lo + 1, dtype=np.float64)
+    _load().cdl_oracle_cpmf(float(theta), float(q), lo, hi, float(alpha), window, _ptr(P))
+    return P
+
+
+def soft(x, q, lo, hi, alpha, window=0):
+    """Q_d(x) element-wise (Sec. IV-B, Eq. (8)); float64, same shape as x."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    y = np.empty(x.shape, dtype=np.float64)
+    _load().cdl_oracle_soft(_ptr(x), x.size, q, lo, hi, alpha, window, _ptr(y))
+    return y
+
+
+def partials(x, q, lo, hi, alpha, window=0):
+    """(dQ_d/dtheta, dQ_d/dq, dQ_d/dalpha, Var{Q_p|theta}) element-wise (Lemma 1)."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    outs = [np.empty(x.shape, dtype=np.float64) for _ in range(4)]
+    _load().cdl_oracle_partials(_ptr(x), x.size, q, lo, hi, alpha, window, *[_ptr(o) for o in outs])
+    return tuple(outs)
+
+
+def hard(x, q, lo, hi):
+    """Hard indices (int32, shape of x) and their histogram (uint64[nlev])."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    idx = np.empty(x.shape, dtype=np.int32)
+    hist = np.zeros(hi - lo + 1, dtype=np.uint64)
+    _load().cdl_oracle_hard(_ptr(x), x.size, q, lo, hi, _ptr(idx), _ptr(hist))
+    return idx, hist
+
+
+def entropy(hist):
+    """(H in bits, level probabilities float64[nlev], n) of a level histogram (Sec. V-C)."""
+    hist = np.ascontiguousarray(hist, dtype=np.uint64)
+    H = np.zeros(1, dtype=np.float64)
+    p = np.empty(hist.size, dtype=np.float64)
+    n = np.zeros(1, dtype=np.uint64)
+    _load().cdl_oracle_entropy(_ptr(hist), hist.size, _ptr(H), _ptr(p), _ptr(n))
+    return float(H[0]), p, int(n[0])
+
+
+def backward(x, g, q, lo, hi, alpha, window=0, rate_weight=0.0, level_prob=None):
+    """Quantizer backward (Sec. V-B).  Returns a dict with grad_x (float64 array),
+    grad_q, grad_alpha and the absolute-term sums abs_q, abs_alpha."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    g = _f32(g)
+    assert x.shape == g.shape
+    lp = None if level_prob is None else np.ascontiguousarray(level_prob, dtype=np.float64)
+    if lp is not None:
+        assert lp.size == hi - lo + 1
+    gx = np.empty(x.shape, dtype=np.float64)
+    s = np.zeros(4, dtype=np.float64)
+    sp = [ctypes.c_void_p(s.ctypes.data + 8 * i) for i in range(4)]
+    _load().cdl_oracle_backward(_ptr(x), _ptr(g), x.size, q, lo, hi, alpha, window, rate_weight,
+                                _ptr(lp), _ptr(gx), *sp)
+    return {"grad_x": gx, "grad_q": float(s[0]), "grad_alpha": float(s[1]),
+            "abs_q": float(s[2]), "abs_alpha": float(s[3])}
+
+
+def _idx_bytes(a):
+    a = np.asarray(a)
+    if a.dtype not in (np.int8, np.uint8):
+        raise TypeError("index operands are int8 or uint8")
+    assert a.ndim == 2 and a.strides[1] == 1
+    return a, a.strides[0], int(a.dtype == np.uint8)
+
+
+def gemm_fwd(A, W):
+    """ACC[m,n] = sum_k A[m,k] W[k,n] as int64; A int8|uint8 [M,K], W int8 [K,N]."""
+    A, lda, au = _idx_bytes(A)
+    W, ldw, wu = _idx_bytes(W)
+    assert not wu and A.shape[1] == W.shape[0]
+    M, K = A.shape
+    N = W.shape[1]
+    acc = np.empty((M, N), dtype=np.int64)
+    _load().cdl_oracle_gemm_fwd(_ptr(A), lda, au, _ptr(W), ldw, M, N, K, _ptr(acc))
+    return acc
+
+
+def gemm_dx(G, W):
+    """ACC[m,k] = sum_n G[m,n] W[k,n] as int64; G int8 [M,N], W int8 [K,N]."""
+    G, ldg, gu = _idx_bytes(G)
+    W, ldw, wu = _idx_bytes(W)
+    assert not gu and not wu and G.shape[1] == W.shape[1]
+    M, N = G.shape
+    K = W.shape[0]
+    acc = np.empty((M, K), dtype=np.int64)
+    _load().cdl_oracle_gemm_dx(_ptr(G), ldg, _ptr(W), ldw, M, N, K, _ptr(acc))
+    return acc
+
+
+def gemm_dw(A, G):
+    """ACC[k,n] = sum_m A[m,k] G[m,n] as int64; A int8|uint8 [M,K], G int8 [M,N]."""
+    A, lda, au = _idx_bytes(A)
+    G, ldg, gu = _idx_bytes(G)
+    assert not gu and A.shape[0] == G.shape[0]
+    M, K = A.shape
+    N = G.shape[1]
+    acc = np.empty((K, N), dtype=np.int64)
+    _load().cdl_oracle_gemm_dw(_ptr(A), lda, au, _ptr(G), ldg, M, N, K, _ptr(acc))
+    return acc
