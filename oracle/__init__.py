@@ -50,7 +50,7 @@ def _load():
         lib.cdl_oracle_hard.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, P, P]
         lib.cdl_oracle_entropy.argtypes = [P, c.c_int, P, P, P]
         lib.cdl_oracle_backward.argtypes = [P, P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int,
-                                            c.c_float, P, P, P, P, P, P]
+                                            c.c_float, P, P, P, P, P, P, P, P]
         lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
@@ -127,7 +127,7 @@ def entropy(hist):
 
 def backward(x, g, q, lo, hi, alpha, window=0, rate_weight=0.0, level_prob=None):
     """Quantizer backward (Sec. V-B).  Returns a dict with grad_x (float64 array),
-    grad_q, grad_alpha and the absolute-term sums abs_q, abs_alpha."""
+    grad_q, grad_alpha and the comparison scales abs_q, abs_alpha, mag_q, mag_alpha."""
     _check_levels(lo, hi)
     x = _f32(x)
     g = _f32(g)
@@ -136,12 +136,12 @@ def backward(x, g, q, lo, hi, alpha, window=0, rate_weight=0.0, level_prob=None)
     if lp is not None:
         assert lp.size == hi - lo + 1
     gx = np.empty(x.shape, dtype=np.float64)
-    s = np.zeros(4, dtype=np.float64)
-    sp = [ctypes.c_void_p(s.ctypes.data + 8 * i) for i in range(4)]
+    s = np.zeros(6, dtype=np.float64)
+    sp = [ctypes.c_void_p(s.ctypes.data + 8 * i) for i in range(6)]
     _load().cdl_oracle_backward(_ptr(x), _ptr(g), x.size, q, lo, hi, alpha, window, rate_weight,
                                 _ptr(lp), _ptr(gx), *sp)
     return {"grad_x": gx, "grad_q": float(s[0]), "grad_alpha": float(s[1]),
-            "abs_q": float(s[2]), "abs_alpha": float(s[3])}
+            "abs_q": float(s[2]), "abs_alpha": float(s[3]), "mag_q": float(s[4]), "mag_alpha": float(s[5])}
 
 
 def _idx_bytes(a):

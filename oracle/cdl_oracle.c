@@ -205,14 +205,19 @@ void cdl_oracle_entropy(const uint64_t *hist, int nlev, double *H_bits,
  *   grad_q     = sum_e g[e] * dQ_d/dq      (Eqs. (21), (22))
  *   grad_alpha = sum_e g[e] * dQ_d/dalpha  (Eqs. (23), (24))
  * level_prob == NULL or rate_weight == 0: no rate term.
- * abs_q / abs_alpha (nullable) receive sum_e |g[e] * partial|, the natural
- * scale for comparing a reduced sum computed in another precision.
+ * Two scales for comparing the reduced sums with a lower-precision result
+ * (all nullable): abs_q / abs_alpha receive sum_e |g[e] * partial|, and
+ * mag_q / mag_alpha receive sum_e |g[e]| * (sum of the magnitudes of the terms
+ * of the printed formula: |E| + |2 alpha theta Var| + |2 alpha Skew_u|, over q;
+ * |2 theta Var| + |Skew_u|), which bounds what cancellation between those
+ * terms can cost.
  * ------------------------------------------------------------------------- */
 void cdl_oracle_backward(const float *x, const float *g, int64_t n, float q,
                          int lo, int hi, float alpha, int window,
                          float rate_weight, const double *level_prob,
                          double *grad_x, double *grad_q, double *grad_alpha,
-                         double *abs_q, double *abs_alpha)
+                         double *abs_q, double *abs_alpha,
+                         double *mag_q, double *mag_alpha)
 {
     const int nlev = hi - lo + 1;
     double log2p[CDL_ORACLE_MAX_LEVELS];
@@ -221,8 +226,8 @@ void cdl_oracle_backward(const float *x, const float *g, int64_t n, float q,
         double p = with_rate ? level_prob[i] : 1.0;
         log2p[i] = (p < ldexp(1.0, -30)) ? -30.0 : log2(p);
     }
-    double sq = 0.0, sa = 0.0, aq = 0.0, aa = 0.0;
-#pragma omp parallel for schedule(static) reduction(+ : sq, sa, aq, aa)
+    double sq = 0.0, sa = 0.0, aq = 0.0, aa = 0.0, mq = 0.0, ma = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : sq, sa, aq, aa, mq, ma)
     for (int64_t e = 0; e < n; ++e) {
         double P[CDL_ORACLE_MAX_LEVELS];
         const double th = (double)x[e], a = (double)alpha, qq = (double)q;
@@ -246,11 +251,15 @@ void cdl_oracle_backward(const float *x, const float *g, int64_t n, float q,
         sa += ta;
         aq += fabs(tq);
         aa += fabs(ta);
+        mq += fabs(ge) * (fabs(E) + fabs(2.0 * a * th * Var) + fabs(2.0 * a * Sk)) / qq;
+        ma += fabs(ge) * (fabs(2.0 * th * Var) + fabs(Sk));
     }
     if (grad_q) *grad_q = sq;
     if (grad_alpha) *grad_alpha = sa;
     if (abs_q) *abs_q = aq;
     if (abs_alpha) *abs_alpha = aa;
+    if (mag_q) *mag_q = mq;
+    if (mag_alpha) *mag_alpha = ma;
 }
 
 /* ---------------------------------------------------------------------------
