@@ -1,0 +1,203 @@
+/*
+ * cdl.h - C ABI of the CDL quantized layer for NVIDIA B200 (sm_100a).
+ *
+ * Method: "Coded Deep Learning: Framework and Algorithm" (arXiv 2501.09849).
+ * The library computes, on the GPU, the per-element probabilistic quantizer of
+ * Sec. IV (CPMF, hard index, soft value Q_d, analytic partial derivatives of
+ * Lemma 1), the per-tensor level histogram and its entropy (Sec. V-C), and the
+ * forward / backward layer products over the integer indices (Sec. V-A,
+ * Algorithm 1, forward pass and backward pass).
+ *
+ * Conventions common to every entry point
+ *  - Pointers marked [dev] are device memory owned by the caller; [host] are
+ *    host memory read during the call only.  The library allocates no device
+ *    memory, keeps no state between calls and never synchronises the device
+ *    (cdl_workspace_status excepted): work is enqueued on `stream` (a
+ *    cudaStream_t passed as void*; NULL is the legacy default stream) and
+ *    outputs are valid once the stream reaches it.
+ *  - All matrices are row-major; leading dimensions are in elements.
+ *  - Return value: CDL_OK (0) or a negative cdl_status.  On an argument error
+ *    nothing has been launched.  No call aborts, throws or traps.
+ *  - Notation follows the paper: theta = a weight or an activation, q = step
+ *    size (q_l for weights, s_l for activations), index set {lo..hi}
+ *    (weights: -2^(b-1)..2^(b-1)-1, activations: 0..2^b-1, Sec. V-A; a
+ *    symmetric set -L..L is lo=-L, hi=L), alpha = CPMF parameter (alpha_l for
+ *    weights, beta_l for activations), rate weight = lambda or gamma (Sec. V-D).
+ */
+#ifndef CDL_H_
+#define CDL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CDL_VERSION 100 /* 0.1.0 */
+#define CDL_MAX_LEVELS 256
+
+typedef enum cdl_status {
+    CDL_OK = 0,
+    CDL_ERR_ARG = -1,           /* NULL where a pointer is required, negative size, even window, bad flag */
+    CDL_ERR_ALIGN = -2,         /* pointer or leading dimension not aligned as documented */
+    CDL_ERR_RANGE = -3,         /* q <= 0, alpha <= 0, non-finite parameter, more than 256 levels,
+                                   index set not representable in the index byte */
+    CDL_ERR_WORKSPACE = -4,     /* workspace NULL, misaligned or smaller than cdl_workspace_bytes() */
+    CDL_ERR_OVERFLOW_RISK = -5, /* an int32 accumulator could overflow for these sizes and index ranges */
+    CDL_ERR_LAUNCH = -6,        /* the CUDA runtime refused a launch or a driver call */
+    CDL_ERR_TIMEOUT = -7,       /* a bounded device-side wait expired (reported by cdl_workspace_status) */
+    CDL_ERR_UNSUPPORTED = -8    /* the current device is not compute capability 10.x */
+} cdl_status;
+
+/* Flags of cdl_quant_params.flags */
+#define CDL_HIST_ACCUMULATE 0x1u /* add to the histogram instead of clearing it first */
+
+/*
+ * One trainable quantizer (Sec. IV-A, Sec. V-A): step size, index set, CPMF parameter.
+ *   q           step size, finite, > 0.
+ *   lo, hi      index set {lo..hi}, 1 <= hi-lo+1 <= 256.  Index bytes are int8 when lo < 0
+ *               (requires -128 <= lo, hi <= 127) and uint8 otherwise (requires hi <= 255).
+ *   alpha       CPMF parameter of Eq. (4), finite, > 0.
+ *   rate_weight lambda (weights) or gamma (activations) of the objective of Sec. V-D, finite, >= 0.
+ *               Only cdl_quantize_backward reads it.
+ *   level_prob  [dev] nlev floats, the level probabilities the rate term differentiates through
+ *               (normally written by cdl_index_entropy), or NULL for "no rate term".  The paper's CPMF
+ *               has no rate term in its logits: the rate acts through the gradient only.
+ *   window      0 = the CPMF over the whole index set (the definition).  An odd k > 0 keeps the k most
+ *               probable levels, i.e. the k in-range levels nearest theta, and renormalises
+ *               (Sec. VI-B.1 uses 5 for activations); of two equally distant levels the lower one is
+ *               kept.  k >= nlev is the same as 0.
+ */
+typedef struct cdl_quant_params {
+    float q;
+    int32_t lo, hi;
+    float alpha;
+    float rate_weight;
+    const float *level_prob;
+    int32_t window;
+    uint32_t flags;
+} cdl_quant_params;
+
+/* An index tensor as a GEMM operand: its step size and the range its entries lie in
+ * (bytes are int8 when lo < 0, uint8 otherwise).  The range only serves the overflow check. */
+typedef struct cdl_index_desc {
+    float q;
+    int32_t lo, hi;
+} cdl_index_desc;
+
+/*
+ * Hard index = uniform quantizer Q_u, the limit of Q_p and Q_d for large alpha (Remark of
+ * Sec. IV-A; end of Sec. IV-B), with the per-tensor level histogram fused in (the empirical
+ * distribution over levels whose entropy Sec. V-C constrains).
+ *   idx = clamp(round_half_even(x / q), lo, hi), quotient in IEEE binary32; NaN -> level nearest 0.
+ *   x        [dev] n floats (4-byte aligned; 16-byte alignment takes the vector path).
+ *   p        [host].
+ *   idx_out  [dev] n bytes (int8 or uint8, see cdl_quant_params), nullable.
+ *   hist     [dev] nlev uint64 counters, nullable; cleared first unless CDL_HIST_ACCUMULATE.
+ * n = 0 is valid (clears hist).  p->alpha, rate_weight, level_prob and window are not read.
+ */
+int cdl_quantize_hard(const float *x, int64_t n, const cdl_quant_params *p,
+                      void *idx_out, uint64_t *hist, void *stream);
+
+/*
+ * Soft deterministic quantizer Q_d(x) = sum_i P_alpha(iq | x) iq of Sec. IV-B, Eq. (8), with the
+ * CPMF of Eq. (4) (optionally truncated to p->window levels), and, in the same pass over x,
+ * optionally the hard index and the histogram exactly as cdl_quantize_hard writes them.
+ *   y_soft   [dev] n floats, required.   idx_out, hist: nullable.
+ * x must be finite for y_soft to be meaningful (NaN and infinities give NaN).
+ */
+int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p,
+                      float *y_soft, void *idx_out, uint64_t *hist, void *stream);
+
+/*
+ * Backward of the quantizer with Q_d as the gradient proxy (Sec. V-B, Eqs. (18), (20)-(24)):
+ *   grad_x[i]  = grad_out[i] * dQ_d/dtheta(x[i])                     Lemma 1, Eq. (9a): 2 alpha Var
+ *                + rate_weight * d(n H)/dtheta_i                      (only if level_prob != NULL)
+ *   grad_q     = sum_i grad_out[i] * dQ_d/dq(x[i])                   Lemma 1, Eq. (9b)
+ *   grad_alpha = sum_i grad_out[i] * dQ_d/dalpha(x[i])               = 2 theta Var - Skew_u (derived
+ *                                                                      with the steps of Appendix B)
+ * The rate term is the derivative of the total bits n*H of Sec. V-C w.r.t. theta_i with the level
+ * probabilities pbar held as passed in:  -2 alpha sum_k P_k log2(pbar_k) (k q - Q_d(theta_i));
+ * log2 of a probability below 2^-30 counts as -30.  The CPMF is recomputed from x; nothing is
+ * kept from the forward pass.
+ *   grad_out [dev] n floats: dL/dQ_p(x), the gradient arriving at the quantized tensor.
+ *   grad_x   [dev] n floats, nullable.
+ *   grad_q, grad_alpha [dev] one double each, nullable, overwritten (not accumulated).  Partial sums
+ *            are combined with floating-point atomics: the last bits can differ from run to run.
+ */
+int cdl_quantize_backward(const float *x, const float *grad_out, int64_t n,
+                          const cdl_quant_params *p, float *grad_x,
+                          double *grad_q, double *grad_alpha, void *stream);
+
+/*
+ * Entropy in bits of the level distribution given by a histogram (Sec. III-A definition of H,
+ * base 2; Sec. V-C: bits per weight / activation), and the level probabilities themselves.
+ *   hist        [dev] nlev uint64 counters.
+ *   H_bits      [dev] one double: -sum_k p_k log2 p_k, p_k = hist[k]/n, 0 log 0 = 0; 0 when n = 0.
+ *   level_prob  [dev] nlev floats p_k, nullable.      n_out [dev] one uint64 (= sum of hist), nullable.
+ */
+int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits,
+                      float *level_prob, uint64_t *n_out, void *stream);
+
+/*
+ * Forward layer product over the indices (Sec. V-A; Algorithm 1, forward pass) with the
+ * q_a * q_w rescale in the epilogue:
+ *   ACC[m,n] = sum_k A_idx[m,k] * W_idx[k,n]   (int32, exact)
+ *   Y[m,n]   = (float)ACC[m,n] * (a->q * w->q) + bias[n]   (a->q * w->q formed once in binary32;
+ *              multiply and add each rounded to binary32)
+ *   A_idx [dev] M x K bytes, leading dimension lda;  W_idx [dev] K x N int8, leading dimension ldw.
+ *   lda, ldw multiples of 16; A_idx, W_idx 16-byte aligned (TMA requirements).
+ *   acc_out [dev] M x N int32 (ld N), nullable.  y_out [dev] M x N floats (ld N), nullable.
+ *   bias [dev] N floats, nullable.  At least one of acc_out, y_out.
+ *   ws [dev]: cdl_workspace_bytes(CDL_OP_QLINEAR_FWD, M, N, K) bytes, 256-byte aligned.
+ * CDL_ERR_OVERFLOW_RISK when K * max|a| * max|w| >= 2^31 for the declared index ranges.
+ */
+int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                    const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                    int32_t M, int32_t N, int32_t K,
+                    int32_t *acc_out, float *y_out, const float *bias,
+                    void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Backward layer products over the indices (Algorithm 1, backward pass over the quantized weights
+ * and activations).  The gradient operand is an index tensor as well: the caller quantizes
+ * dL/dY with cdl_quantize_hard (for example lo=-127, hi=127 and a step g->q of its choice) - a
+ * reading of the paper, which does not say how the arriving gradient is represented.
+ *   dXACC[m,k] = sum_n G_idx[m,n] * W_idx[k,n]     dX[m,k] = (float)dXACC * (g->q * w->q)
+ *   dWACC[k,n] = sum_m A_idx[m,k] * G_idx[m,n]     dW[k,n] = (float)dWACC * (g->q * a->q)
+ *   G_idx [dev] M x N int8 (ld ldg);  A_idx M x K (ld lda);  W_idx K x N (ld ldw); all ld % 16 == 0,
+ *   all base pointers 16-byte aligned.
+ *   dXacc, dWacc [dev] int32 (ld K, ld N), dX, dW [dev] floats; each nullable.  A_idx may be NULL
+ *   when neither dWacc nor dW is wanted, W_idx when neither dXacc nor dX is.
+ *   ws [dev]: cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K) bytes, 256-byte aligned.
+ * CDL_ERR_OVERFLOW_RISK when N*max|g|*max|w| or M*max|a|*max|g| reaches 2^31.
+ */
+int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
+                    const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                    const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                    int32_t M, int32_t N, int32_t K,
+                    int32_t *dXacc, float *dX, int32_t *dWacc, float *dW,
+                    void *ws, size_t ws_bytes, void *stream);
+
+#define CDL_OP_QLINEAR_FWD 1
+#define CDL_OP_QLINEAR_BWD 2
+
+/* Bytes of device workspace the GEMM entry points need for these sizes; never less than the
+ * 256-byte status block at its start.  0 for an unknown op or non-positive sizes. */
+size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K);
+
+/* Synchronises `stream`, reads the status block at the start of a GEMM workspace and returns CDL_OK
+ * or CDL_ERR_TIMEOUT (a device-side wait gave up; the outputs of that call are then undefined). */
+int cdl_workspace_status(const void *ws, void *stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *cdl_strerror(int status);
+
+/* CDL_VERSION of the built library. */
+int cdl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CDL_H_ */

@@ -1,0 +1,311 @@
+// extern "C" entry points of libcdl.so: argument validation and launch plumbing.  See include/cdl.h
+// for the contract of every call.
+#include <math.h>
+#include <string.h>
+
+#include "cdl_internal.h"
+
+namespace cdl {
+
+namespace {
+constexpr int kMaxDevices = 64;
+int g_dev_ok[kMaxDevices];    // 0 unknown, 1 supported, -1 unsupported (cached device properties only)
+int g_dev_sms[kMaxDevices];
+}  // namespace
+
+int check_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    if (dev < 0 || dev >= kMaxDevices) return CDL_ERR_UNSUPPORTED;
+    if (g_dev_ok[dev] == 0) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+        g_dev_sms[dev] = sms;
+        g_dev_ok[dev] = (major == 10) ? 1 : -1;
+    }
+    return g_dev_ok[dev] == 1 ? CDL_OK : CDL_ERR_UNSUPPORTED;
+}
+
+int sm_count()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    return g_dev_sms[dev];
+}
+
+int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out)
+{
+    if (p == nullptr) return CDL_ERR_ARG;
+    if (p->flags & ~CDL_HIST_ACCUMULATE) return CDL_ERR_ARG;
+    if (!(p->q > 0.0f) || !isfinite(p->q)) return CDL_ERR_RANGE;
+    if (p->hi < p->lo) return CDL_ERR_RANGE;
+    const int64_t nlev = (int64_t)p->hi - (int64_t)p->lo + 1;
+    if (nlev > CDL_MAX_LEVELS) return CDL_ERR_RANGE;
+    if (p->lo < 0) {
+        if (p->lo < -128 || p->hi > 127) return CDL_ERR_RANGE;
+    } else if (p->hi > 255) {
+        return CDL_ERR_RANGE;
+    }
+    QuantDev d;
+    memset(&d, 0, sizeof d);
+    d.q = p->q;
+    d.half_q = 0.5f * p->q;
+    d.lo = p->lo;
+    d.hi = p->hi;
+    d.nlev = (int)nlev;
+    d.flo = (float)p->lo;
+    d.fhi = (float)p->hi;
+    if (need_alpha) {
+        if (!(p->alpha > 0.0f) || !isfinite(p->alpha)) return CDL_ERR_RANGE;
+        if (!(p->rate_weight >= 0.0f) || !isfinite(p->rate_weight)) return CDL_ERR_RANGE;
+        if (p->window < 0) return CDL_ERR_ARG;
+        if (p->window > 0 && (p->window & 1) == 0) return CDL_ERR_ARG;
+        const double q = (double)p->q, al = (double)p->alpha;
+        const double a = al * q * q;
+        d.c1 = (float)(al * q * 1.4426950408889634074);
+        d.decay = (float)exp(-2.0 * a);
+        d.a2 = (float)(2.0 * a);
+        d.two_aq = (float)(2.0 * al * q);
+        d.q2 = (float)(q * q);
+        d.rate_c = (float)((double)p->rate_weight * (-2.0 * al * q));
+        if (!isfinite(d.c1) || !isfinite(d.a2) || !isfinite(d.two_aq) || !isfinite(d.rate_c) || !(d.q2 > 0.0f))
+            return CDL_ERR_RANGE;
+        d.window = (p->window >= (int)nlev) ? 0 : p->window;
+        // e_j <= 2^(-a log2e j (j - 1)) for the levels j steps beyond the nearest one: below 2^-40 past jmax
+        double jm = ceil(0.5 + sqrt(0.25 + 40.0 * 0.69314718055994530942 / a)) + 1.0;
+        if (!(jm < 256.0)) jm = 256.0;
+        d.jmax = (int)jm;
+        d.level_prob = p->level_prob;
+    }
+    *out = d;
+    return CDL_OK;
+}
+
+namespace {
+
+inline bool bad_f32_ptr(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3u) != 0; }
+
+struct IndexRange {
+    bool is_unsigned;
+    int64_t absmax;
+};
+
+int index_range(const cdl_index_desc *d, IndexRange *r)
+{
+    if (d == nullptr) return CDL_ERR_ARG;
+    if (!(d->q > 0.0f) || !isfinite(d->q)) return CDL_ERR_RANGE;
+    if (d->hi < d->lo) return CDL_ERR_RANGE;
+    if (d->lo < 0) {
+        if (d->lo < -128 || d->hi > 127) return CDL_ERR_RANGE;
+    } else if (d->hi > 255) {
+        return CDL_ERR_RANGE;
+    }
+    r->is_unsigned = d->lo >= 0;
+    const int64_t a = d->lo < 0 ? -(int64_t)d->lo : (int64_t)d->lo;
+    const int64_t b = d->hi < 0 ? -(int64_t)d->hi : (int64_t)d->hi;
+    r->absmax = a > b ? a : b;
+    return CDL_OK;
+}
+
+inline bool overflow_risk(int64_t terms, const IndexRange &x, const IndexRange &y)
+{
+    return terms * x.absmax * y.absmax >= (int64_t)1 << 31;
+}
+
+constexpr size_t kStatusBytes = 256;
+
+}  // namespace
+}  // namespace cdl
+
+using namespace cdl;
+
+extern "C" {
+
+int cdl_version(void) { return CDL_VERSION; }
+
+const char *cdl_strerror(int status)
+{
+    switch (status) {
+        case CDL_OK: return "ok";
+        case CDL_ERR_ARG: return "invalid argument";
+        case CDL_ERR_ALIGN: return "pointer or leading dimension not aligned as required";
+        case CDL_ERR_RANGE: return "parameter out of range";
+        case CDL_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CDL_ERR_OVERFLOW_RISK: return "int32 accumulator could overflow for these sizes and index ranges";
+        case CDL_ERR_LAUNCH: return "CUDA launch or runtime call failed";
+        case CDL_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case CDL_ERR_UNSUPPORTED: return "device is not compute capability 10.x";
+        default: return "unknown status";
+    }
+}
+
+int cdl_quantize_hard(const float *x, int64_t n, const cdl_quant_params *p, void *idx_out, uint64_t *hist,
+                      void *stream)
+{
+    if (n < 0 || (n > 0 && x == nullptr)) return CDL_ERR_ARG;
+    if (bad_f32_ptr(x) || (reinterpret_cast<uintptr_t>(hist) & 7u)) return CDL_ERR_ALIGN;
+    QuantDev qd;
+    int rc = make_quant_dev(p, false, &qd);
+    if (rc != CDL_OK) return rc;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    return launch_quantize(MODE_HARD, x, nullptr, n, qd, nullptr, idx_out,
+                           reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
+                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p, float *y_soft, void *idx_out,
+                      uint64_t *hist, void *stream)
+{
+    if (n < 0 || (n > 0 && (x == nullptr || y_soft == nullptr))) return CDL_ERR_ARG;
+    if (bad_f32_ptr(x) || bad_f32_ptr(y_soft) || (reinterpret_cast<uintptr_t>(hist) & 7u)) return CDL_ERR_ALIGN;
+    QuantDev qd;
+    int rc = make_quant_dev(p, true, &qd);
+    if (rc != CDL_OK) return rc;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    return launch_quantize(MODE_SOFT, x, nullptr, n, qd, y_soft, idx_out,
+                           reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
+                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int cdl_quantize_backward(const float *x, const float *grad_out, int64_t n, const cdl_quant_params *p,
+                          float *grad_x, double *grad_q, double *grad_alpha, void *stream)
+{
+    if (n < 0 || (n > 0 && (x == nullptr || grad_out == nullptr))) return CDL_ERR_ARG;
+    if (bad_f32_ptr(x) || bad_f32_ptr(grad_out) || bad_f32_ptr(grad_x)) return CDL_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(grad_q) & 7u) || (reinterpret_cast<uintptr_t>(grad_alpha) & 7u)) return CDL_ERR_ALIGN;
+    QuantDev qd;
+    int rc = make_quant_dev(p, true, &qd);
+    if (rc != CDL_OK) return rc;
+    if (bad_f32_ptr(qd.level_prob)) return CDL_ERR_ALIGN;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    return launch_quantize(MODE_BWD, x, grad_out, n, qd, nullptr, nullptr, nullptr, false, grad_x, grad_q,
+                           grad_alpha, static_cast<cudaStream_t>(stream));
+}
+
+int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits, float *level_prob, uint64_t *n_out,
+                      void *stream)
+{
+    if (hist == nullptr || H_bits == nullptr) return CDL_ERR_ARG;
+    if (nlev < 1 || nlev > CDL_MAX_LEVELS) return CDL_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(hist) & 7u) || (reinterpret_cast<uintptr_t>(H_bits) & 7u) ||
+        (reinterpret_cast<uintptr_t>(n_out) & 7u) || bad_f32_ptr(level_prob))
+        return CDL_ERR_ALIGN;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    return launch_entropy(reinterpret_cast<const unsigned long long *>(hist), nlev, H_bits, level_prob,
+                          reinterpret_cast<unsigned long long *>(n_out), static_cast<cudaStream_t>(stream));
+}
+
+size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    switch (op) {
+        case CDL_OP_QLINEAR_FWD: return kStatusBytes;
+        case CDL_OP_QLINEAR_BWD: return kStatusBytes;
+        default: return 0;
+    }
+}
+
+int cdl_workspace_status(const void *ws, void *stream)
+{
+    if (ws == nullptr) return CDL_ERR_WORKSPACE;
+    int32_t word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, ws, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    return word == 0 ? CDL_OK : CDL_ERR_TIMEOUT;
+}
+
+int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, const void *W_idx, int64_t ldw,
+                    const cdl_index_desc *w, int32_t M, int32_t N, int32_t K, int32_t *acc_out, float *y_out,
+                    const float *bias, void *ws, size_t ws_bytes, void *stream)
+{
+    if (A_idx == nullptr || W_idx == nullptr || M <= 0 || N <= 0 || K <= 0) return CDL_ERR_ARG;
+    if (acc_out == nullptr && y_out == nullptr) return CDL_ERR_ARG;
+    if (lda < K || ldw < N) return CDL_ERR_ARG;
+    IndexRange ra, rw;
+    int rc;
+    if ((rc = index_range(a, &ra)) != CDL_OK) return rc;
+    if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+    if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+    if ((lda & 15) || (ldw & 15) || (reinterpret_cast<uintptr_t>(A_idx) & 15u) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))
+        return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(acc_out) || bad_f32_ptr(y_out) || bad_f32_ptr(bias)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_workspace_bytes(CDL_OP_QLINEAR_FWD, M, N, K))
+        return CDL_ERR_WORKSPACE;
+    if (overflow_risk(K, ra, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    const float scale = (a->q * w->q);
+    GemmOperand X{A_idx, lda, 1, ra.is_unsigned};
+    GemmOperand Y{W_idx, 1, ldw, false};
+    return launch_index_gemm(X, Y, M, N, K, acc_out, y_out, scale, bias, st);
+}
+
+int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, const void *A_idx, int64_t lda,
+                    const cdl_index_desc *a, const void *W_idx, int64_t ldw, const cdl_index_desc *w, int32_t M,
+                    int32_t N, int32_t K, int32_t *dXacc, float *dX, int32_t *dWacc, float *dW, void *ws,
+                    size_t ws_bytes, void *stream)
+{
+    const bool want_dx = dXacc != nullptr || dX != nullptr;
+    const bool want_dw = dWacc != nullptr || dW != nullptr;
+    if (G_idx == nullptr || M <= 0 || N <= 0 || K <= 0) return CDL_ERR_ARG;
+    if (!want_dx && !want_dw) return CDL_ERR_ARG;
+    if ((want_dx && W_idx == nullptr) || (want_dw && A_idx == nullptr)) return CDL_ERR_ARG;
+    if (ldg < N || (want_dw && lda < K) || (want_dx && ldw < N)) return CDL_ERR_ARG;
+    IndexRange rg, ra{false, 0}, rw{false, 0};
+    int rc;
+    if ((rc = index_range(g, &rg)) != CDL_OK) return rc;
+    if (rg.is_unsigned && g->hi > 127) return CDL_ERR_RANGE;
+    if (want_dw && (rc = index_range(a, &ra)) != CDL_OK) return rc;
+    if (want_dx) {
+        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+    }
+    if ((ldg & 15) || (reinterpret_cast<uintptr_t>(G_idx) & 15u)) return CDL_ERR_ALIGN;
+    if (want_dw && ((lda & 15) || (reinterpret_cast<uintptr_t>(A_idx) & 15u))) return CDL_ERR_ALIGN;
+    if (want_dx && ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K))
+        return CDL_ERR_WORKSPACE;
+    if (want_dx && overflow_risk(N, rg, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (want_dw && overflow_risk(M, ra, rg)) return CDL_ERR_OVERFLOW_RISK;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    if (want_dx) {
+        // dX[m,k] = sum_n G[m,n] W[k,n]
+        GemmOperand X{G_idx, ldg, 1, false};
+        GemmOperand Y{W_idx, ldw, 1, false};
+        rc = launch_index_gemm(X, Y, M, K, N, dXacc, dX, (g->q * w->q), nullptr, st);
+        if (rc != CDL_OK) return rc;
+    }
+    if (want_dw) {
+        // dW[k,n] = sum_m A[m,k] G[m,n]
+        GemmOperand X{A_idx, 1, lda, ra.is_unsigned};
+        GemmOperand Y{G_idx, 1, ldg, false};
+        rc = launch_index_gemm(X, Y, K, N, M, dWacc, dW, (g->q * a->q), nullptr, st);
+        if (rc != CDL_OK) return rc;
+    }
+    return CDL_OK;
+}
+
+}  // extern "C"

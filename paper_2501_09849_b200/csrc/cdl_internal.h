@@ -1,0 +1,51 @@
+// Internal declarations shared by the translation units of libcdl.so (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cdl.h"
+
+namespace cdl {
+
+// Quantizer parameters in the form the kernels consume; derived on the host in double
+// precision from (q, lo, hi, alpha, rate weight) and rounded once to binary32.
+struct QuantDev {
+    float q;          // step size
+    float half_q;     // q / 2 (exact)
+    float flo, fhi;   // index range as floats
+    int lo, hi, nlev;
+    float c1;         // alpha * q * log2(e): the logit of level kn+j relative to level kn is -c1 * j * (j q - 2 d)
+    float decay;      // exp(-2 alpha q^2): ratio step of the neighbour recurrence
+    float a2;         // 2 alpha q^2: dQ_d/dtheta = a2 * Var{J}
+    float two_aq;     // 2 alpha q
+    float q2;         // q^2
+    float rate_c;     // rate_weight * (-2 alpha q)
+    int window;       // 0 = whole index set, else an odd window smaller than nlev
+    int jmax;         // levels further than jmax from the nearest one carry < 2^-40 of its weight
+    const float *level_prob;  // nullptr: no rate term
+};
+
+enum QuantMode { MODE_HARD = 0, MODE_SOFT = 1, MODE_BWD = 2 };
+
+int check_device();   // CDL_OK, CDL_ERR_UNSUPPORTED or CDL_ERR_LAUNCH
+int sm_count();       // multiprocessors of the current device (0 on error)
+int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out);
+
+int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, const QuantDev &qd,
+                    float *y, void *idx, unsigned long long *hist, bool hist_accumulate,
+                    float *grad_x, double *grad_q, double *grad_alpha, cudaStream_t stream);
+int launch_entropy(const unsigned long long *hist, int nlev, double *H, float *prob,
+                   unsigned long long *n_out, cudaStream_t stream);
+
+// Plain index GEMM: C[i,j] = sum_r X(i,r) * Y(r,j) over index bytes with arbitrary strides.
+struct GemmOperand {
+    const void *ptr;
+    int64_t stride_outer;   // stride of the non-reduced dimension (i for X, j for Y)
+    int64_t stride_red;     // stride of the reduced dimension r
+    bool is_unsigned;
+};
+int launch_index_gemm(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R,
+                      int32_t *acc_out, float *f_out, float scale, const float *bias,
+                      cudaStream_t stream);
+
+}  // namespace cdl
