@@ -95,8 +95,10 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
     const float m2d = -2.0f * dh;
     const float dl2 = 2.0f * dl;
 
+    // The rate term is a covariance with L, so L may be shifted by a constant: measuring it from the
+    // nearest level's value makes the j = 0 term vanish and a flat L give exactly zero.
     float S = 1.0f, S1 = 0.0f, S2 = 0.0f, S3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
-    if (RATE) R0 = Ltab[kni - P.lo];
+    const float Lc = RATE ? Ltab[kni - P.lo] : 0.0f;
 
     if (WIN5) {
         const float w1 = __fsub_rn(__fadd_rn(q, m2d), dl2);   // (q - 2 dh) - 2 dl
@@ -122,7 +124,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                 S2 = fmaf(j2, e, S2);
                 S3 = fmaf(j2 * jf, e, S3);
                 if (RATE) {
-                    const float le = Ltab[kni - P.lo + j] * e;
+                    const float le = (Ltab[kni - P.lo + j] - Lc) * e;
                     R0 += le;
                     R1 = fmaf(jf, le, R1);
                 }
@@ -141,7 +143,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                 S2 = fmaf(j2, e, S2);
                 S3 = fmaf(j2 * jf, e, S3);
                 if (RATE) {
-                    const float le = Ltab[kni - P.lo + j] * e;
+                    const float le = (Ltab[kni - P.lo + j] - Lc) * e;
                     R0 += le;
                     R1 = fmaf(jf, le, R1);
                 }

@@ -1,0 +1,191 @@
+"""GPU parity of the index GEMMs (forward, dX, dW) against the CPU oracle: int32 accumulators bit-exact,
+float outputs equal to the accumulator times the binary32 product of the steps."""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2501_09849_b200 as cdl
+from paper_2501_09849_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    cdl.load_library()
+    return torch
+
+
+def dev(torch, a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def padded(a, ld):
+    out = np.zeros((a.shape[0], ld), dtype=a.dtype)
+    out[:, :a.shape[1]] = a
+    return out
+
+
+def ld16(n):
+    return (n + 15) // 16 * 16
+
+
+def run_fwd(torch, A, W, a, w, bias=None, want_acc=True, want_y=True):
+    M, K = A.shape
+    N = W.shape[1]
+    lda, ldw = ld16(K), ld16(N)
+    Ad, Wd = dev(torch, padded(A, lda)), dev(torch, padded(W, ldw))
+    acc = torch.full((M, N), -7, dtype=torch.int32, device="cuda") if want_acc else None
+    y = torch.full((M, N), -7.0, dtype=torch.float32, device="cuda") if want_y else None
+    nb = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_FWD, M, N, K)
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    bd = None if bias is None else dev(torch, bias)
+    cdl.cdl_qlinear_fwd(Ad, lda, a, Wd, ldw, w, M, N, K, acc, y, bd, ws, nb)
+    cdl.cdl_workspace_status(ws)
+    return (None if acc is None else acc.cpu().numpy()), (None if y is None else y.cpu().numpy())
+
+
+def run_bwd(torch, G, A, W, g, a, w, want=("dXacc", "dX", "dWacc", "dW")):
+    M, N = G.shape
+    K = A.shape[1] if A is not None else W.shape[0]
+    ldg, lda, ldw = ld16(N), ld16(K), ld16(N)
+    Gd = dev(torch, padded(G, ldg))
+    Ad = None if A is None else dev(torch, padded(A, lda))
+    Wd = None if W is None else dev(torch, padded(W, ldw))
+    out = {}
+    if "dXacc" in want:
+        out["dXacc"] = torch.full((M, K), -7, dtype=torch.int32, device="cuda")
+    if "dX" in want:
+        out["dX"] = torch.full((M, K), -7.0, dtype=torch.float32, device="cuda")
+    if "dWacc" in want:
+        out["dWacc"] = torch.full((K, N), -7, dtype=torch.int32, device="cuda")
+    if "dW" in want:
+        out["dW"] = torch.full((K, N), -7.0, dtype=torch.float32, device="cuda")
+    nb = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K)
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    cdl.cdl_qlinear_bwd(Gd, ldg, g, Ad, lda, a, Wd, ldw, w, M, N, K, out.get("dXacc"), out.get("dX"),
+                        out.get("dWacc"), out.get("dW"), ws, nb)
+    cdl.cdl_workspace_status(ws)
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def scaled(acc, qa, qb, bias=None):
+    s = f32(qa) * f32(qb)                       # product of the steps formed once in binary32
+    y = acc.astype(f32) * s                     # int32 -> binary32 (round to nearest), one binary32 multiply
+    if bias is not None:
+        y = y + bias.astype(f32)[None, :]
+    return y
+
+
+def check_all_products(torch, A, W, G, a, w, g):
+    ref_f = oracle.gemm_fwd(A, W)
+    ref_x = oracle.gemm_dx(G, W)
+    ref_w = oracle.gemm_dw(A, G)
+    for r in (ref_f, ref_x, ref_w):
+        assert np.abs(r).max() < 2 ** 31
+    acc, y = run_fwd(torch, A, W, a, w)
+    assert np.array_equal(acc.astype(np.int64), ref_f)
+    assert np.array_equal(y, scaled(ref_f, a.q, w.q))
+    out = run_bwd(torch, G, A, W, g, a, w)
+    assert np.array_equal(out["dXacc"].astype(np.int64), ref_x)
+    assert np.array_equal(out["dWacc"].astype(np.int64), ref_w)
+    assert np.array_equal(out["dX"], scaled(ref_x, g.q, w.q))
+    assert np.array_equal(out["dW"], scaled(ref_w, g.q, a.q))
+
+
+def test_tiny_layer_products_from_quantized_tensors(torch):
+    # the whole tiny layer: quantize on the GPU, multiply the GPU's own indices, compare with the oracle chain
+    case, wt, at = inputs.tiny_layer(seed=0)
+    M, K, N = case.M, case.K, case.N
+    ref_wi, _ = oracle.hard(wt, f32(case.wq.q), case.wq.lo, case.wq.hi)
+    ref_ai, _ = oracle.hard(at, f32(case.aq.q), case.aq.lo, case.aq.hi)
+    gt = inputs.normal((M, N), 1e-2, seed=0, stream=9)
+    qg = float(f32(np.abs(gt).max() / 127.0))
+    ref_gi, _ = oracle.hard(gt, f32(qg), -127, 127)
+    wi = torch.empty((K, N), dtype=torch.int8, device="cuda")
+    ai = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+    gi = torch.empty((M, N), dtype=torch.int8, device="cuda")
+    cdl.cdl_quantize_hard(dev(torch, wt), wt.size, cdl.QuantParams(case.wq.q, case.wq.lo, case.wq.hi), wi)
+    cdl.cdl_quantize_hard(dev(torch, at), at.size, cdl.QuantParams(case.aq.q, case.aq.lo, case.aq.hi), ai)
+    cdl.cdl_quantize_hard(dev(torch, gt), gt.size, cdl.QuantParams(qg, -127, 127), gi)
+    A, W, G = ai.cpu().numpy(), wi.cpu().numpy(), gi.cpu().numpy()
+    assert np.array_equal(A, ref_ai.astype(np.uint8)) and np.array_equal(W, ref_wi.astype(np.int8))
+    assert np.array_equal(G, ref_gi.astype(np.int8))
+    a, w, g = cdl.IndexDesc(case.aq.q, 0, 15), cdl.IndexDesc(case.wq.q, -7, 7), cdl.IndexDesc(qg, -127, 127)
+    check_all_products(torch, A, W, G, a, w, g)
+    bias = inputs.normal((N,), 1.0, seed=3)
+    _, y = run_fwd(torch, A, W, a, w, bias=bias, want_acc=False)
+    assert np.array_equal(y, scaled(oracle.gemm_fwd(A, W), a.q, w.q, bias))
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 16, 16), (5, 20, 7), (130, 147, 64), (257, 144, 16), (300, 520, 130),
+                                   (64, 2304, 256), (1000, 64, 1000)])
+def test_ragged_shapes_and_signedness(torch, M, K, N):
+    for a_lo, a_hi in ((0, 255), (-128, 127), (0, 15)):
+        A = inputs.uniform_indices((M, K), a_lo, a_hi, seed=M + K)
+        W = inputs.uniform_indices((K, N), -128, 127, seed=N + 1)
+        G = inputs.uniform_indices((M, N), -127, 127, seed=M + 2)
+        a, w, g = cdl.IndexDesc(0.25, a_lo, a_hi), cdl.IndexDesc(0.02, -128, 127), cdl.IndexDesc(1e-3, -127, 127)
+        check_all_products(torch, A, W, G, a, w, g)
+
+
+def test_optional_outputs_and_operands(torch):
+    M, K, N = 70, 96, 40
+    A = inputs.uniform_indices((M, K), 0, 15, seed=1)
+    W = inputs.uniform_indices((K, N), -7, 7, seed=2)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=3)
+    a, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    acc, y = run_fwd(torch, A, W, a, w, want_y=False)
+    assert y is None and np.array_equal(acc.astype(np.int64), oracle.gemm_fwd(A, W))
+    out = run_bwd(torch, G, None, W, g, None, w, want=("dX",))
+    assert np.array_equal(out["dX"], scaled(oracle.gemm_dx(G, W), g.q, w.q))
+    out = run_bwd(torch, G, A, None, g, a, None, want=("dWacc",))
+    assert np.array_equal(out["dWacc"].astype(np.int64), oracle.gemm_dw(A, G))
+
+
+def test_cifar_resnet20_conv_shape_full_compare(torch):
+    # (M, K, N) = (131072, 144, 16): operands drawn from the quantized tensors' own level histograms
+    case, wt, at = inputs.cifar_resnet20_conv()
+    M, K, N = case.M, case.K, case.N
+    wi, _ = oracle.hard(wt, f32(case.wq.q), case.wq.lo, case.wq.hi)
+    _, ah = oracle.hard(at, f32(case.aq.q), case.aq.lo, case.aq.hi)
+    A = inputs.indices_from_histogram((M, K), ah, 0, seed=case.seed, stream=3)
+    W = wi.astype(np.int8)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=case.seed, stream=4)
+    a, w, g = cdl.IndexDesc(case.aq.q, 0, 15), cdl.IndexDesc(case.wq.q, -1, 1), cdl.IndexDesc(1e-3, -127, 127)
+    check_all_products(torch, A, W, G, a, w, g)
+
+
+def test_resnet18_layer3_shape_sampled_compare(torch):
+    # (M, K, N) = (50176, 2304, 256) in the launch configuration the benchmark times.  The oracle checks
+    # whole rows of the forward / dX outputs (both M edges and rows spread over every tile row) and, for dW
+    # (which reduces over all of M), whole K x N sub-blocks spread over every tile of the output.
+    case, wt, at = inputs.resnet18_layer3_conv()
+    M, K, N = case.M, case.K, case.N
+    wi, _ = oracle.hard(wt, f32(case.wq.q), case.wq.lo, case.wq.hi)
+    _, ah = oracle.hard(at[:8], f32(case.aq.q), case.aq.lo, case.aq.hi)
+    A = inputs.indices_from_histogram((M, K), ah, 0, seed=case.seed, stream=3)
+    W = wi.astype(np.int8)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=case.seed, stream=4)
+    a, w, g = cdl.IndexDesc(case.aq.q, 0, 15), cdl.IndexDesc(case.wq.q, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    acc, y = run_fwd(torch, A, W, a, w)
+    out = run_bwd(torch, G, A, W, g, a, w)
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([np.arange(0, 3), np.arange(M - 3, M), np.arange(125, 131),
+                                     rng.integers(0, M, size=180)]))
+    ref_f = oracle.gemm_fwd(A[rows], W)
+    assert np.array_equal(acc[rows].astype(np.int64), ref_f)
+    assert np.array_equal(y[rows], scaled(ref_f, a.q, w.q))
+    ref_x = oracle.gemm_dx(G[rows], W)
+    assert np.array_equal(out["dXacc"][rows].astype(np.int64), ref_x)
+    assert np.array_equal(out["dX"][rows], scaled(ref_x, g.q, w.q))
+    ks = np.unique(np.concatenate([np.arange(0, 2), np.arange(K - 2, K), np.arange(127, 129), rng.integers(0, K, size=40)]))
+    ns = np.unique(np.concatenate([np.arange(0, 2), np.arange(N - 2, N), rng.integers(0, N, size=20)]))
+    ref_w = oracle.gemm_dw(np.ascontiguousarray(A[:, ks]), np.ascontiguousarray(G[:, ns]))
+    assert np.array_equal(out["dWacc"][np.ix_(ks, ns)].astype(np.int64), ref_w)
+    assert np.array_equal(out["dW"][np.ix_(ks, ns)], scaled(ref_w, g.q, a.q))
+    # properties that hold at any size: column sums of the forward accumulators
+    colsum = A.astype(np.int64).sum(axis=0) @ W.astype(np.int64)
+    assert np.array_equal(acc.astype(np.int64).sum(axis=0), colsum)
