@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the CDL quantized layer on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic input: quantize weights and activations
+(soft value + hard index + histogram), entropy, forward index GEMM, quantize the arriving gradient, the two
+backward index GEMMs, and the analytic quantizer backward for activations and weights.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl cdl|reference]
+
+Prints ONE JSON line (rank 0).  `value` counts the tensor elements that went through a quantizer pass per
+second of whole-step time, summed over ranks (each rank runs its own batch: weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "quantizer Gelem/s (% of HBM peak); CDL layer fwd+bwd ms and int8 TOPS"
+UNIT = "Gelem/s"
+G_STD = 1e-2                 # standard deviation of the synthetic dL/dY
+INT8_OVER_BF16 = 2.0         # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture, keyed by
+# (workload, call); None until captured for the current kernel.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cdl", choices=["cdl", "reference"])
+    ap.add_argument("--workload", default="resnet18_layer3_conv",
+                    choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        p = json.loads(f.read_text())
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def make_case(name, seed_offset=0):
+    from paper_2501_09849_b200 import inputs
+    if name == "resnet18_layer3_conv":
+        case, w, x = inputs.resnet18_layer3_conv(seed=3 + seed_offset)
+    elif name == "cifar_resnet20_conv":
+        case, w, x = inputs.cifar_resnet20_conv(seed=2 + seed_offset)
+    else:
+        case, w, x = inputs.tiny_layer(seed=0 + seed_offset)
+        case.aq.window = 5
+    return case, w, x
+
+
+def host_inputs(case, w, x, hist_x):
+    """Remaining inputs of a step: im2col index matrix (drawn from the activations' own level histogram),
+    gradient arriving at the output, gradient arriving at the quantized activations."""
+    import numpy as np
+    from paper_2501_09849_b200 import inputs
+    A = inputs.indices_from_histogram((case.M, case.K), hist_x, case.aq.lo, seed=case.seed, stream=3)
+    dY = inputs.normal((case.M, case.N), G_STD, seed=case.seed, stream=4)
+    gx = inputs.normal((x.size,), 1.0, seed=case.seed, stream=5)
+    return {"w": w.reshape(-1), "x": x.reshape(-1), "A_idx": A, "dY": dY, "gx_in": gx}
+
+
+def call_model(case, n_x):
+    """Algorithmic bytes and integer operations per call of a step (what the method must move / compute)."""
+    M, K, N = case.M, case.K, case.N
+    n_w = K * N
+    return {
+        "quantize_soft_w": {"bytes": n_w * 9, "elems": n_w},
+        "entropy_w": {"bytes": case.wq.nlev * 12, "elems": 0},
+        "quantize_soft_x": {"bytes": n_x * 9, "elems": n_x},
+        "entropy_x": {"bytes": case.aq.nlev * 12, "elems": 0},
+        "qlinear_fwd": {"bytes": M * K + K * N + 4 * M * N, "ops": 2 * M * K * N, "elems": 0},
+        "quantize_hard_g": {"bytes": M * N * 5, "elems": M * N},
+        "qlinear_bwd_dx": {"bytes": M * N + K * N + 4 * M * K, "ops": 2 * M * K * N, "elems": 0},
+        "qlinear_bwd_dw": {"bytes": M * K + M * N + 4 * K * N, "ops": 2 * M * K * N, "elems": 0},
+        "quantize_backward_x": {"bytes": n_x * 12, "elems": n_x},
+        "quantize_backward_w": {"bytes": n_w * 12, "elems": n_w},
+    }
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [c.strip() for c in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_step_sample(case, host, n_x_sample=1 << 24, rows=1 << 16):
+    """Times the CPU oracle, as it stands, on a bounded sample of one step and scales every part to the full
+    step by the units it processed.  Returns (estimated seconds of a full step, description, threads)."""
+    import numpy as np
+    import oracle
+    f32 = np.float32
+    wq, aq = case.wq, case.aq
+    n_x = host["x"].size
+    ns = min(n_x, n_x_sample)
+    xs, gs = host["x"][:ns], host["gx_in"][:ns]
+    w = host["w"]
+    t_total = 0.0
+
+    def timed(fn, scale):
+        nonlocal t_total
+        t0 = time.perf_counter()
+        r = fn()
+        t_total += (time.perf_counter() - t0) * scale
+        return r
+
+    sx = n_x / ns
+    timed(lambda: oracle.soft(w, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window), 1.0)
+    _, hw = timed(lambda: oracle.hard(w, f32(wq.q), wq.lo, wq.hi), 1.0)
+    _, pw, _ = timed(lambda: oracle.entropy(hw), 1.0)
+    timed(lambda: oracle.soft(xs, f32(aq.q), aq.lo, aq.hi, f32(aq.alpha), aq.window), sx)
+    _, hx = timed(lambda: oracle.hard(xs, f32(aq.q), aq.lo, aq.hi), sx)
+    _, px, _ = timed(lambda: oracle.entropy(hx), 1.0)
+    r = min(rows, case.M)
+    sm = case.M / r
+    A, W8 = host["A_idx"][:r], oracle.hard(w, f32(wq.q), wq.lo, wq.hi)[0].reshape(case.K, case.N).astype(np.int8)
+    timed(lambda: oracle.gemm_fwd(A, W8), sm)
+    q_g = 4.0 * G_STD / 127.0
+    gi, _ = timed(lambda: oracle.hard(host["dY"][:r], f32(q_g), -127, 127), sm)
+    G8 = gi.astype(np.int8)
+    timed(lambda: oracle.gemm_dx(G8, W8), sm)
+    dW = timed(lambda: oracle.gemm_dw(A, G8), sm)
+    timed(lambda: oracle.backward(xs, gs, f32(aq.q), aq.lo, aq.hi, f32(aq.alpha), aq.window, f32(aq.rate_weight), px), sx)
+    gw = (dW.astype(np.float64) * q_g * aq.q).astype(f32).reshape(-1)
+    timed(lambda: oracle.backward(w, gw, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window, f32(wq.rate_weight), pw), 1.0)
+    desc = (f"oracle on {ns} of {n_x} activations (quantize, backward), all {w.size} weights, "
+            f"{r} of {case.M} GEMM rows (fwd, dX, dW); each part scaled to the full step")
+    return t_total, desc, oracle.threads()
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle on a bounded sample of the same workload (rank 0 only)."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    oracle.build()
+    case, w, x = make_case(args.workload)
+    f32 = np.float32
+    _, hist_x = oracle.hard(x.reshape(-1)[: 1 << 20], f32(case.aq.q), case.aq.lo, case.aq.hi)
+    host = host_inputs(case, w, x, hist_x)
+    quant_elems = 2 * (w.size + x.size) + case.M * case.N
+    for _ in range(max(args.warmup, 0)):
+        oracle_step_sample(case, host, n_x_sample=1 << 14, rows=2)
+    ts = []
+    for _ in range(args.steps):
+        t, desc, thr = oracle_step_sample(case, host, n_x_sample=1 << 22, rows=2048)
+        ts.append(t)
+    t_step = sum(ts) / len(ts)
+    value = quant_elems / t_step / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "M": case.M, "K": case.K, "N": case.N},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2501_09849_b200 as cdl
+    from paper_2501_09849_b200 import build as cdl_build
+    from paper_2501_09849_b200.layer import CALLS, CdlLayerStep
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if local_rank == 0:
+        cdl_build.build()
+    if world > 1:
+        dist.barrier()
+    cdl.load_library()
+
+    # ---- inputs: seeded, host-generated, one independent batch per rank (weak scaling)
+    case, w, x = make_case(args.workload, seed_offset=100 * rank)
+    M, K, N, n_x = case.M, case.K, case.N, x.size
+    q_g = float(np.float32(4.0 * G_STD / 127.0))
+    step = CdlLayerStep(torch, M, K, N, n_x, case.wq, case.aq, q_g)
+    xd = torch.from_numpy(x.reshape(-1)).cuda()
+    hist = torch.zeros(case.aq.nlev, dtype=torch.int64, device="cuda")
+    cdl.cdl_quantize_hard(xd, n_x, cdl.QuantParams(case.aq.q, case.aq.lo, case.aq.hi), None, hist)
+    host = host_inputs(case, w, x, hist.cpu().numpy().view(np.uint64))
+    pinned = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in host.items()}
+    dev_in = step.input_tensors()
+    for k, t in dev_in.items():
+        t.copy_(pinned[k].view(t.shape), non_blocking=True)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def exchange():
+        # data-parallel exchange of a step: the weight-side results are sums over the global batch
+        if world > 1:
+            dist.all_reduce(step.dW)
+            dist.all_reduce(step.hist_x)
+            dist.all_reduce(step.scalars)
+
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+        exchange()
+    torch.cuda.synchronize()
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(args.steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for it in range(args.steps):
+        ev = iter(events[it])
+        step.run(mark=lambda name: next(ev).record(stream))
+        exchange()
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_start.elapsed_time(t_end)
+    per_call_ms = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(args.steps)) / args.steps
+                   for i, name in enumerate(CALLS)}
+    status = cdl.cdl_workspace_status(step.ws, check=False)
+
+    # ---- end to end: host buffers in, results out, every step
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+    out_host = {"scalars": torch.empty(6, dtype=torch.float64).pin_memory(),
+                "dw": torch.empty(step.n_w, dtype=torch.float32).pin_memory()}
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+    e_steps = max(3, min(args.steps, 10))
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e_steps):
+        for k, t in dev_in.items():
+            t.copy_(pinned[k].view(t.shape), non_blocking=True)
+        step.run()
+        exchange()
+        out_host["scalars"].copy_(step.scalars, non_blocking=True)
+        out_host["dw"].copy_(step.dw, non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e_steps
+
+    ms_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_step, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        pk, pk_kind = peaks()
+        model = call_model(case, n_x)
+        quant_elems = sum(m["elems"] for m in model.values())
+        value = world * quant_elems / (ms_step * 1e-3) / 1e9
+        e2e_value = world * quant_elems / (e2e_ms * 1e-3) / 1e9
+        hbm = float(pk["hbm_gbs"])
+        int8_tops = float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])) * INT8_OVER_BF16
+        kernels = {}
+        for name in CALLS:
+            m, ms = model[name], per_call_ms[name]
+            k = {"ms": round(ms, 5), "GBps": round(m["bytes"] / (ms * 1e-3) / 1e9, 1)}
+            if m["elems"]:
+                k["Gelem_per_s"] = round(m["elems"] / (ms * 1e-3) / 1e9, 2)
+                k["hbm_frac_measured"] = round(k["GBps"] / hbm, 4)
+                k["hbm_frac_8TBps"] = round(k["GBps"] / 8000.0, 4)
+            if "ops" in m:
+                k["int8_TOPS"] = round(m["ops"] / (ms * 1e-3) / 1e12, 1)
+                t_tensor, t_hbm = m["ops"] / (int8_tops * 1e12), m["bytes"] / (hbm * 1e9)
+                k["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
+                k["roofline_frac"] = round(max(t_tensor, t_hbm) / (ms * 1e-3), 4)
+            kernels[name] = k
+        dom = max(CALLS, key=lambda c: per_call_ms[c])
+        dm, dms = model[dom], per_call_ms[dom]
+        if "ops" in dm and dm["ops"] / (int8_tops * 1e12) >= dm["bytes"] / (hbm * 1e9):
+            roof = {"kernel": dom, "bound": "tensor", "achieved": dm["ops"] / (dms * 1e-3) / 1e12, "peak": int8_tops,
+                    "unit": "TFLOP/s", "peak_source": f"{pk_kind} sustained bf16 x {INT8_OVER_BF16:g} (nominal int8:bf16)"}
+        else:
+            roof = {"kernel": dom, "bound": "hbm", "achieved": dm["bytes"] / (dms * 1e-3) / 1e9, "peak": hbm,
+                    "unit": "GB/s", "peak_source": f"{pk_kind} copy bandwidth"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.workload, dom))
+        gemm_ms = sum(per_call_ms[c] for c in ("qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_dw"))
+        quant_ms = sum(per_call_ms[c] for c in CALLS if model[c]["elems"])
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32+s8", "data": "synthetic",
+            "config": {"workload": args.workload, "M": M, "K": K, "N": N, "activation_elems": n_x,
+                       "weight_levels": case.wq.nlev, "activation_levels": case.aq.nlev,
+                       "alpha": case.wq.alpha, "rate_weight": case.wq.rate_weight, "window_x": case.aq.window,
+                       "l2": "per-step working set is several times the 126 MB L2 (inputs larger than L2)",
+                       "parallelism": f"replicas x{world}, all-reduce of dW / histogram / scalars" if world > 1 else "single GPU"},
+            "layer_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": 6.0 * M * K * N / (gemm_ms * 1e-3) / 1e12,
+            "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": quant_elems / (quant_ms * 1e-3) / 1e9,
+            "quantizer_hbm_frac_measured": sum(model[c]["bytes"] for c in CALLS if model[c]["elems"]) / (quant_ms * 1e-3) / 1e9 / hbm,
+            "kernels": kernels, "roofline": roof, "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e_steps},
+            "gpu_launches": args.steps * len(CALLS), "device_status": status,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            t_cpu, desc, thr = oracle_step_sample(case, host)
+            line["cpu_baseline"] = {"value": quant_elems / t_cpu / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle",
+                                    "sample": desc, "ms_per_step_estimate": t_cpu * 1e3}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,97 @@
+"""One training step of a CDL quantized layer as a fixed sequence of C-ABI calls (Algorithm 1, the
+per-layer part of its forward and backward passes).  This module only owns device buffers and issues the
+calls in order on one stream; every number is produced by the kernels behind the ABI.
+
+Step (names follow the paper: w weights, x activations, q / s step sizes, alpha / beta CPMF parameters):
+   1  quantize w        -> soft value Q_d(w), index W_idx, level histogram          cdl_quantize_soft
+   2  entropy of w      -> H(w) in bits, level probabilities                        cdl_index_entropy
+   3  quantize x        -> Q_d(x), index X_idx, histogram (window of 5)             cdl_quantize_soft
+   4  entropy of x                                                                   cdl_index_entropy
+   5  forward product   Y = (s q) A_idx W_idx   (A_idx: the im2col index matrix)    cdl_qlinear_fwd
+   6  quantize dL/dY    -> G_idx (hard index, 255 levels, caller-chosen step)       cdl_quantize_hard
+   7  backward products dA = (q_g q) G_idx W_idx^T, dW = (q_g s) A_idx^T G_idx      cdl_qlinear_bwd (two calls)
+   8  quantizer backward on x: dL/dx, dL/ds, dL/dbeta (+ gamma * rate term)         cdl_quantize_backward
+   9  quantizer backward on w with grad_out = dW: dL/dw, dL/dq, dL/dalpha (+ lambda * rate term)
+The im2col gather / scatter between the activation tensor and the GEMM operand is outside the library:
+A_idx and the gradient arriving at the quantized activations are inputs of the step.
+"""
+from __future__ import annotations
+
+from . import api as cdl
+
+CALLS = ("quantize_soft_w", "entropy_w", "quantize_soft_x", "entropy_x", "qlinear_fwd", "quantize_hard_g",
+         "qlinear_bwd_dx", "qlinear_bwd_dw", "quantize_backward_x", "quantize_backward_w")
+
+
+class CdlLayerStep:
+    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda"):
+        """wq / xq: objects with q, lo, hi, alpha, rate_weight, window (weights / activations); n_x: number of
+        activation elements quantized per step (the layer's input tensor, before im2col)."""
+        self.torch = torch
+        self.M, self.K, self.N, self.n_x, self.n_w = M, K, N, n_x, K * N
+        self.wq, self.xq, self.q_g = wq, xq, float(q_g)
+        t, dev = torch, device
+        f32, i8, u8 = t.float32, t.int8, t.uint8
+
+        def idt(lo):
+            return i8 if lo < 0 else u8
+        # inputs of a step
+        self.w = t.empty(self.n_w, dtype=f32, device=dev)
+        self.x = t.empty(n_x, dtype=f32, device=dev)
+        self.A_idx = t.empty((M, K), dtype=idt(xq.lo), device=dev)
+        self.dY = t.empty((M, N), dtype=f32, device=dev)
+        self.gx_in = t.empty(n_x, dtype=f32, device=dev)         # dL/dQ(x) after the scatter back from dA
+        # outputs
+        self.w_soft = t.empty(self.n_w, dtype=f32, device=dev)
+        self.W_idx = t.empty((K, N), dtype=idt(wq.lo), device=dev)
+        self.x_soft = t.empty(n_x, dtype=f32, device=dev)
+        self.X_idx = t.empty(n_x, dtype=idt(xq.lo), device=dev)
+        self.hist_w = t.zeros(wq.hi - wq.lo + 1, dtype=t.int64, device=dev)
+        self.hist_x = t.zeros(xq.hi - xq.lo + 1, dtype=t.int64, device=dev)
+        self.prob_w = t.empty(wq.hi - wq.lo + 1, dtype=f32, device=dev)
+        self.prob_x = t.empty(xq.hi - xq.lo + 1, dtype=f32, device=dev)
+        self.Y = t.empty((M, N), dtype=f32, device=dev)
+        self.G_idx = t.empty((M, N), dtype=i8, device=dev)
+        self.dA = t.empty((M, K), dtype=f32, device=dev)
+        self.dW = t.empty((K, N), dtype=f32, device=dev)
+        self.dx = t.empty(n_x, dtype=f32, device=dev)
+        self.dw = t.empty(self.n_w, dtype=f32, device=dev)
+        # scalars: H(w), H(x) | dq, dalpha, ds, dbeta
+        self.scalars = t.zeros(6, dtype=t.float64, device=dev)
+        self.ws_bytes = max(cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_FWD, M, N, K),
+                            cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K))
+        self.ws = t.empty(self.ws_bytes, dtype=u8, device=dev)
+        self.Pw = cdl.QuantParams(wq.q, wq.lo, wq.hi, wq.alpha, wq.rate_weight, None, wq.window)
+        self.Px = cdl.QuantParams(xq.q, xq.lo, xq.hi, xq.alpha, xq.rate_weight, None, xq.window)
+        self.Pw_b = cdl.QuantParams(wq.q, wq.lo, wq.hi, wq.alpha, wq.rate_weight, self.prob_w, wq.window)
+        self.Px_b = cdl.QuantParams(xq.q, xq.lo, xq.hi, xq.alpha, xq.rate_weight, self.prob_x, xq.window)
+        self.Pg = cdl.QuantParams(self.q_g, -127, 127)
+        self.da = cdl.IndexDesc(xq.q, xq.lo, xq.hi)
+        self.dw_desc = cdl.IndexDesc(wq.q, wq.lo, wq.hi)
+        self.dg = cdl.IndexDesc(self.q_g, -127, 127)
+
+    def input_tensors(self):
+        return {"w": self.w, "x": self.x, "A_idx": self.A_idx, "dY": self.dY, "gx_in": self.gx_in}
+
+    def run(self, stream=None, mark=None):
+        """Enqueue one step.  mark(name), if given, is called before each ABI call and once at the end
+        (used to drop CUDA events between the calls)."""
+        s = self.scalars
+        M, K, N = self.M, self.K, self.N
+        nlw, nlx = self.Pw.nlev, self.Px.nlev
+        m = mark if mark is not None else (lambda name: None)
+        m(CALLS[0]); cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, stream)
+        m(CALLS[1]); cdl.cdl_index_entropy(self.hist_w, nlw, s[0:1], self.prob_w, None, stream)
+        m(CALLS[2]); cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, stream)
+        m(CALLS[3]); cdl.cdl_index_entropy(self.hist_x, nlx, s[1:2], self.prob_x, None, stream)
+        m(CALLS[4]); cdl.cdl_qlinear_fwd(self.A_idx, K, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
+                                         None, self.ws, self.ws_bytes, stream)
+        m(CALLS[5]); cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, stream)
+        # the two backward products are issued as two calls so that each can be timed on its own
+        m(CALLS[6]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
+                                         M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
+        m(CALLS[7]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, K, self.da, None, N, None,
+                                         M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
+        m(CALLS[8]); cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, s[4:5], s[5:6], stream)
+        m(CALLS[9]); cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, s[2:3], s[3:4], stream)
+        m("end")
