@@ -208,8 +208,11 @@ size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
 {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
     switch (op) {
-        case CDL_OP_QLINEAR_FWD: return kStatusBytes;
-        case CDL_OP_QLINEAR_BWD: return kStatusBytes;
+        case CDL_OP_QLINEAR_FWD: return kStatusBytes + tc_gemm_scratch_bytes(M, N, K);
+        case CDL_OP_QLINEAR_BWD: {
+            const size_t dx = tc_gemm_scratch_bytes(M, K, N), dw = tc_gemm_scratch_bytes(K, N, M);
+            return kStatusBytes + (dx > dw ? dx : dw);
+        }
         default: return 0;
     }
 }
@@ -254,7 +257,8 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, con
     const float scale = (a->q * w->q);
     GemmOperand X{A_idx, lda, 1, ra.is_unsigned};
     GemmOperand Y{W_idx, 1, ldw, false};
-    return launch_index_gemm(X, Y, M, N, K, acc_out, y_out, scale, bias, st);
+    return launch_index_gemm_tc(X, Y, M, N, K, acc_out, y_out, scale, bias, static_cast<char *>(ws) + kStatusBytes,
+                                static_cast<int *>(ws), st);
 }
 
 int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, const void *A_idx, int64_t lda,
@@ -295,14 +299,16 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
         // dX[m,k] = sum_n G[m,n] W[k,n]
         GemmOperand X{G_idx, ldg, 1, false};
         GemmOperand Y{W_idx, ldw, 1, false};
-        rc = launch_index_gemm(X, Y, M, K, N, dXacc, dX, (g->q * w->q), nullptr, st);
+        rc = launch_index_gemm_tc(X, Y, M, K, N, dXacc, dX, (g->q * w->q), nullptr,
+                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st);
         if (rc != CDL_OK) return rc;
     }
     if (want_dw) {
         // dW[k,n] = sum_m A[m,k] G[m,n]
         GemmOperand X{A_idx, 1, lda, ra.is_unsigned};
         GemmOperand Y{G_idx, 1, ldg, false};
-        rc = launch_index_gemm(X, Y, K, N, M, dWacc, dW, (g->q * a->q), nullptr, st);
+        rc = launch_index_gemm_tc(X, Y, K, N, M, dWacc, dW, (g->q * a->q), nullptr,
+                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st);
         if (rc != CDL_OK) return rc;
     }
     return CDL_OK;

@@ -1,0 +1,518 @@
+// Index GEMM on the 5th-generation tensor cores of sm_100a: D[i,j] = sum_r X(i,r) Y(r,j) over int8/uint8
+// index bytes, exact int32 accumulation (tcgen05.mma kind::i8, accumulator in TMEM), operands staged in
+// shared memory by TMA (no multicast), float / int32 epilogue read back with tcgen05.ld.
+//
+// One kernel serves the three layer products; they differ only in which dimension of each stored matrix is
+// contiguous, which is expressed by the "major" of the shared-memory operand descriptor:
+//   forward  Y  = A W      X = A [M,K] (r = k contiguous: K-major)   Y-op = W [K,N] (j contiguous: MN-major)
+//   dX       dA = G W^T    X = G [M,N] (r = n contiguous: K-major)   Y-op = W [K,N] (r = n contiguous: K-major)
+//   dW       dW = A^T G    X = A [M,K] (i = k contiguous: MN-major)  Y-op = G [M,N] (j contiguous: MN-major)
+//
+// Tiling: 128 x TN output tile per work unit (TN in {16..256}), 128 bytes of the reduced dimension per
+// pipeline stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is
+// [rows][128 bytes] with the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or
+// columns outside the matrix are zero-filled by TMA, which makes ragged edges and R tails exact.
+// Warp roles (192 threads): warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2-5 run the
+// epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
+// Work units are (tile, split of the reduced dimension); with more than one split the epilogue adds its
+// partial sums into an int32 buffer with red.global.add (integer, so the result does not depend on order).
+// Every wait is bounded: on expiry the kernel records CDL_ERR_TIMEOUT in the status word and winds down.
+#include <cuda.h>
+
+#include "cdl_internal.h"
+
+namespace cdl {
+namespace {
+
+constexpr int kThreadsTC = 192;
+constexpr int kStages = 4;
+constexpr int TM = 128;                 // output rows per tile = UMMA M
+constexpr int BR = 128;                 // bytes (= elements) of the reduced dimension per stage
+constexpr int kABytes = TM * BR;        // 16 KB
+constexpr int kBBytesMax = 256 * BR;    // 32 KB
+constexpr int kStageBytes = kABytes + kBBytesMax;
+// The whole 227 KB opt-in window is requested (stages need 193 KB): operand descriptors then address
+// allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
+constexpr int kSmemBytes = 232448 - 1024;
+constexpr int kPlanSMs = 148;           // B200: splits are planned for this count so that workspace sizes are fixed
+constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s
+
+struct TcParams {
+    int I, J, R;            // output rows, output columns, reduced extent
+    int TN;                 // output columns per tile (multiple of 16, <= 256)
+    int tiles_i, tiles_j;   // tile grid
+    int splits;             // splits of the reduced dimension
+    int rblocks;            // ceil(R / BR)
+    int a_mn_major, b_mn_major;
+    unsigned int idesc;
+    int32_t *acc_out;       // int32 output or accumulation buffer (required when splits > 1)
+    float *f_out;           // float output (written by the epilogue only when splits == 1)
+    float scale;
+    const float *bias;
+    int *status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the barrier did not complete within kWaitNs or another thread already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (int fast = 0; fast < 64; ++fast)
+        if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag != 0) return false;
+        if (global_ns() - t0 > kWaitNs) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor (sm_100 format): start address, leading / stride byte offsets in 16-byte
+// units, version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fffu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+__global__ void __launch_bounds__(kThreadsTC, 1)
+index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const TcParams P)
+{
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ __align__(8) unsigned long long bars[2 * kStages + 4];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    volatile int *abort_flag = &abort_s;
+
+    auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };
+    auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * kStages + b]); };
+    auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * kStages + 2 + b]); };
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int units = P.tiles_i * P.tiles_j * P.splits;
+    const int b_blocks = (P.TN + 127) / 128;                              // 128-wide blocks of an MN-major B tile
+    const uint32_t b_bytes = P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR);
+    const uint32_t stage_tx = (uint32_t)kABytes + b_bytes;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int u = blockIdx.x; u < units && !failed; u += gridDim.x) {
+                const int split = u % P.splits;
+                const int tile = u / P.splits;
+                const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
+                const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
+                const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
+                for (int rb = rb0; rb < rb1; ++rb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                        failed = true;
+                        break;
+                    }
+                    const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
+                    const uint32_t sb = sa + kABytes;
+                    mbar_expect_tx(full_bar(s), stage_tx);
+                    if (P.a_mn_major) tma_load_2d(sa, &map_a, ti * TM, rb * BR, full_bar(s));   // {i (inner), r}
+                    else tma_load_2d(sa, &map_a, rb * BR, ti * TM, full_bar(s));                 // {r (inner), i}
+                    if (P.b_mn_major) {
+                        for (int bb = 0; bb < b_blocks; ++bb)
+                            tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, tj * P.TN + bb * 128, rb * BR, full_bar(s));
+                    } else {
+                        tma_load_2d(sb, &map_b, rb * BR, tj * P.TN, full_bar(s));
+                    }
+                }
+            }
+            if (failed) {
+                abort_s = 1;
+                atomicExch(P.status, CDL_ERR_TIMEOUT);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0, tcount = 0;
+            for (int u = blockIdx.x; u < units && !failed; u += gridDim.x, ++tcount) {
+                const int split = u % P.splits;
+                const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
+                const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
+                const int buf = tcount & 1;
+                const uint32_t tph = (tcount >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag)) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256u;
+                for (int rb = rb0; rb < rb1; ++rb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+                        failed = true;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
+                    const uint32_t sb = sa + kABytes;
+                    // K-major: rows are 128-byte lines, 8-row groups 1024 bytes apart, 32 bytes per MMA along r.
+                    // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of
+                    // the non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
+                    const uint64_t adesc = P.a_mn_major ? make_desc(sa, 128 * BR, 1024) : make_desc(sa, 16, 1024);
+                    const uint64_t bdesc = P.b_mn_major ? make_desc(sb, 128 * BR, 1024) : make_desc(sb, 16, 1024);
+                    const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
+                    const uint32_t b_step = P.b_mn_major ? (4096u >> 4) : (32u >> 4);
+#pragma unroll
+                    for (int k = 0; k < BR / 32; ++k)
+                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc,
+                                  (rb > rb0 || k > 0) ? 1u : 0u);
+                    tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
+                }
+                if (!failed) tc_commit(tfull_bar(buf));  // accumulator complete
+            }
+            if (failed) {
+                abort_s = 1;
+                atomicExch(P.status, CDL_ERR_TIMEOUT);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps 2..5
+        const int quarter = warp & 3;               // TMEM lanes this warp may read: 32 * (warp % 4) ..
+        uint32_t tcount = 0;
+        for (int u = blockIdx.x; u < units && !failed; u += gridDim.x, ++tcount) {
+            const int tile = u / P.splits;
+            const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
+            const int buf = tcount & 1;
+            const uint32_t tph = (tcount >> 1) & 1u;
+            if (!mbar_wait(tfull_bar(buf), tph, abort_flag)) {
+                failed = true;
+                break;
+            }
+            tc_fence_after();
+            const int row = ti * TM + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
+            const bool vec_ok = (P.J & 3) == 0;
+            for (int c0 = 0; c0 < P.TN; c0 += 32) {
+                uint32_t v[32];
+                tc_ld32(taddr + (uint32_t)c0, v);
+                tc_wait_ld();
+                const int col0 = tj * P.TN + c0;
+                if (row < P.I && col0 < P.J) {
+                    const long long off = (long long)row * P.J + col0;
+                    const int ncol = min(min(32, P.TN - c0), P.J - col0);
+                    if (P.splits > 1) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c < ncol)
+                                asm volatile("red.global.add.s32 [%0], %1;" ::"l"(P.acc_out + off + c), "r"(v[c]) : "memory");
+                    } else {
+                        if (P.acc_out != nullptr) {
+                            if (vec_ok && ncol == 32) {
+#pragma unroll
+                                for (int c = 0; c < 32; c += 4)
+                                    *reinterpret_cast<int4 *>(P.acc_out + off + c) =
+                                        make_int4((int)v[c], (int)v[c + 1], (int)v[c + 2], (int)v[c + 3]);
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (c < ncol) P.acc_out[off + c] = (int)v[c];
+                            }
+                        }
+                        if (P.f_out != nullptr) {
+                            float f[32];
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) f[c] = __fmul_rn((float)(int)v[c], P.scale);
+                            if (P.bias != nullptr) {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (c < ncol) f[c] = __fadd_rn(f[c], P.bias[col0 + c]);
+                            }
+                            if (vec_ok && ncol == 32) {
+#pragma unroll
+                                for (int c = 0; c < 32; c += 4)
+                                    *reinterpret_cast<float4 *>(P.f_out + off + c) = make_float4(f[c], f[c + 1], f[c + 2], f[c + 3]);
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (c < ncol) P.f_out[off + c] = f[c];
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+        }
+        if (failed && lane == 0) {
+            abort_s = 1;
+            atomicExch(P.status, CDL_ERR_TIMEOUT);
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// float output of a split run: f = (float)acc * scale (+ bias[j])
+__global__ void scale_acc_kernel(const int32_t *__restrict__ acc, float *__restrict__ f, long long n, int J, float scale,
+                                 const float *__restrict__ bias)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float v = __fmul_rn((float)acc[i], scale);
+        if (bias != nullptr) v = __fadd_rn(v, bias[i % J]);
+        f[i] = v;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2D byte tensor [outer][inner] with row pitch `pitch` bytes; box = {128 bytes, box_rows}, 128-byte swizzle.
+bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t pitch, uint32_t box_rows)
+{
+    EncodeTiledFn fn = get_encode();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {pitch};
+    const cuuint32_t box[2] = {128u, box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace {
+// Split of the reduced dimension: only when the tiles alone cannot occupy half of the device.
+void plan(int I, int J, int R, int *TN_out, int *splits_out)
+{
+    int TN = 256;
+    while (TN > 16 && TN / 2 >= J) TN /= 2;
+    const long long tiles = (long long)((I + TM - 1) / TM) * ((J + TN - 1) / TN);
+    const int rblocks = (R + BR - 1) / BR;
+    int splits = 1;
+    if (tiles * 2 <= kPlanSMs) {
+        splits = (int)(kPlanSMs / tiles);
+        const int max_splits = (rblocks + 3) / 4;      // keep at least four stages of work per unit
+        if (splits > max_splits) splits = max_splits;
+        if (splits < 1) splits = 1;
+    }
+    *TN_out = TN;
+    *splits_out = splits;
+}
+}  // namespace
+
+// Scratch bytes the product needs when no int32 output is passed: the int32 accumulation buffer of a split run.
+size_t tc_gemm_scratch_bytes(int I, int J, int R)
+{
+    int TN, splits;
+    plan(I, J, R, &TN, &splits);
+    if (splits <= 1) return 0;
+    return ((size_t)I * (size_t)J * sizeof(int32_t) + 255u) & ~(size_t)255u;
+}
+
+// X: the operand whose non-reduced dimension indexes output rows; Y: output columns.  An operand is MN-major
+// when its non-reduced dimension is the contiguous one (stride_outer == 1).  scratch: tc_gemm_scratch_bytes(I, J, R)
+// bytes, used only when the reduced dimension is split and no int32 output was requested.
+int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
+                         float *f_out, float scale, const float *bias, void *scratch, int *status,
+                         cudaStream_t stream)
+{
+    const bool a_mn = X.stride_outer == 1 && X.stride_red != 1;
+    const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
+    TcParams P;
+    P.I = I;
+    P.J = J;
+    P.R = R;
+    int TN, splits;
+    plan(I, J, R, &TN, &splits);
+    P.TN = TN;
+    P.tiles_i = (I + TM - 1) / TM;
+    P.tiles_j = (J + TN - 1) / TN;
+    P.rblocks = (R + BR - 1) / BR;
+    const int sms = sm_count();
+    if (sms <= 0) return CDL_ERR_LAUNCH;
+    const long long tiles = (long long)P.tiles_i * P.tiles_j;
+    if (tiles > 0x3fffffff) return CDL_ERR_ARG;
+    P.splits = splits;
+    P.a_mn_major = a_mn ? 1 : 0;
+    P.b_mn_major = b_mn ? 1 : 0;
+    P.idesc = (2u << 4) | ((X.is_unsigned ? 0u : 1u) << 7) | ((Y.is_unsigned ? 0u : 1u) << 10) |
+              ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+    P.scale = scale;
+    P.bias = bias;
+    P.status = status;
+    P.f_out = f_out;
+    P.acc_out = acc_out;
+    const long long n_out = (long long)I * J;
+    if (splits > 1) {
+        if (P.acc_out == nullptr) P.acc_out = static_cast<int32_t *>(scratch);
+        if (P.acc_out == nullptr) return CDL_ERR_WORKSPACE;
+        if (cudaMemsetAsync(P.acc_out, 0, (size_t)n_out * sizeof(int32_t), stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+    }
+
+    CUtensorMap map_a, map_b;
+    bool ok;
+    // K-major operand: stored [outer][r], r contiguous -> inner = r.  MN-major: stored [r][outer] -> inner = outer.
+    if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
+    else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
+    if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
+    else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, (uint32_t)TN);
+    if (!ok) return CDL_ERR_LAUNCH;
+
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(index_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+        attr_set[dev] = true;
+    }
+    const long long units = tiles * splits;
+    const int grid = (int)(units < sms ? units : sms);
+    index_gemm_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, P);
+    if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
+    if (splits > 1 && f_out != nullptr) {
+        const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
+        scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias);
+        if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
+    }
+    return CDL_OK;
+}
+
+}  // namespace cdl

@@ -37,15 +37,18 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
 int launch_entropy(const unsigned long long *hist, int nlev, double *H, float *prob,
                    unsigned long long *n_out, cudaStream_t stream);
 
-// Plain index GEMM: C[i,j] = sum_r X(i,r) * Y(r,j) over index bytes with arbitrary strides.
+// Operand of an index GEMM D[i,j] = sum_r X(i,r) * Y(r,j): index bytes with arbitrary strides.
 struct GemmOperand {
     const void *ptr;
     int64_t stride_outer;   // stride of the non-reduced dimension (i for X, j for Y)
     int64_t stride_red;     // stride of the reduced dimension r
     bool is_unsigned;
 };
-int launch_index_gemm(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R,
-                      int32_t *acc_out, float *f_out, float scale, const float *bias,
-                      cudaStream_t stream);
+
+// Tensor-core index GEMM (TMA + tcgen05 + TMEM); operands need 16-byte aligned bases and pitches.
+size_t tc_gemm_scratch_bytes(int I, int J, int R);
+int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
+                         float *f_out, float scale, const float *bias, void *scratch, int *status,
+                         cudaStream_t stream);
 
 }  // namespace cdl
