@@ -11,7 +11,8 @@
  * Conventions common to every entry point
  *  - Pointers marked [dev] are device memory owned by the caller; [host] are
  *    host memory read during the call only.  The library allocates no device
- *    memory, keeps no state between calls and never synchronises the device
+ *    memory, keeps no state between calls (the built-in scratch of
+ *    cdl_qlinear_bwd_dw_noalloc excepted) and never synchronises the device
  *    (cdl_workspace_status excepted): work is enqueued on `stream` (a
  *    cudaStream_t passed as void*; NULL is the legacy default stream) and
  *    outputs are valid once the stream reaches it.
@@ -47,7 +48,8 @@ typedef enum cdl_status {
     CDL_ERR_OVERFLOW_RISK = -5, /* an int32 accumulator could overflow for these sizes and index ranges */
     CDL_ERR_LAUNCH = -6,        /* the CUDA runtime refused a launch or a driver call */
     CDL_ERR_TIMEOUT = -7,       /* a bounded device-side wait expired (reported by cdl_workspace_status) */
-    CDL_ERR_UNSUPPORTED = -8    /* the current device is not compute capability 10.x */
+    CDL_ERR_UNSUPPORTED = -8,   /* the current device is not compute capability 10.x */
+    CDL_ERR_TOO_LARGE = -9      /* problem exceeds the built-in scratch of cdl_qlinear_bwd_dw_noalloc */
 } cdl_status;
 
 /* Flags of cdl_quant_params.flags */
@@ -179,6 +181,36 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
                     int32_t M, int32_t N, int32_t K,
                     int32_t *dXacc, float *dX, int32_t *dWacc, float *dW,
                     void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Weight-gradient product for callers that cannot allocate device memory.  (The paper has no counterpart
+ * of this entry point; it is a packaging variant of the dW half of cdl_qlinear_bwd.)
+ *
+ * Who needs it: code that runs where a cudaMalloc is off the table - for example inside a training process
+ * whose framework allocator has already reserved nearly all device memory, so that a raw allocation fails
+ * or fragments the pool, or inside a latency-bound step loop that must not hit the implicit device
+ * synchronisation of cudaMalloc / cudaFree.  Such a caller has nowhere to get the workspace that
+ * cdl_qlinear_bwd asks for.  Here the split-reduction scratch (int32 accumulators) and the status word sit in
+ * a static device array inside the library instead; every GPU that loads the library holds that array
+ * (256 bytes + 4 * CDL_NOALLOC_MAX_DW_ELEMS bytes = 4 MiB + 256 B) until the process exits.
+ *
+ *   dW[k,n] = (float)(sum_m A_idx[m,k] * G_idx[m,n]) * (g->q * a->q)      -- same values as cdl_qlinear_bwd
+ *   G_idx [dev] M x N int8 (ld ldg), A_idx [dev] M x K bytes (ld lda), dW [dev] K x N floats; alignment and
+ *   leading-dimension rules as for cdl_qlinear_bwd.  The caller still owns inputs and output.
+ *
+ * Limit: K * N <= CDL_NOALLOC_MAX_DW_ELEMS, otherwise CDL_ERR_TOO_LARGE and nothing is launched.
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ * Set-up: the first call on each device (with that device current) looks up the array's device address;
+ * make that first call before any stream capture begins.
+ * Sharing: all calls on a device use the same array, which still holds the previous call's contents; the
+ * call clears what it needs before use.  Two calls whose GPU work can overlap (different streams, no
+ * dependency) race on it: serialise them.  A device-side timeout is recorded only in the library's own
+ * status word and is not reported by this entry point.
+ */
+#define CDL_NOALLOC_MAX_DW_ELEMS (1 << 20)
+int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
+                               const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                               int32_t M, int32_t N, int32_t K, float *dW, void *stream);
 
 #define CDL_OP_QLINEAR_FWD 1
 #define CDL_OP_QLINEAR_BWD 2

@@ -12,7 +12,8 @@ from pathlib import Path
 __all__ = [
     "CdlError", "QuantParams", "IndexDesc", "library_path", "load_library",
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward",
-    "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_workspace_bytes", "cdl_workspace_status",
+    "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
+    "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
 
@@ -20,6 +21,7 @@ CDL_HIST_ACCUMULATE = 0x1
 CDL_OP_QLINEAR_FWD = 1
 CDL_OP_QLINEAR_BWD = 2
 CDL_MAX_LEVELS = 256
+CDL_NOALLOC_MAX_DW_ELEMS = 1 << 20
 
 _PKG = Path(__file__).resolve().parent
 _LIB = None
@@ -91,11 +93,12 @@ def load_library():
     lib.cdl_index_entropy.argtypes = [P, I32, P, P, P, P]
     lib.cdl_qlinear_fwd.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd.argtypes = [P, I64, P, P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, C.c_size_t, P]
+    lib.cdl_qlinear_bwd_dw_noalloc.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P]
     lib.cdl_workspace_bytes.argtypes = [I32, I32, I32, I32]
     lib.cdl_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_status.argtypes = [P, P]
     for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_index_entropy",
-                 "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_workspace_status"):
+                 "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status"):
         getattr(lib, name).restype = C.c_int
     _LIB = lib
     return lib
@@ -188,3 +191,12 @@ def cdl_qlinear_bwd(G_idx, ldg, g: IndexDesc, A_idx, lda, a, W_idx, ldw, w, M, N
                                         C.byref(wc) if wc is not None else None, M, N, K, _ptr(dXacc), _ptr(dX),
                                         _ptr(dWacc), _ptr(dW), _ptr(ws), ws_bytes, _stream(stream))
     return _check(rc, "cdl_qlinear_bwd", check)
+
+
+def cdl_qlinear_bwd_dw_noalloc(G_idx, ldg, g: IndexDesc, A_idx, lda, a: IndexDesc, M, N, K, dW, stream=None, check=True):
+    """dW = (g.q a.q) A_idx^T G_idx for callers that cannot allocate device memory: the scratch is a static array
+    inside the library (K * N <= CDL_NOALLOC_MAX_DW_ELEMS).  Calls that overlap on the GPU race on that array."""
+    gc, ac = g._c(), a._c()
+    rc = load_library().cdl_qlinear_bwd_dw_noalloc(_ptr(G_idx), ldg, C.byref(gc), _ptr(A_idx), lda, C.byref(ac), M, N, K,
+                                                   _ptr(dW), _stream(stream))
+    return _check(rc, "cdl_qlinear_bwd_dw_noalloc", check)

@@ -143,6 +143,7 @@ const char *cdl_strerror(int status)
         case CDL_ERR_LAUNCH: return "CUDA launch or runtime call failed";
         case CDL_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case CDL_ERR_UNSUPPORTED: return "device is not compute capability 10.x";
+        case CDL_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

@@ -516,3 +516,61 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
 }
 
 }  // namespace cdl
+
+// ------------------------------------------------------------------------------------------------
+// Weight-gradient product without any caller-provided or allocated scratch (see include/cdl.h).
+// The int32 accumulation buffer of the split reduction and the status word live in this file-scope
+// device array.  Host code must not pass the symbol itself to a kernel: its device address is looked
+// up once per device with cudaGetSymbolAddress and cached.
+namespace {
+constexpr size_t kStaticStatusBytes = 256;
+constexpr size_t kStaticAccElems = CDL_NOALLOC_MAX_DW_ELEMS;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticStatusBytes + kStaticAccElems * sizeof(int32_t)];
+unsigned char *g_static_ptr[64];   // device address of g_static_scratch, per device
+}  // namespace
+
+extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_desc *g, const void *A_idx,
+                                          int64_t lda, const cdl_index_desc *a, int32_t M, int32_t N, int32_t K,
+                                          float *dW, void *stream)
+{
+    using namespace cdl;
+    if (G_idx == nullptr || A_idx == nullptr || dW == nullptr || g == nullptr || a == nullptr) return CDL_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || ldg < N || lda < K) return CDL_ERR_ARG;
+    if ((int64_t)K * (int64_t)N > (int64_t)kStaticAccElems) return CDL_ERR_TOO_LARGE;
+    if (!(g->q > 0.0f) || !(a->q > 0.0f) || g->hi < g->lo || a->hi < a->lo) return CDL_ERR_RANGE;
+    if (g->lo < -128 || g->hi > 127 || a->lo < -128 || a->hi > 255 || (a->lo < 0 && a->hi > 127)) return CDL_ERR_RANGE;
+    if ((ldg & 15) || (lda & 15) || (reinterpret_cast<uintptr_t>(G_idx) & 15u) || (reinterpret_cast<uintptr_t>(A_idx) & 15u) ||
+        (reinterpret_cast<uintptr_t>(dW) & 3u))
+        return CDL_ERR_ALIGN;
+    auto absmax = [](int64_t lo, int64_t hi) {
+        const int64_t x = lo < 0 ? -lo : lo, y = hi < 0 ? -hi : hi;
+        return x > y ? x : y;
+    };
+    const int64_t amax = absmax(a->lo, a->hi), gmax = absmax(g->lo, g->hi);
+    if ((int64_t)M * amax * gmax >= ((int64_t)1 << 31)) return CDL_ERR_OVERFLOW_RISK;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
+    if (g_static_ptr[dev] == nullptr) {
+        // one-time set-up for this device (the device is current): resolve the array's device address
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+        g_static_ptr[dev] = static_cast<unsigned char *>(p);
+    }
+    unsigned char *base = g_static_ptr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: clear the status word here; the accumulation buffer is
+    // cleared by the launcher whenever the reduction is split
+    if (cudaMemsetAsync(base, 0, kStaticStatusBytes, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    GemmOperand X{A_idx, 1, lda, a->lo >= 0};
+    GemmOperand Y{G_idx, 1, ldg, false};
+    return launch_index_gemm_tc(X, Y, K, N, M, nullptr, dW, g->q * a->q, nullptr, base + kStaticStatusBytes,
+                                reinterpret_cast<int *>(base), st);
+}
