@@ -14,8 +14,12 @@
 // columns outside the matrix are zero-filled by TMA, which makes ragged edges and R tails exact.
 // Warp roles (192 threads): warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2-5 run the
 // epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
-// Work units are (tile, split of the reduced dimension); with more than one split the epilogue adds its
-// partial sums into an int32 buffer with red.global.add (integer, so the result does not depend on order).
+// Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to a
+// swizzled 128 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that
+// global memory sees whole 128-byte lines.  Work units are (tile, split of the reduced dimension); with more
+// than one split the staging block is added into an int32 buffer with a TMA bulk reduce-add (integer, so the
+// result does not depend on order).  Outputs whose pitch or base is not 16-byte aligned, and tiles 16 columns
+// wide, are written straight from registers instead.
 // Every wait is bounded: on expiry the kernel records CDL_ERR_TIMEOUT in the status word and winds down.
 #include <cuda.h>
 
@@ -31,6 +35,7 @@ constexpr int BR = 128;                 // bytes (= elements) of the reduced dim
 constexpr int kABytes = TM * BR;        // 16 KB
 constexpr int kBBytesMax = 256 * BR;    // 32 KB
 constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kOutBytes = TM * 128;     // epilogue staging block: 128 rows x 32 four-byte columns
 // The whole 227 KB opt-in window is requested (stages need 193 KB): operand descriptors then address
 // allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
 constexpr int kSmemBytes = 232448 - 1024;
@@ -50,6 +55,7 @@ struct TcParams {
     float scale;
     const float *bias;
     int *status;
+    int tma_f, tma_acc;     // the float / int32 output goes through shared memory and TMA
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -106,6 +112,36 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int c0, int c1, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int c0, int c1, uint32_t src)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// AND over the 128 epilogue threads (named barrier 1)
+__device__ __forceinline__ bool epi_all(bool v)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)v)
+        : "memory");
+    return out != 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -154,6 +190,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 
 __global__ void __launch_bounds__(kThreadsTC, 1)
 index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ CUtensorMap map_f, const __grid_constant__ CUtensorMap map_acc,
                      const TcParams P)
 {
     extern __shared__ unsigned char smem_dyn[];
@@ -283,64 +320,102 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     } else {
         // ------------------------------------------------------------ epilogue warps 2..5
         const int quarter = warp & 3;               // TMEM lanes this warp may read: 32 * (warp % 4) ..
-        uint32_t tcount = 0;
-        for (int u = blockIdx.x; u < units && !failed; u += gridDim.x, ++tcount) {
+        const int erow = quarter * 32 + lane;       // row of the tile owned by this thread
+        const bool leader = threadIdx.x == 64;      // issues and tracks the bulk stores
+        const uint32_t out_base = smem_base + (uint32_t)(kStages * kStageBytes);
+        const bool vec_ok = (P.J & 3) == 0;
+        uint32_t tcount = 0, ocount = 0;
+
+        // 32 four-byte values of this thread's row -> swizzled staging block -> TMA store or reduce-add
+        auto stage_and_send = [&](const uint32_t (&w)[32], const CUtensorMap *map, bool reduce, int col0, int row0) {
+            const uint32_t blk = out_base + (ocount & 1u) * (uint32_t)kOutBytes;
+            if (leader) bulk_wait_read_1();         // the block used two sends ago has been read out
+            epi_barrier();
+            const uint32_t dst = blk + (uint32_t)erow * 128u;
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c4 ^ (erow & 7)) << 4)),
+                             "r"(w[4 * c4]), "r"(w[4 * c4 + 1]), "r"(w[4 * c4 + 2]), "r"(w[4 * c4 + 3])
+                             : "memory");
+            fence_async_smem();
+            epi_barrier();
+            if (leader) {
+                if (reduce) tma_reduce_add_2d(map, col0, row0, blk);
+                else tma_store_2d(map, col0, row0, blk);
+                bulk_commit();
+            }
+            ++ocount;
+        };
+
+        for (int u = blockIdx.x; u < units; u += gridDim.x, ++tcount) {
             const int tile = u / P.splits;
             const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(buf), tph, abort_flag)) {
+            // the four warps must agree on the outcome: the staging code below uses CTA-level named barriers
+            if (!epi_all(mbar_wait(tfull_bar(buf), tph, abort_flag))) {
                 failed = true;
                 break;
             }
             tc_fence_after();
-            const int row = ti * TM + quarter * 32 + lane;
+            const int row = ti * TM + erow;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
-            const bool vec_ok = (P.J & 3) == 0;
             for (int c0 = 0; c0 < P.TN; c0 += 32) {
+                const int col0 = tj * P.TN + c0;
+                if (col0 >= P.J) break;             // uniform over the CTA
                 uint32_t v[32];
                 tc_ld32(taddr + (uint32_t)c0, v);
                 tc_wait_ld();
-                const int col0 = tj * P.TN + c0;
-                if (row < P.I && col0 < P.J) {
-                    const long long off = (long long)row * P.J + col0;
-                    const int ncol = min(min(32, P.TN - c0), P.J - col0);
-                    if (P.splits > 1) {
+                const int ncol = min(min(32, P.TN - c0), P.J - col0);
+                const long long off = (long long)row * P.J + col0;
+                const bool in_rows = row < P.I;
+                if (P.splits > 1) {
+                    if (P.tma_acc) {
+                        stage_and_send(v, &map_acc, true, col0, ti * TM);
+                    } else if (in_rows) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol)
                                 asm volatile("red.global.add.s32 [%0], %1;" ::"l"(P.acc_out + off + c), "r"(v[c]) : "memory");
-                    } else {
-                        if (P.acc_out != nullptr) {
-                            if (vec_ok && ncol == 32) {
+                    }
+                    continue;
+                }
+                if (P.acc_out != nullptr) {
+                    if (P.tma_acc) {
+                        stage_and_send(v, &map_acc, false, col0, ti * TM);
+                    } else if (in_rows) {
+                        if (vec_ok && ncol == 32) {
 #pragma unroll
-                                for (int c = 0; c < 32; c += 4)
-                                    *reinterpret_cast<int4 *>(P.acc_out + off + c) =
-                                        make_int4((int)v[c], (int)v[c + 1], (int)v[c + 2], (int)v[c + 3]);
-                            } else {
+                            for (int c = 0; c < 32; c += 4)
+                                *reinterpret_cast<int4 *>(P.acc_out + off + c) =
+                                    make_int4((int)v[c], (int)v[c + 1], (int)v[c + 2], (int)v[c + 3]);
+                        } else {
 #pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c < ncol) P.acc_out[off + c] = (int)v[c];
-                            }
+                            for (int c = 0; c < 32; ++c)
+                                if (c < ncol) P.acc_out[off + c] = (int)v[c];
                         }
-                        if (P.f_out != nullptr) {
-                            float f[32];
+                    }
+                }
+                if (P.f_out != nullptr) {
+                    uint32_t f[32];
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) f[c] = __fmul_rn((float)(int)v[c], P.scale);
-                            if (P.bias != nullptr) {
+                    for (int c = 0; c < 32; ++c) f[c] = __float_as_uint(__fmul_rn((float)(int)v[c], P.scale));
+                    if (P.bias != nullptr) {
 #pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c < ncol) f[c] = __fadd_rn(f[c], P.bias[col0 + c]);
-                            }
-                            if (vec_ok && ncol == 32) {
+                        for (int c = 0; c < 32; ++c)
+                            if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
+                    }
+                    if (P.tma_f) {
+                        stage_and_send(f, &map_f, false, col0, ti * TM);
+                    } else if (in_rows) {
+                        if (vec_ok && ncol == 32) {
 #pragma unroll
-                                for (int c = 0; c < 32; c += 4)
-                                    *reinterpret_cast<float4 *>(P.f_out + off + c) = make_float4(f[c], f[c + 1], f[c + 2], f[c + 3]);
-                            } else {
+                            for (int c = 0; c < 32; c += 4)
+                                *reinterpret_cast<uint4 *>(P.f_out + off + c) = make_uint4(f[c], f[c + 1], f[c + 2], f[c + 3]);
+                        } else {
 #pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c < ncol) P.f_out[off + c] = f[c];
-                            }
+                            for (int c = 0; c < 32; ++c)
+                                if (c < ncol) P.f_out[off + c] = __uint_as_float(f[c]);
                         }
                     }
                 }
@@ -349,6 +424,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
         }
+        if (leader) bulk_wait_all();                // staged blocks are out before shared memory goes away
         if (failed && lane == 0) {
             abort_s = 1;
             atomicExch(P.status, CDL_ERR_TIMEOUT);
@@ -394,6 +470,20 @@ EncodeTiledFn get_encode()
         fn = reinterpret_cast<EncodeTiledFn>(p);
     }
     return fn;
+}
+
+// Output matrix [rows][cols] of 4-byte elements, row pitch cols * 4; box = {32 columns (128 bytes), 128 rows}.
+bool encode_out_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows, bool is_float)
+{
+    EncodeTiledFn fn = get_encode();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 4};
+    const cuuint32_t box[2] = {32u, (cuuint32_t)TM};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, is_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 2, const_cast<void *>(base),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // 2D byte tensor [outer][inner] with row pitch `pitch` bytes; box = {128 bytes, box_rows}, 128-byte swizzle.
@@ -491,6 +581,19 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
     else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, (uint32_t)TN);
+    // outputs through shared memory + TMA when their pitch and base allow it and the tile is at least one box wide
+    CUtensorMap map_f = map_a, map_acc = map_a;      // placeholders when unused
+    const bool out_ok = TN >= 32 && (J & 3) == 0;
+    P.tma_f = 0;
+    P.tma_acc = 0;
+    if (out_ok && splits == 1 && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
+        ok = ok && encode_out_map(&map_f, f_out, (uint64_t)J, (uint64_t)I, true);
+        P.tma_f = 1;
+    }
+    if (out_ok && P.acc_out != nullptr && (reinterpret_cast<uintptr_t>(P.acc_out) & 15u) == 0) {
+        ok = ok && encode_out_map(&map_acc, P.acc_out, (uint64_t)J, (uint64_t)I, false);
+        P.tma_acc = 1;
+    }
     if (!ok) return CDL_ERR_LAUNCH;
 
     static bool attr_set[64];
@@ -505,7 +608,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     }
     const long long units = tiles * splits;
     const int grid = (int)(units < sms ? units : sms);
-    index_gemm_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, P);
+    index_gemm_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (splits > 1 && f_out != nullptr) {
         const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
