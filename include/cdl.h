@@ -92,7 +92,7 @@ typedef struct cdl_index_desc {
  * Hard index = uniform quantizer Q_u, the limit of Q_p and Q_d for large alpha (Remark of
  * Sec. IV-A; end of Sec. IV-B), with the per-tensor level histogram fused in (the empirical
  * distribution over levels whose entropy Sec. V-C constrains).
- *   idx = clamp(round_half_even(x / q), lo, hi), quotient in IEEE binary32; NaN -> level nearest 0.
+ *   idx = clamp(round_half_even(x / q), lo, hi), quotient in IEEE binary32; a NaN input gives lo.
  *   x        [dev] n floats (4-byte aligned; 16-byte alignment takes the vector path).
  *   p        [host].
  *   idx_out  [dev] n bytes (int8 or uint8, see cdl_quant_params), nullable.

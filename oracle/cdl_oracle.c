@@ -161,7 +161,7 @@ void cdl_oracle_partials(const float *x, int64_t n, float q, int lo, int hi,
 
 /* ---------------------------------------------------------------------------
  * Hard index = uniform quantizer Q_u (nearest level), binary32 quotient,
- * round-half-even, clamped; a NaN input takes the level nearest 0.
+ * round-half-even, clamped; a NaN quotient takes the lowest level lo.
  * hist (nullable, nlev counters) is incremented, not cleared.
  * ------------------------------------------------------------------------- */
 void cdl_oracle_hard(const float *x, int64_t n, float q, int lo, int hi,
@@ -170,8 +170,7 @@ void cdl_oracle_hard(const float *x, int64_t n, float q, int lo, int hi,
     for (int64_t e = 0; e < n; ++e) {
         const float u = x[e] / q;            /* IEEE binary32 division */
         float r = nearbyintf(u);             /* default mode: ties to even */
-        if (r != r) r = 0.0f;
-        if (r < (float)lo) r = (float)lo;
+        if (!(r >= (float)lo)) r = (float)lo;    /* also catches NaN */
         if (r > (float)hi) r = (float)hi;
         const int k = (int)r;
         if (idx) idx[e] = k;

@@ -71,12 +71,14 @@ int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out)
         const double q = (double)p->q, al = (double)p->alpha;
         const double a = al * q * q;
         d.c1 = (float)(al * q * 1.4426950408889634074);
-        d.decay = (float)exp(-2.0 * a);
+        d.A = (float)(a * 1.4426950408889634074);
+        d.c1x2 = (float)(2.0 * al * q * 1.4426950408889634074);
+        d.near3 = a > 12.0 ? 1 : 0;
         d.a2 = (float)(2.0 * a);
         d.two_aq = (float)(2.0 * al * q);
         d.q2 = (float)(q * q);
         d.rate_c = (float)((double)p->rate_weight * (-2.0 * al * q));
-        if (!isfinite(d.c1) || !isfinite(d.a2) || !isfinite(d.two_aq) || !isfinite(d.rate_c) || !(d.q2 > 0.0f))
+        if (!isfinite(d.c1) || !isfinite(d.c1x2) || !isfinite(d.A) || !isfinite(d.a2) || !isfinite(d.two_aq) || !isfinite(d.rate_c) || !(d.q2 > 0.0f))
             return CDL_ERR_RANGE;
         d.window = (p->window >= (int)nlev) ? 0 : p->window;
         // e_j <= 2^(-a log2e j (j - 1)) for the levels j steps beyond the nearest one: below 2^-40 past jmax

@@ -15,7 +15,9 @@ struct QuantDev {
     float flo, fhi;   // index range as floats
     int lo, hi, nlev;
     float c1;         // alpha * q * log2(e): the logit of level kn+j relative to level kn is -c1 * j * (j q - 2 d)
-    float decay;      // exp(-2 alpha q^2): ratio step of the neighbour recurrence
+    float A;          // alpha * q^2 * log2(e) = c1 * q
+    float c1x2;       // 2 * c1
+    int near3;        // alpha q^2 > 12: only the nearest level and its two neighbours carry weight (> 2^-34 relative)
     float a2;         // 2 alpha q^2: dQ_d/dtheta = a2 * Var{J}
     float two_aq;     // 2 alpha q
     float q2;         // q^2

@@ -2,24 +2,30 @@
 // analytic backward.  One pass over the tensor each; HBM-bound by design.
 //
 // Arithmetic (per element theta, Sec. IV of the paper):
-//   k0  = clamp(rint(theta / q))                 the hard index (binary32 quotient, ties to even)
-//   d   = theta - kn q  as an unevaluated sum dh + dl of two floats (kn = nearest in-range level):
-//         k0 q is split exactly with one fma, theta - fl(k0 q) is exact (operands within a factor
-//         of two), so d carries ~48 bits.  This matters next to the midpoints between levels when
-//         alpha q^2 is large: there dQ_d/dtheta ~ alpha q^2 / 2 and a 2^-24 error in d is visible.
-//   e_j = exp(-alpha ((d - j q)^2 - d^2)) = 2^(-c1 j (j q - 2 d)),  c1 = alpha q log2 e,
-//         the CPMF of Eq. (4) relative to level kn: P_{kn+j} = e_j / sum_j e_j, e_0 = 1, e_j <= 1.
-//   J   = index offset from kn under that CPMF; moments m1 = E J, m2 = E J^2, m3 = E J^3.
-//   Q_d = kn q + q m1                                                   (Eq. (8))
+//   k0  = rint(clamp(theta / q, lo, hi))         the hard index (binary32 quotient, ties to even).  Rounding
+//         is done by adding 1.5 * 2^23 (no conversion instruction); the integer is read from the mantissa.
+//   d   = theta - kn q, kn the reference level (k0, or the exact nearest level when a window is used).
+//   e_j = exp(-alpha ((d - j q)^2 - d^2)) = 2^(j (B - A j)),  A = alpha q^2 log2 e, B = 2 alpha q d log2 e:
+//         the CPMF of Eq. (4) relative to level kn, P_{kn+j} = e_j / sum e_j, e_0 = 1, e_j <= 1 (no max pass).
+//   Moments of the index offset under that CPMF give everything else:
+//   Q_d = kn q + q E J                                                   (Eq. (8))
 //   dQ_d/dtheta = 2 alpha q^2 Var J                                      (Lemma 1, Eq. (9a))
-//   dQ_d/dq     = kn + m1 + 2 alpha q ((d - kn q) Var J - q Cov(J, J^2)) (Eq. (9b), re-centred on kn)
+//   dQ_d/dq     = kn + E J + 2 alpha q ((d - kn q) Var J - q Cov(J, J^2)) (Eq. (9b), re-centred on kn)
 //   dQ_d/dalpha = q^2 (2 d Var J - q Cov(J, J^2))                        (Appendix B steps, re-centred)
-//   rate term   = rate_weight * (-2 alpha q) * (E[L J] - m1 E[L]),  L = log2 of the level probability.
+//   rate term   = rate_weight * (-2 alpha q) * Cov(L, J),  L = log2 of the level probability.
 // The re-centred forms equal the printed ones (expand X = q (kn + J)) without their cancellation.
 //
-// Window of 5 (Sec. VI-B.1): the five in-range levels nearest theta form a contiguous block that
-// contains kn.  Their e_j come from two ex2 (j = +1, -1) and the lattice recurrence
-// e_{j+1} = e_j r_j, r_{j+1} = r_j exp(-2 alpha q^2), which keeps the MUFU count at 2 per element.
+// Three evaluation paths, chosen per launch from alpha q^2 and the window (both uniform over the tensor):
+//   NEAR3  alpha q^2 > 12: levels two or more steps from the nearest one weigh < e^-24; only kn-1, kn, kn+1 are
+//          summed.  Here d must be exact next to the midpoints (dQ_d/dtheta ~ alpha q^2 / 2 there), so d is
+//          carried as an unevaluated sum dh + dl of two floats: k0 q is split exactly with one fma and
+//          theta - fl(k0 q) is exact (operands within a factor of two).
+//   WIN5   alpha q^2 <= 12, window of 5 (Sec. VI-B.1): the five in-range levels nearest theta, st .. st+4, each
+//          with its own ex2; moments are taken about st with compile-time weights 0..4 and shifted to kn.
+//          The window needs the exact nearest level (ties: the lower one), decided from dh + dl on a rarely
+//          taken branch.
+//   LOOP   everything else (whole index set, or another odd window): a loop over the levels within jmax
+//          steps of kn (further ones weigh < 2^-40).
 #include "cdl_internal.h"
 
 #include <math.h>
@@ -29,11 +35,21 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kBatch = 4;  // float4 loads in flight per thread
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
+constexpr int kMagicBits = 0x4B400000;
+
+enum QuantPath { PATH_NEAR3 = 0, PATH_WIN5 = 1, PATH_LOOP = 2 };
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
@@ -45,97 +61,136 @@ struct ElemOut {
     float ta;     // g * dQ_d/dalpha
 };
 
-template <int MODE, bool WIN5, bool RATE>
+// d = x - k q as dh + dl (dl: what dh lost), k an integer-valued float near x / q
+__device__ __forceinline__ void residual2(float x, float k, float q, float &dh, float &dl)
+{
+    const float ph = __fmul_rn(k, q);
+    const float pl = __fmaf_rn(k, q, -ph);
+    const float s = __fsub_rn(x, ph);
+    dh = __fsub_rn(s, pl);
+    dl = __fsub_rn(__fsub_rn(s, dh), pl);
+}
+
+// Moves (kn, ki, dh) to the exact nearest in-range level; of two equally near levels the lower one.
+__device__ __noinline__ void nearest_fixup(const QuantDev &P, float &kn, int &ki, float &dh, float dl)
+{
+    if ((dh > P.half_q || (dh == P.half_q && dl > 0.0f)) && kn < P.fhi) {
+        kn += 1.0f;
+        ki += 1;
+        dh = __fsub_rn(dh, P.q);
+    } else if ((dh < -P.half_q || (dh == -P.half_q && dl <= 0.0f)) && kn > P.flo) {
+        kn -= 1.0f;
+        ki -= 1;
+        dh = __fadd_rn(dh, P.q);
+    }
+}
+
+template <int MODE, int PATH, bool RATE>
 __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__restrict__ Ltab, float x, float g)
 {
     ElemOut o;
-    // ---- hard index: the defining binary32 expression
-    const float u = __fdiv_rn(x, P.q);
-    float r = rintf(u);
-    r = (r != r) ? 0.0f : r;
-    const float k0 = fminf(fmaxf(r, P.flo), P.fhi);
-    o.k0 = (int)k0;
+    const float q = P.q;
+    // ---- hard index: the defining binary32 expression; a NaN quotient clamps to lo
+    const float u = __fdiv_rn(x, q);
+    const float c = fminf(fmaxf(u, P.flo), P.fhi);
+    const float t = __fadd_rn(c, kMagic);
+    float kn = __fsub_rn(t, kMagic);
+    int ki = __float_as_int(t) - kMagicBits;
+    o.k0 = ki;
     o.y = 0.0f;
     o.gx = 0.0f;
     o.tq = 0.0f;
     o.ta = 0.0f;
     if (MODE == MODE_HARD) return o;
 
-    // ---- d = theta - k0 q as dh + dl
-    const float q = P.q;
-    const float ph = __fmul_rn(k0, q);
-    const float pl = __fmaf_rn(k0, q, -ph);
-    const float s = __fsub_rn(x, ph);
-    float dh = __fsub_rn(s, pl);
-    const float dl = __fsub_rn(__fsub_rn(s, dh), pl);
-    float kn = k0;
-    int jlo, jhi;
-    if (P.window > 0) {
-        // exact nearest level; of two equally near levels the lower one
-        const bool up = (dh > P.half_q || (dh == P.half_q && dl > 0.0f)) && (kn < P.fhi);
-        if (up) {
-            kn += 1.0f;
-            dh = __fsub_rn(dh, q);
-        }
-        const bool dn = (dh < -P.half_q || (dh == -P.half_q && dl <= 0.0f)) && (kn > P.flo);
-        if (dn) {
-            kn -= 1.0f;
-            dh = __fadd_rn(dh, q);
-        }
-        const int kni = (int)kn;
-        const int st = min(max(kni - (P.window >> 1), P.lo), P.hi - P.window + 1);
-        jlo = st - kni;
-        jhi = jlo + P.window - 1;
-    } else {
-        const int kni = (int)kn;
-        jlo = max(P.lo - kni, -P.jmax);
-        jhi = min(P.hi - kni, P.jmax);
-    }
-    const int kni = (int)kn;
-    const float m2d = -2.0f * dh;
-    const float dl2 = 2.0f * dl;
-
-    // The rate term is a covariance with L, so L may be shifted by a constant: measuring it from the
-    // nearest level's value makes the j = 0 term vanish and a flat L give exactly zero.
-    float S = 1.0f, S1 = 0.0f, S2 = 0.0f, S3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
-    const float Lc = RATE ? Ltab[kni - P.lo] : 0.0f;
-
-    if (WIN5) {
-        const float w1 = __fsub_rn(__fadd_rn(q, m2d), dl2);   // (q - 2 dh) - 2 dl
+    float m1, varj = 0.0f, covj = 0.0f, rate = 0.0f, dh;   // moments of J about kn
+    if (PATH == PATH_NEAR3) {
+        float dl;
+        residual2(x, kn, q, dh, dl);
+        const float m2d = -2.0f * dh, dl2 = 2.0f * dl;
+        const float w1 = __fsub_rn(__fadd_rn(q, m2d), dl2);   // (q - 2 dh) - 2 dl, exact near the midpoint
         const float wm = __fadd_rn(__fsub_rn(q, m2d), dl2);   // (q + 2 dh) + 2 dl
-        const float e1 = ex2_approx(-P.c1 * w1);
-        const float em = ex2_approx(-P.c1 * wm);
-        const int nneg = -jlo;  // levels below kn in the window: 0..4
-        float e = 1.0f, rr = em;
-#pragma unroll
-        for (int i = 1; i <= 4; ++i) {
-            if (i == nneg + 1) {  // switch from the downward to the upward chain
-                e = 1.0f;
-                rr = e1;
+        float e1 = ex2_approx(-P.c1 * w1);
+        float em = ex2_approx(-P.c1 * wm);
+        e1 = (kn < P.fhi) ? e1 : 0.0f;
+        em = (kn > P.flo) ? em : 0.0f;
+        const float rS = rcp_approx(1.0f + e1 + em);
+        m1 = (e1 - em) * rS;
+        o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
+        if (MODE == MODE_BWD) {
+            const float m2 = (e1 + em) * rS;         // E J^2; E J^3 = E J
+            varj = fmaf(-m1, m1, m2);
+            covj = m1 - m1 * m2;
+            if (RATE) {
+                const float Lc = Ltab[ki - P.lo];
+                const float l1 = (Ltab[min(ki + 1, P.hi) - P.lo] - Lc) * e1;
+                const float lm = (Ltab[max(ki - 1, P.lo) - P.lo] - Lc) * em;
+                rate = ((l1 - lm) - m1 * (l1 + lm)) * rS;
             }
-            e *= rr;
-            rr *= P.decay;
-            const int j = (i <= nneg) ? -i : (i - nneg);
-            const float jf = (float)j;
-            S += e;
-            S1 = fmaf(jf, e, S1);
+        }
+    } else if (PATH == PATH_WIN5) {
+        float dl;
+        residual2(x, kn, q, dh, dl);
+        if (fabsf(dh) >= P.half_q) nearest_fixup(P, kn, ki, dh, dl);
+        const float stf = fminf(fmaxf(kn - 2.0f, P.flo), P.fhi - 4.0f);
+        const float j0 = stf - kn;                    // -4 .. 0
+        const float B = P.c1x2 * dh;
+        float T0 = 0.0f, T1 = 0.0f, T2 = 0.0f, T3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
+        const float *Lp = Ltab;
+        float Lc = 0.0f;
+        if (RATE) {
+            Lc = Ltab[ki - P.lo];
+            Lp = Ltab + (min(max(ki - 2, P.lo), P.hi - 4) - P.lo);
+        }
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+            const float jf = j0 + (float)i;
+            const float e = ex2_approx(jf * fmaf(-P.A, jf, B));
+            T0 += e;
+            if (i > 0) T1 = fmaf((float)i, e, T1);
             if (MODE == MODE_BWD) {
-                const float j2 = jf * jf;
-                S2 = fmaf(j2, e, S2);
-                S3 = fmaf(j2 * jf, e, S3);
+                if (i > 0) {
+                    T2 = fmaf((float)(i * i), e, T2);
+                    T3 = fmaf((float)(i * i * i), e, T3);
+                }
                 if (RATE) {
-                    const float le = (Ltab[kni - P.lo + j] - Lc) * e;
+                    const float le = (Lp[i] - Lc) * e;
                     R0 += le;
-                    R1 = fmaf(jf, le, R1);
+                    if (i > 0) R1 = fmaf((float)i, le, R1);
                 }
             }
+        }
+        const float rT = rcp_approx(T0);
+        const float mi = T1 * rT;                      // E I, I = level - st
+        o.y = __fmaf_rn(stf, q, __fmul_rn(q, mi));
+        m1 = mi + j0;
+        if (MODE == MODE_BWD) {
+            const float m2i = T2 * rT, m3i = T3 * rT;
+            varj = fmaf(-mi, mi, m2i);
+            covj = fmaf(-mi, m2i, m3i) + 2.0f * j0 * varj;   // Cov(J, J^2) with J = I + j0
+            if (RATE) rate = (R1 - mi * R0) * rT;
         }
     } else {
-        for (int j = jlo; j <= jhi; ++j) {
-            if (j == 0) continue;
-            const float jf = (float)j;
-            const float w = __fsub_rn(__fmaf_rn(jf, q, m2d), dl2);   // (j q - 2 dh) - 2 dl
-            const float e = ex2_approx((-P.c1 * jf) * w);
+        int jlo, jhi;
+        if (P.window > 0) {
+            float dl;
+            residual2(x, kn, q, dh, dl);
+            if (fabsf(dh) >= P.half_q) nearest_fixup(P, kn, ki, dh, dl);
+            const int st = min(max(ki - (P.window >> 1), P.lo), P.hi - P.window + 1);
+            jlo = st - ki;
+            jhi = jlo + P.window - 1;
+        } else {
+            dh = __fmaf_rn(-kn, q, x);
+            jlo = max(P.lo - ki, -P.jmax);
+            jhi = min(P.hi - ki, P.jmax);
+        }
+        const float B = P.c1x2 * dh;
+        float S = 0.0f, S1 = 0.0f, S2 = 0.0f, S3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
+        const float Lc = RATE ? Ltab[ki - P.lo] : 0.0f;
+        const float *Lp = Ltab + (ki - P.lo);
+        float jf = (float)jlo;
+        for (int j = jlo; j <= jhi; ++j, jf += 1.0f) {
+            const float e = ex2_approx(jf * fmaf(-P.A, jf, B));
             S += e;
             S1 = fmaf(jf, e, S1);
             if (MODE == MODE_BWD) {
@@ -143,27 +198,29 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                 S2 = fmaf(j2, e, S2);
                 S3 = fmaf(j2 * jf, e, S3);
                 if (RATE) {
-                    const float le = (Ltab[kni - P.lo + j] - Lc) * e;
+                    const float le = (Lp[j] - Lc) * e;
                     R0 += le;
                     R1 = fmaf(jf, le, R1);
                 }
             }
         }
+        const float rS = rcp_approx(S);
+        m1 = S1 * rS;
+        o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
+        if (MODE == MODE_BWD) {
+            const float m2 = S2 * rS, m3 = S3 * rS;
+            varj = fmaf(-m1, m1, m2);
+            covj = fmaf(-m1, m2, m3);
+            if (RATE) rate = (R1 - m1 * R0) * rS;
+        }
     }
-    const float rS = __frcp_rn(S);
-    const float m1 = S1 * rS;
-    o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
     if (MODE == MODE_BWD) {
-        const float m2 = S2 * rS;
-        const float m3 = S3 * rS;
-        const float varj = fmaf(-m1, m1, m2);
-        const float cov3 = fmaf(-m1, m2, m3);
         float gx = g * (P.a2 * varj);
-        if (RATE) gx = fmaf(P.rate_c, (R1 - m1 * R0) * rS, gx);
+        if (RATE) gx = fmaf(P.rate_c, rate, gx);
         o.gx = gx;
-        const float dmk = fmaf(-kn, q, dh);  // d - kn q
-        const float dq = (kn + m1) + P.two_aq * (dmk * varj - q * cov3);
-        const float da = P.q2 * (2.0f * dh * varj - q * cov3);
+        const float dmk = fmaf(-kn, q, dh);            // d - kn q
+        const float dq = (kn + m1) + P.two_aq * (dmk * varj - q * covj);
+        const float da = P.q2 * (2.0f * dh * varj - q * covj);
         o.tq = g * dq;
         o.ta = g * da;
     }
@@ -177,7 +234,7 @@ __device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane
 
 // Vector region: elements [head, head + 4 n4); the remaining head + tail elements are done one by one.
 // When the pointers do not allow 128-bit access the host passes n4 = 0 and everything is scalar.
-template <int MODE, bool WIN5, bool RATE>
+template <int MODE, int PATH, bool RATE>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__restrict__ g, int64_t n,
                 int64_t head, int64_t n4, float *__restrict__ y, unsigned char *__restrict__ idx,
@@ -237,7 +294,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 unsigned int packed = 0u;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const ElemOut o = quant_elem<MODE, WIN5, RATE>(P, Ltab, xs[c], gs[c]);
+                    const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c]);
                     ys[c] = o.y;
                     gxs[c] = o.gx;
                     part_q += o.tq;
@@ -262,7 +319,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     for (int64_t t = tid; t < nrem; t += stride) {
         const int64_t i = (t < head) ? t : (tail0 + (t - head));
         const float gi = (MODE == MODE_BWD) ? g[i] : 0.0f;
-        const ElemOut o = quant_elem<MODE, WIN5, RATE>(P, Ltab, x[i], gi);
+        const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, x[i], gi);
         if (MODE == MODE_SOFT) y[i] = o.y;
         if (MODE == MODE_BWD) {
             if (gx != nullptr) gx[i] = o.gx;
@@ -307,13 +364,13 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     }
 }
 
-template <int MODE, bool WIN5, bool RATE>
+template <int MODE, int PATH, bool RATE>
 int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int64_t head, int64_t n4,
              float *y, unsigned char *idx, unsigned long long *hist, float *gx, double *gq, double *ga,
              cudaStream_t stream)
 {
     const size_t smem = CDL_MAX_LEVELS * sizeof(float) + (hist ? (size_t)qd.nlev * 32 * sizeof(unsigned int) : 0);
-    auto kern = quantize_kernel<MODE, WIN5, RATE>;
+    auto kern = quantize_kernel<MODE, PATH, RATE>;
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem) != cudaSuccess || per_sm < 1) {
         (void)cudaGetLastError();
@@ -365,23 +422,29 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     if (n4 == 0) head = 0;
 
     unsigned char *ib = static_cast<unsigned char *>(idx);
-    const bool win5 = qd.window == 5;
+    const int path = qd.near3 ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
     const bool rate = (mode == MODE_BWD) && qd.level_prob != nullptr && qd.rate_c != 0.0f;
+#define CDL_Q(M, PTH, RT) \
+    launch_t<M, PTH, RT>(qd, x, grad_out, n, head, n4, y, ib, hist, grad_x, grad_q, grad_alpha, stream)
     switch (mode) {
         case MODE_HARD:
-            return launch_t<MODE_HARD, false, false>(qd, x, nullptr, n, head, n4, nullptr, ib, hist, nullptr, nullptr, nullptr, stream);
+            return CDL_Q(MODE_HARD, PATH_LOOP, false);
         case MODE_SOFT:
-            return win5 ? launch_t<MODE_SOFT, true, false>(qd, x, nullptr, n, head, n4, y, ib, hist, nullptr, nullptr, nullptr, stream)
-                        : launch_t<MODE_SOFT, false, false>(qd, x, nullptr, n, head, n4, y, ib, hist, nullptr, nullptr, nullptr, stream);
+            return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, false)
+                 : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, false)
+                                     : CDL_Q(MODE_SOFT, PATH_LOOP, false);
         case MODE_BWD:
-            if (win5)
-                return rate ? launch_t<MODE_BWD, true, true>(qd, x, grad_out, n, head, n4, nullptr, nullptr, nullptr, grad_x, grad_q, grad_alpha, stream)
-                            : launch_t<MODE_BWD, true, false>(qd, x, grad_out, n, head, n4, nullptr, nullptr, nullptr, grad_x, grad_q, grad_alpha, stream);
-            return rate ? launch_t<MODE_BWD, false, true>(qd, x, grad_out, n, head, n4, nullptr, nullptr, nullptr, grad_x, grad_q, grad_alpha, stream)
-                        : launch_t<MODE_BWD, false, false>(qd, x, grad_out, n, head, n4, nullptr, nullptr, nullptr, grad_x, grad_q, grad_alpha, stream);
+            if (rate)
+                return path == PATH_NEAR3 ? CDL_Q(MODE_BWD, PATH_NEAR3, true)
+                     : path == PATH_WIN5 ? CDL_Q(MODE_BWD, PATH_WIN5, true)
+                                         : CDL_Q(MODE_BWD, PATH_LOOP, true);
+            return path == PATH_NEAR3 ? CDL_Q(MODE_BWD, PATH_NEAR3, false)
+                 : path == PATH_WIN5 ? CDL_Q(MODE_BWD, PATH_WIN5, false)
+                                     : CDL_Q(MODE_BWD, PATH_LOOP, false);
         default:
             return CDL_ERR_ARG;
     }
+#undef CDL_Q
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -208,7 +208,7 @@ def test_exact_midpoints_clamping_nan_and_signed_zero(torch):
     ref_idx, ref_hist = oracle.hard(x, q, -2, 3)
     idx, hist = run_hard(torch, x, P)
     assert np.array_equal(idx, ref_idx) and np.array_equal(hist, ref_hist)
-    assert list(idx[:12]) == [0, 2, 2, 0, -2, 3, -2, 3, -2, 0, 0, 0]
+    assert list(idx[:12]) == [0, 2, 2, 0, -2, 3, -2, 3, -2, -2, 0, 0]
     # exact midpoints with the 5-level window: the lower of two equally near levels centres the window
     xm = ((np.arange(0, 15) + 0.5) * 0.25).astype(f32)
     Pw = cdl.QuantParams(0.25, 0, 15, 2.0, window=5)

@@ -244,9 +244,9 @@ def test_hard_ties_clamp_and_nan():
     x = np.array([0.25, 0.75, 1.25, -0.25, -0.75, 100.0, -100.0, np.inf, -np.inf, np.nan, 0.0, -0.0], dtype=f32)
     idx, hist = oracle.hard(x, q, -2, 3)
     # quotients .5, 1.5, 2.5, -.5, -1.5 round to the even neighbour
-    assert list(idx) == [0, 2, 2, 0, -2, 3, -2, 3, -2, 0, 0, 0]
+    assert list(idx) == [0, 2, 2, 0, -2, 3, -2, 3, -2, -2, 0, 0]      # NaN -> lo
     idx_u, _ = oracle.hard(np.array([np.nan, -3.0], dtype=f32), q, 2, 5)
-    assert list(idx_u) == [2, 2]                       # level nearest 0 inside [lo, hi]
+    assert list(idx_u) == [2, 2]                       # NaN and values below the range -> lo
     assert hist.sum() == x.size
 
 
