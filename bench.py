@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--workload", default="resnet18_layer3_conv",
                     choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
+    ap.add_argument("--sweep-max-log2n", type=int, default=28)
     return ap.parse_args()
 
 
@@ -222,8 +225,100 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Quantizer-only bandwidth sweep: fp32 tensors of 2^20 .. 2^max elements (50/50 N(0,1) / Laplace(0,1) mixture
+    drawn on the device), L in {1,3,7,15,127}, alpha in {1,100,1e4}, step 4/L; hard, hard+hist, soft, soft+idx+hist,
+    backward and backward+rate timed separately with CUDA events."""
+    import torch
+
+    import paper_2501_09849_b200 as cdl
+    from paper_2501_09849_b200 import build as cdl_build
+    cdl_build.build()
+    cdl.load_library()
+    torch.cuda.set_device(0)
+    pk, pk_kind = peaks()
+    hbm = float(pk["hbm_gbs"])
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    nmax = 1 << args.sweep_max_log2n
+    pick = torch.rand(nmax, device="cuda", generator=gen) < 0.5
+    xn = torch.randn(nmax, device="cuda", generator=gen)
+    u = torch.rand(nmax, device="cuda", generator=gen) - 0.5
+    xl = -torch.sign(u) * torch.log1p(-2.0 * u.abs())           # Laplace(0,1) by inversion
+    x = torch.where(pick, xn, xl).contiguous()
+    del pick, xn, xl, u
+    g = torch.randn(nmax, device="cuda", generator=gen)
+    y = torch.empty(nmax, dtype=torch.float32, device="cuda")
+    idx = torch.empty(nmax, dtype=torch.int8, device="cuda")
+    s = torch.zeros(2, dtype=torch.float64, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    reps = max(3, args.steps // 4)
+
+    def timed(make_fn, n):
+        """Median time of one launch.  Launches are issued back to back on distinct slices of the big buffers
+        (so that none finds its input in L2 and the CPU-side launch cost is hidden), one event pair around all."""
+        k = max(1, min(16, nmax // n))
+        fns = [make_fn(i * n) for i in range(k)]
+        for f in fns[:2]:
+            f()
+        ts = []
+        for _ in range(reps):
+            if k * n * 12 < (512 << 20):
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for f in fns:
+                f()
+            e1.record(stream)
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1) / k)
+        return statistics.median(ts)
+
+    rows = []
+    for log2n in range(20, args.sweep_max_log2n + 1, 2):
+        n = 1 << log2n
+        for L in (1, 3, 7, 15, 127):
+            hist = torch.zeros(2 * L + 1, dtype=torch.int64, device="cuda")
+            lp = torch.full((2 * L + 1,), 1.0 / (2 * L + 1), dtype=torch.float32, device="cuda")
+            lp[L] *= 1.5
+            for alpha in (1.0, 100.0, 1e4):
+                P = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01)
+                Pr = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01, lp)
+
+                def mk(kind, PP=P):
+                    def make(o):
+                        xs, gs, ys, ix = x[o:o + n], g[o:o + n], y[o:o + n], idx[o:o + n]
+                        if kind == "hard":
+                            return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, None)
+                        if kind == "hard_hist":
+                            return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, hist)
+                        if kind == "soft":
+                            return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, None, None)
+                        if kind == "soft_idx_hist":
+                            return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, ix, hist)
+                        return lambda: cdl.cdl_quantize_backward(xs, gs, n, PP, ys, s[0:1], s[1:2])
+                    return make
+                passes = {"hard": (5, mk("hard")), "hard_hist": (5, mk("hard_hist")), "soft": (8, mk("soft")),
+                          "soft_idx_hist": (9, mk("soft_idx_hist")), "backward": (12, mk("backward")),
+                          "backward_rate": (12, mk("backward", Pr))}
+                if alpha != 1.0:
+                    passes.pop("hard"), passes.pop("hard_hist")      # the hard passes do not depend on alpha
+                for name, (bpe, make) in passes.items():
+                    ms = timed(make, n)
+                    gbs = n * bpe / (ms * 1e-3) / 1e9
+                    rows.append({"log2n": log2n, "L": L, "alpha": alpha, "pass": name, "ms": round(ms, 4),
+                                 "Gelem_per_s": round(n / (ms * 1e-3) / 1e9, 2), "GBps": round(gbs, 1),
+                                 "hbm_frac_measured": round(gbs / hbm, 4), "hbm_frac_8TBps": round(gbs / 8000.0, 4)})
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "peak_hbm_gbs": hbm, "peak_source": pk_kind,
+                      "data": "synthetic", "config": {"workload": "quantizer_sweep", "max_log2n": args.sweep_max_log2n}}),
+          flush=True)
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -58,6 +58,8 @@ int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out)
     memset(&d, 0, sizeof d);
     d.q = p->q;
     d.half_q = 0.5f * p->q;
+    d.rq = (float)(1.0 / (double)p->q);
+    d.fast_div = (p->q > 1e-30f && p->q < 1e30f) ? 1 : 0;
     d.lo = p->lo;
     d.hi = p->hi;
     d.nlev = (int)nlev;

@@ -12,6 +12,8 @@ namespace cdl {
 struct QuantDev {
     float q;          // step size
     float half_q;     // q / 2 (exact)
+    float rq;         // RN(1/q)
+    int fast_div;     // q and 1/q are normal numbers well inside the exponent range: x * rq may stand in for x / q
     float flo, fhi;   // index range as floats
     int lo, hi, nlev;
     float c1;         // alpha * q * log2(e): the logit of level kn+j relative to level kn is -c1 * j * (j q - 2 d)

@@ -37,6 +37,9 @@ constexpr int kThreads = 256;
 constexpr int kBatch = 4;  // float4 loads in flight per thread
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
+// |quotient - nearest integer| above this may be a rounding tie once the 3-ulp error of the reciprocal product is
+// allowed for: indices lie in [-128, 255], where an ulp is at most 2^-16; 0.5 - 2^-12 leaves 16 ulp of margin.
+constexpr float kTieGuard = 0.5f - 0.000244140625f;
 
 enum QuantPath { PATH_NEAR3 = 0, PATH_WIN5 = 1, PATH_LOOP = 2 };
 
@@ -90,11 +93,17 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
 {
     ElemOut o;
     const float q = P.q;
-    // ---- hard index: the defining binary32 expression; a NaN quotient clamps to lo
-    const float u = __fdiv_rn(x, q);
-    const float c = fminf(fmaxf(u, P.flo), P.fhi);
-    const float t = __fadd_rn(c, kMagic);
+    // ---- hard index: rint(clamp(RN(x / q))), a NaN quotient clamps to lo.  x * RN(1/q) is within 3 ulp of the
+    // correctly rounded quotient, so both round to the same integer unless the quotient lies within a few ulp
+    // of a half-integer; only then (about 5 elements in 10^4) is the IEEE division itself evaluated.
+    float c = fminf(fmaxf(P.fast_div ? __fmul_rn(x, P.rq) : __fdiv_rn(x, q), P.flo), P.fhi);
+    float t = __fadd_rn(c, kMagic);
     float kn = __fsub_rn(t, kMagic);
+    if (P.fast_div && fabsf(__fsub_rn(c, kn)) > kTieGuard) {
+        c = fminf(fmaxf(__fdiv_rn(x, q), P.flo), P.fhi);
+        t = __fadd_rn(c, kMagic);
+        kn = __fsub_rn(t, kMagic);
+    }
     int ki = __float_as_int(t) - kMagicBits;
     o.k0 = ki;
     o.y = 0.0f;
@@ -378,8 +387,9 @@ int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int6
     }
     const int sms = sm_count();
     if (sms <= 0) return CDL_ERR_LAUNCH;
-    const int64_t work = (n4 > 0) ? n4 : n;   // float4 groups, or single elements on the scalar path
-    int64_t blocks = (work + (int64_t)kThreads * kBatch - 1) / ((int64_t)kThreads * kBatch);
+    // one float4 group (or one scalar element) per thread until the device is full, then kBatch in flight each
+    const int64_t work = (n4 > 0) ? n4 : n;
+    int64_t blocks = (work + kThreads - 1) / kThreads;
     const int64_t cap = (int64_t)sms * per_sm;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
