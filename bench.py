@@ -39,8 +39,8 @@ NCU_TRAFFIC_BYTES = {}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="cdl", choices=["cdl", "reference"])
     ap.add_argument("--workload", default="resnet18_layer3_conv",
                     choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny"])
@@ -101,7 +101,7 @@ def call_model(case, n_x):
 
 
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
@@ -120,8 +120,11 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t0=None, t1=None):
+        """Median SM clock and throttle reasons of the samples taken between wall-clock times t0 and t1 (the timed
+        region); if the region was too short to contain a sample, of all samples since start()."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "timed region"}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -129,26 +132,27 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         try:
             for line in open(self.path):
                 f = [c.strip() for c in line.split(",")]
                 if len(f) < 9:
                     continue
                 try:
-                    sm.append(float(f[1]))
-                    mx.append(float(f[2]))
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[1]), float(f[2]), [n for n, v in zip(names, f[5:9]) if v.lower().startswith("active")]))
                 except ValueError:
                     continue
-                for name, v in zip(names, f[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1]
+        if not inside:
+            inside, out["window"] = rows, "warm-up + timed region (timed region shorter than the sampling period)"
+        if inside:
+            out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                       reasons=sorted({n for r in inside for n in r[3]}), samples=len(inside))
         return out
 
 
@@ -332,6 +336,7 @@ def main():
 
     import paper_2501_09849_b200 as cdl
     from paper_2501_09849_b200 import build as cdl_build
+    from paper_2501_09849_b200 import sharding
     from paper_2501_09849_b200.layer import CALLS, CdlLayerStep
 
     if not torch.cuda.is_available():
@@ -363,25 +368,23 @@ def main():
 
     def exchange():
         # data-parallel exchange of a step: the weight-side results are sums over the global batch
-        if world > 1:
-            dist.all_reduce(step.dW)
-            dist.all_reduce(step.hist_x)
-            dist.all_reduce(step.scalars)
+        sharding.exchange(dist, world, step.dW, step.hist_x, step.scalars)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step.run()
         exchange()
     torch.cuda.synchronize()
 
     # ---- timed region: device-resident inputs
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(args.steps)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     t_start.record(stream)
     for it in range(args.steps):
         ev = iter(events[it])
@@ -389,9 +392,10 @@ def main():
         exchange()
     t_end.record(stream)
     torch.cuda.synchronize()
+    wall1 = time.time()
     if world > 1:
         dist.barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
     per_call_ms = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(args.steps)) / args.steps
                    for i, name in enumerate(CALLS)}
