@@ -29,6 +29,7 @@ if str(ROOT) not in sys.path:
 METRIC = "quantizer Gelem/s (% of HBM peak); CDL layer fwd+bwd ms and int8 TOPS"
 UNIT = "Gelem/s"
 G_STD = 1e-2                 # standard deviation of the synthetic dL/dY
+CPU_BASELINE_SECONDS = 20.0   # host time the cpu_baseline leg may spend (it samples the step to fit)
 INT8_OVER_BF16 = 2.0         # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture, keyed by
@@ -156,36 +157,39 @@ class ClockSampler:
         return out
 
 
-def oracle_step_sample(case, host, n_x_sample=1 << 24, rows=1 << 16):
-    """Times the CPU oracle, as it stands, on a bounded sample of one step and scales every part to the full
-    step by the units it processed.  Returns (estimated seconds of a full step, description, threads)."""
+def oracle_step_sample(case, host, frac=1.0):
+    """Times the CPU oracle, as it stands, on a fraction `frac` of one step (leading elements / rows of every
+    tensor) and scales every part to the full step by the units it processed.
+    Returns (estimated seconds of a full step, description, threads, wall seconds actually spent)."""
     import numpy as np
     import oracle
     f32 = np.float32
     wq, aq = case.wq, case.aq
-    n_x = host["x"].size
-    ns = min(n_x, n_x_sample)
+    n_x, n_w = host["x"].size, host["w"].size
+    ns = int(max(min(n_x, 1 << 10), min(n_x, round(frac * n_x))))
+    nw = int(max(min(n_w, 1 << 10), min(n_w, round(frac * n_w))))
+    r = int(max(2, min(case.M, round(frac * case.M))))
     xs, gs = host["x"][:ns], host["gx_in"][:ns]
-    w = host["w"]
+    w, ws = host["w"], host["w"][:nw]
     t_total = 0.0
+    t_wall0 = time.perf_counter()
 
     def timed(fn, scale):
         nonlocal t_total
         t0 = time.perf_counter()
-        r = fn()
+        out = fn()
         t_total += (time.perf_counter() - t0) * scale
-        return r
+        return out
 
-    sx = n_x / ns
-    timed(lambda: oracle.soft(w, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window), 1.0)
-    _, hw = timed(lambda: oracle.hard(w, f32(wq.q), wq.lo, wq.hi), 1.0)
+    sx, sw, sm = n_x / ns, n_w / nw, case.M / r
+    timed(lambda: oracle.soft(ws, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window), sw)
+    _, hw = timed(lambda: oracle.hard(ws, f32(wq.q), wq.lo, wq.hi), sw)
     _, pw, _ = timed(lambda: oracle.entropy(hw), 1.0)
     timed(lambda: oracle.soft(xs, f32(aq.q), aq.lo, aq.hi, f32(aq.alpha), aq.window), sx)
     _, hx = timed(lambda: oracle.hard(xs, f32(aq.q), aq.lo, aq.hi), sx)
     _, px, _ = timed(lambda: oracle.entropy(hx), 1.0)
-    r = min(rows, case.M)
-    sm = case.M / r
-    A, W8 = host["A_idx"][:r], oracle.hard(w, f32(wq.q), wq.lo, wq.hi)[0].reshape(case.K, case.N).astype(np.int8)
+    W8 = oracle.hard(w, f32(wq.q), wq.lo, wq.hi)[0].reshape(case.K, case.N).astype(np.int8)   # operand set-up, untimed
+    A = host["A_idx"][:r]
     timed(lambda: oracle.gemm_fwd(A, W8), sm)
     q_g = 4.0 * G_STD / 127.0
     gi, _ = timed(lambda: oracle.hard(host["dY"][:r], f32(q_g), -127, 127), sm)
@@ -193,11 +197,11 @@ def oracle_step_sample(case, host, n_x_sample=1 << 24, rows=1 << 16):
     timed(lambda: oracle.gemm_dx(G8, W8), sm)
     dW = timed(lambda: oracle.gemm_dw(A, G8), sm)
     timed(lambda: oracle.backward(xs, gs, f32(aq.q), aq.lo, aq.hi, f32(aq.alpha), aq.window, f32(aq.rate_weight), px), sx)
-    gw = (dW.astype(np.float64) * q_g * aq.q).astype(f32).reshape(-1)
-    timed(lambda: oracle.backward(w, gw, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window, f32(wq.rate_weight), pw), 1.0)
-    desc = (f"oracle on {ns} of {n_x} activations (quantize, backward), all {w.size} weights, "
+    gw = (dW.astype(np.float64) * q_g * aq.q).astype(f32).reshape(-1)[:nw]
+    timed(lambda: oracle.backward(ws, gw, f32(wq.q), wq.lo, wq.hi, f32(wq.alpha), wq.window, f32(wq.rate_weight), pw), sw)
+    desc = (f"oracle on {ns} of {n_x} activations and {nw} of {n_w} weights (quantize, entropy, backward), "
             f"{r} of {case.M} GEMM rows (fwd, dX, dW); each part scaled to the full step")
-    return t_total, desc, oracle.threads()
+    return t_total, desc, oracle.threads(), time.perf_counter() - t_wall0
 
 
 def run_reference(args, rank):
@@ -212,11 +216,15 @@ def run_reference(args, rank):
     _, hist_x = oracle.hard(x.reshape(-1)[: 1 << 20], f32(case.aq.q), case.aq.lo, case.aq.hi)
     host = host_inputs(case, w, x, hist_x)
     quant_elems = 2 * (w.size + x.size) + case.M * case.N
+    # size the per-step sample so that warm-up + K steps take about 60 s of host time whatever K is
+    _, _, _, wall_cal = oracle_step_sample(case, host, frac=1.0 / 256)
+    budget = 60.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, budget / max(256.0 * wall_cal, 1e-9))
     for _ in range(max(args.warmup, 0)):
-        oracle_step_sample(case, host, n_x_sample=1 << 14, rows=2)
+        oracle_step_sample(case, host, frac)
     ts = []
     for _ in range(args.steps):
-        t, desc, thr = oracle_step_sample(case, host, n_x_sample=1 << 22, rows=2048)
+        t, desc, thr, _ = oracle_step_sample(case, host, frac)
         ts.append(t)
     t_step = sum(ts) / len(ts)
     value = quant_elems / t_step / 1e9
@@ -483,7 +491,7 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            t_cpu, desc, thr = oracle_step_sample(case, host)
+            t_cpu, desc, thr, _ = oracle_step_sample(case, host, frac=min(1.0, CPU_BASELINE_SECONDS / max(256.0 * oracle_step_sample(case, host, 1.0 / 256)[3], 1e-9)))
             line["cpu_baseline"] = {"value": quant_elems / t_cpu / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle",
                                     "sample": desc, "ms_per_step_estimate": t_cpu * 1e3}
         print(json.dumps(line), flush=True)
