@@ -34,7 +34,11 @@ INT8_OVER_BF16 = 2.0         # nominal dense int8 : bf16 tensor throughput on B2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture, keyed by
 # (workload, call); None until captured for the current kernel.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/index_gemm_tc_resnet18_layer3_conv.md: 13.5 MB read + 403.3 MB written while the kernel ran (the
+    # write-back of the 462 MB output continues after it ends)
+    ("resnet18_layer3_conv", "qlinear_bwd_dx"): 416.8e6,
+}
 
 
 def parse_args():
