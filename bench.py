@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
     ap.add_argument("--sweep-max-log2n", type=int, default=28)
+    ap.add_argument("--gemm", type=int, nargs=3, metavar=("M", "K", "N"), action="append",
+                    help="index-GEMM-only timing of the forward, dX and dW products for this shape (repeatable)")
     return ap.parse_args()
 
 
@@ -330,10 +332,76 @@ def run_sweep(args):
           flush=True)
 
 
+def run_gemm(args):
+    """Index GEMMs alone: forward, dX and dW for each requested (M, K, N), 4-bit activation / weight indices and
+    8-bit gradient indices drawn uniformly on the device, float outputs; operands are rotated over several
+    buffer sets when one set would fit in L2."""
+    import torch
+
+    import paper_2501_09849_b200 as cdl
+    from paper_2501_09849_b200 import build as cdl_build
+    cdl_build.build()
+    cdl.load_library()
+    torch.cuda.set_device(0)
+    pk, pk_kind = peaks()
+    hbm = float(pk["hbm_gbs"])
+    int8_tops = float(pk["bf16_tflops"]) * INT8_OVER_BF16          # kernels timed alone: burst figure
+    stream = torch.cuda.current_stream()
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    a, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    out = []
+    for M, K, N in args.gemm:
+        set_bytes = M * K + K * N + M * N + 4 * (M * N + M * K + K * N)
+        nset = max(1, min(4, (400 << 20) // set_bytes + 1))
+        sets = []
+        for _ in range(nset):
+            A = torch.randint(0, 16, (M, K), device="cuda", generator=gen, dtype=torch.uint8)
+            W = torch.randint(-7, 8, (K, N), device="cuda", generator=gen, dtype=torch.int8)
+            G = torch.randint(-127, 128, (M, N), device="cuda", generator=gen, dtype=torch.int8)
+            sets.append((A, W, G, torch.empty((M, N), dtype=torch.float32, device="cuda"),
+                         torch.empty((M, K), dtype=torch.float32, device="cuda"),
+                         torch.empty((K, N), dtype=torch.float32, device="cuda")))
+        nb = max(cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_FWD, M, N, K), cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K))
+        ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        calls = {
+            "fwd": lambda t: cdl.cdl_qlinear_fwd(t[0], K, a, t[1], N, w, M, N, K, None, t[3], None, ws, nb),
+            "dx": lambda t: cdl.cdl_qlinear_bwd(t[2], N, g, None, K, None, t[1], N, w, M, N, K, None, t[4], None, None, ws, nb),
+            "dw": lambda t: cdl.cdl_qlinear_bwd(t[2], N, g, t[0], K, a, None, N, None, M, N, K, None, None, None, t[5], ws, nb),
+        }
+        bytes_ = {"fwd": M * K + K * N + 4 * M * N, "dx": M * N + K * N + 4 * M * K, "dw": M * K + M * N + 4 * K * N}
+        row = {"M": M, "K": K, "N": N, "buffer_sets": nset}
+        for name, fn in calls.items():
+            for t in sets:
+                fn(t)
+            reps = max(4, min(40, args.steps))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(reps):
+                fn(sets[i % nset])
+            e1.record(stream)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            ops = 2.0 * M * K * N
+            t_tensor, t_hbm = ops / (int8_tops * 1e12), bytes_[name] / (hbm * 1e9)
+            row[name] = {"ms": round(ms, 5), "int8_TOPS": round(ops / (ms * 1e-3) / 1e12, 1),
+                         "int8_frac_of_peak": round(ops / (ms * 1e-3) / 1e12 / int8_tops, 4),
+                         "GBps": round(bytes_[name] / (ms * 1e-3) / 1e9, 1), "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                         "roofline_frac": round(max(t_tensor, t_hbm) / (ms * 1e-3), 4)}
+        row["status"] = cdl.cdl_workspace_status(ws, check=False)
+        out.append(row)
+        del sets
+    print(json.dumps({"metric": METRIC, "unit": "int8 TOPS", "gemm": out, "int8_peak_tops": int8_tops,
+                      "peak_source": f"{pk_kind} burst bf16 x {INT8_OVER_BF16:g} (nominal int8:bf16)", "peak_hbm_gbs": hbm,
+                      "data": "synthetic", "config": {"workload": "index_gemm"}}), flush=True)
+
+
 def main():
     args = parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.gemm:
+        run_gemm(args)
         return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
