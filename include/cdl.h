@@ -153,7 +153,9 @@ int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits,
  *   acc_out [dev] M x N int32 (ld N), nullable.  y_out [dev] M x N floats (ld N), nullable.
  *   bias [dev] N floats, nullable.  At least one of acc_out, y_out.
  *   ws [dev]: cdl_workspace_bytes(CDL_OP_QLINEAR_FWD, M, N, K) bytes, 256-byte aligned.
- * CDL_ERR_OVERFLOW_RISK when K * max|a| * max|w| >= 2^31 for the declared index ranges.
+ * CDL_ERR_OVERFLOW_RISK when acc_out is requested and K * max|a| * max|w| >= 2^31 for the declared index ranges
+ * (the float output alone is always available: long reductions are then cut into exact int32 parts that are
+ * summed in int64 before the single conversion to float).
  */
 int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a,
                     const void *W_idx, int64_t ldw, const cdl_index_desc *w,
@@ -173,7 +175,9 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a,
  *   dXacc, dWacc [dev] int32 (ld K, ld N), dX, dW [dev] floats; each nullable.  A_idx may be NULL
  *   when neither dWacc nor dW is wanted, W_idx when neither dXacc nor dX is.
  *   ws [dev]: cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K) bytes, 256-byte aligned.
- * CDL_ERR_OVERFLOW_RISK when N*max|g|*max|w| or M*max|a|*max|g| reaches 2^31.
+ * CDL_ERR_OVERFLOW_RISK when dXacc (dWacc) is requested and N*max|g|*max|w| (M*max|a|*max|g|) reaches 2^31; the
+ * float outputs alone are always available (exact int32 parts summed in int64, as for cdl_qlinear_fwd), which is
+ * what lets dW reduce over millions of rows.
  */
 int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
                     const void *A_idx, int64_t lda, const cdl_index_desc *a,

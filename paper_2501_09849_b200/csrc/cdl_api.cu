@@ -252,7 +252,7 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, con
     if (bad_f32_ptr(acc_out) || bad_f32_ptr(y_out) || bad_f32_ptr(bias)) return CDL_ERR_ALIGN;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_workspace_bytes(CDL_OP_QLINEAR_FWD, M, N, K))
         return CDL_ERR_WORKSPACE;
-    if (overflow_risk(K, ra, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (acc_out != nullptr && overflow_risk(K, ra, rw)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
@@ -260,8 +260,8 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, con
         return CDL_ERR_LAUNCH;
     }
     const float scale = (a->q * w->q);
-    GemmOperand X{A_idx, lda, 1, ra.is_unsigned};
-    GemmOperand Y{W_idx, 1, ldw, false};
+    GemmOperand X{A_idx, lda, 1, ra.is_unsigned, (int)ra.absmax};
+    GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
     return launch_index_gemm_tc(X, Y, M, N, K, acc_out, y_out, scale, bias, static_cast<char *>(ws) + kStatusBytes,
                                 static_cast<int *>(ws), st);
 }
@@ -292,8 +292,8 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
     if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K))
         return CDL_ERR_WORKSPACE;
-    if (want_dx && overflow_risk(N, rg, rw)) return CDL_ERR_OVERFLOW_RISK;
-    if (want_dw && overflow_risk(M, ra, rg)) return CDL_ERR_OVERFLOW_RISK;
+    if (dXacc != nullptr && overflow_risk(N, rg, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (dWacc != nullptr && overflow_risk(M, ra, rg)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
@@ -302,16 +302,16 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
     }
     if (want_dx) {
         // dX[m,k] = sum_n G[m,n] W[k,n]
-        GemmOperand X{G_idx, ldg, 1, false};
-        GemmOperand Y{W_idx, ldw, 1, false};
+        GemmOperand X{G_idx, ldg, 1, false, (int)rg.absmax};
+        GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
         rc = launch_index_gemm_tc(X, Y, M, K, N, dXacc, dX, (g->q * w->q), nullptr,
                                   static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st);
         if (rc != CDL_OK) return rc;
     }
     if (want_dw) {
         // dW[k,n] = sum_m A[m,k] G[m,n]
-        GemmOperand X{A_idx, 1, lda, ra.is_unsigned};
-        GemmOperand Y{G_idx, 1, ldg, false};
+        GemmOperand X{A_idx, 1, lda, ra.is_unsigned, (int)ra.absmax};
+        GemmOperand Y{G_idx, 1, ldg, false, (int)rg.absmax};
         rc = launch_index_gemm_tc(X, Y, K, N, M, dWacc, dW, (g->q * a->q), nullptr,
                                   static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st);
         if (rc != CDL_OK) return rc;

@@ -56,6 +56,8 @@ struct TcParams {
     const float *bias;
     int *status;
     int tma_f, tma_acc;     // the float / int32 output goes through shared memory and TMA
+    int slab_rows;          // 0: splits add into one I x J buffer.  > 0: split s stores its partial tile into rows
+                            // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -350,6 +352,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         for (int u = blockIdx.x; u < units; u += gridDim.x, ++tcount) {
             const int tile = u / P.splits;
             const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
+            const int slab_row0 = (u % P.splits) * P.slab_rows;     // 0 unless partial tiles go to per-split slabs
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
             // the four warps must agree on the outcome: the staging code below uses CTA-level named barriers
@@ -371,12 +374,17 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const bool in_rows = row < P.I;
                 if (P.splits > 1) {
                     if (P.tma_acc) {
-                        stage_and_send(v, &map_acc, true, col0, ti * TM);
+                        stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + ti * TM);
                     } else if (in_rows) {
+                        int32_t *dst = P.acc_out + off + (long long)slab_row0 * P.J;
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c < ncol)
-                                asm volatile("red.global.add.s32 [%0], %1;" ::"l"(P.acc_out + off + c), "r"(v[c]) : "memory");
+                            if (c < ncol) {
+                                if (P.slab_rows == 0)
+                                    asm volatile("red.global.add.s32 [%0], %1;" ::"l"(dst + c), "r"(v[c]) : "memory");
+                                else
+                                    dst[c] = (int)v[c];
+                            }
                     }
                     continue;
                 }
@@ -452,6 +460,21 @@ __global__ void scale_acc_kernel(const int32_t *__restrict__ acc, float *__restr
     }
 }
 
+// float output of a split run whose partial sums sit in per-split slabs: the slabs are summed in int64 (each
+// slab is exact in int32, the total need not be), converted once and scaled.
+__global__ void sum_slabs_kernel(const int32_t *__restrict__ slabs, int splits, long long slab_elems, float *__restrict__ f,
+                                 long long n, int J, float scale, const float *__restrict__ bias)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        long long acc = 0;
+        for (int sp = 0; sp < splits; ++sp) acc += (long long)slabs[sp * slab_elems + i];
+        float v = __fmul_rn(__ll2float_rn(acc), scale);
+        if (bias != nullptr) v = __fadd_rn(v, bias[i % J]);
+        f[i] = v;
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -503,8 +526,9 @@ bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t out
 }  // namespace
 
 namespace {
-// Split of the reduced dimension: only when the tiles alone cannot occupy half of the device.
-void plan(int I, int J, int R, int *TN_out, int *splits_out)
+// Split of the reduced dimension: when the tiles alone cannot occupy half of the device, and always into at
+// least min_splits parts (the caller's bound that keeps every part's int32 partial sums exact).
+void plan(int I, int J, int R, int min_splits, int *TN_out, int *splits_out)
 {
     int TN = 256;
     while (TN > 16 && TN / 2 >= J) TN /= 2;
@@ -517,18 +541,37 @@ void plan(int I, int J, int R, int *TN_out, int *splits_out)
         if (splits > max_splits) splits = max_splits;
         if (splits < 1) splits = 1;
     }
+    if (splits < min_splits) splits = min_splits;
     *TN_out = TN;
     *splits_out = splits;
 }
+
+// Parts the reduced dimension must be cut into so that a part's sum of |x| * |y| stays below 2^31 (whole r-blocks).
+int min_exact_splits(int R, long long xmax, long long ymax)
+{
+    const long long per_term = xmax * ymax > 0 ? xmax * ymax : 1;
+    const long long rows = (((long long)1 << 31) - 1) / per_term;     // rows one part may hold
+    const long long rb_max = rows / BR;
+    if (rb_max < 1) return -1;                                        // cannot happen for byte operands
+    const long long rblocks = (R + BR - 1) / BR;
+    return (int)((rblocks + rb_max - 1) / rb_max);
+}
 }  // namespace
 
-// Scratch bytes the product needs when no int32 output is passed: the int32 accumulation buffer of a split run.
+// Scratch bytes a product may need: the int32 accumulation buffer of a split run and, when the reduced dimension
+// is long enough that its int32 total could overflow for byte operands of the widest range, the per-split slabs.
 size_t tc_gemm_scratch_bytes(int I, int J, int R)
 {
     int TN, splits;
-    plan(I, J, R, &TN, &splits);
-    if (splits <= 1) return 0;
-    return ((size_t)I * (size_t)J * sizeof(int32_t) + 255u) & ~(size_t)255u;
+    plan(I, J, R, 1, &TN, &splits);
+    size_t need = 0;
+    if (splits > 1) need = (size_t)I * (size_t)J * sizeof(int32_t);
+    if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
+        plan(I, J, R, min_exact_splits(R, 255, 128), &TN, &splits);
+        const size_t slab = (size_t)((I + TM - 1) / TM) * TM * (size_t)J * sizeof(int32_t);
+        if (slab * splits > need) need = slab * splits;
+    }
+    return (need + 255u) & ~(size_t)255u;
 }
 
 // X: the operand whose non-reduced dimension indexes output rows; Y: output columns.  An operand is MN-major
@@ -544,9 +587,15 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.I = I;
     P.J = J;
     P.R = R;
+    // Exactness: a part of the reduced dimension is summed in int32, so |sum| <= rows * xmax * ymax must stay
+    // below 2^31 per part.  When the whole dimension does not satisfy that, it is cut into enough parts, each part
+    // keeps its own slab, and the slabs are summed in int64 (float output only).
+    const bool wide = (long long)R * X.absmax * Y.absmax >= ((long long)1 << 31);
+    if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
     int TN, splits;
-    plan(I, J, R, &TN, &splits);
+    plan(I, J, R, wide ? min_exact_splits(R, X.absmax, Y.absmax) : 1, &TN, &splits);
     P.TN = TN;
+    P.slab_rows = wide ? ((I + TM - 1) / TM) * TM : 0;
     P.tiles_i = (I + TM - 1) / TM;
     P.tiles_j = (J + TN - 1) / TN;
     P.rblocks = (R + BR - 1) / BR;
@@ -565,7 +614,10 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.f_out = f_out;
     P.acc_out = acc_out;
     const long long n_out = (long long)I * J;
-    if (splits > 1) {
+    if (wide) {
+        P.acc_out = static_cast<int32_t *>(scratch);       // slabs: every element is written, nothing to clear
+        if (P.acc_out == nullptr) return CDL_ERR_WORKSPACE;
+    } else if (splits > 1) {
         if (P.acc_out == nullptr) P.acc_out = static_cast<int32_t *>(scratch);
         if (P.acc_out == nullptr) return CDL_ERR_WORKSPACE;
         if (cudaMemsetAsync(P.acc_out, 0, (size_t)n_out * sizeof(int32_t), stream) != cudaSuccess) {
@@ -586,12 +638,13 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const bool out_ok = TN >= 32 && (J & 3) == 0;
     P.tma_f = 0;
     P.tma_acc = 0;
-    if (out_ok && splits == 1 && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
+    if (out_ok && splits == 1 && !wide && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
         ok = ok && encode_out_map(&map_f, f_out, (uint64_t)J, (uint64_t)I, true);
         P.tma_f = 1;
     }
     if (out_ok && P.acc_out != nullptr && (reinterpret_cast<uintptr_t>(P.acc_out) & 15u) == 0) {
-        ok = ok && encode_out_map(&map_acc, P.acc_out, (uint64_t)J, (uint64_t)I, false);
+        const uint64_t acc_rows = wide ? (uint64_t)splits * (uint64_t)P.slab_rows : (uint64_t)I;
+        ok = ok && encode_out_map(&map_acc, P.acc_out, (uint64_t)J, acc_rows, false);
         P.tma_acc = 1;
     }
     if (!ok) return CDL_ERR_LAUNCH;
@@ -610,9 +663,12 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const int grid = (int)(units < sms ? units : sms);
     index_gemm_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
-    if (splits > 1 && f_out != nullptr) {
+    if (f_out != nullptr && (splits > 1 || wide)) {
         const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
-        scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias);
+        if (wide)
+            sum_slabs_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, splits, (long long)P.slab_rows * J, f_out, n_out, J, scale, bias);
+        else
+            scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias);
         if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     }
     return CDL_OK;
@@ -672,8 +728,8 @@ extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const 
         (void)cudaGetLastError();
         return CDL_ERR_LAUNCH;
     }
-    GemmOperand X{A_idx, 1, lda, a->lo >= 0};
-    GemmOperand Y{G_idx, 1, ldg, false};
+    GemmOperand X{A_idx, 1, lda, a->lo >= 0, (int)amax};
+    GemmOperand Y{G_idx, 1, ldg, false, (int)gmax};
     return launch_index_gemm_tc(X, Y, K, N, M, nullptr, dW, g->q * a->q, nullptr, base + kStaticStatusBytes,
                                 reinterpret_cast<int *>(base), st);
 }

@@ -47,6 +47,7 @@ struct GemmOperand {
     int64_t stride_outer;   // stride of the non-reduced dimension (i for X, j for Y)
     int64_t stride_red;     // stride of the reduced dimension r
     bool is_unsigned;
+    int absmax;             // bound on |entry| (from the operand's declared index range)
 };
 
 // Tensor-core index GEMM (TMA + tcgen05 + TMEM); operands need 16-byte aligned bases and pitches.

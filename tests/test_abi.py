@@ -100,7 +100,7 @@ def test_qlinear_argument_errors_need_no_device(lib):
     assert f(p, 256, a, p, 128, w, **ok, y_out=p, ws=ws + 16, ws_bytes=nb, check=False) == WS
     assert f(p, 256, a, p, 128, w, **ok, y_out=p, ws=ws, ws_bytes=nb - 1, check=False) == WS
     big = 1 << 18
-    assert f(p, big, D(1.0, 0, 255), p, 128, D(1.0, -128, 127), M=64, N=128, K=big, y_out=p, ws=ws,
+    assert f(p, big, D(1.0, 0, 255), p, 128, D(1.0, -128, 127), M=64, N=128, K=big, acc_out=p, ws=ws,
              ws_bytes=cdl.cdl_workspace_bytes(1, 64, 128, big), check=False) == OVF
     b = cdl.cdl_qlinear_bwd
     nbb = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, 64, 128, 256)
@@ -110,7 +110,7 @@ def test_qlinear_argument_errors_need_no_device(lib):
     assert b(p, 120, g, p, 256, a, p, 128, w, **ok, dX=p, ws=ws, ws_bytes=nbb, check=False) == ARG
     assert b(p, 128, g, p, 256, a, p, 128, w, **ok, dX=p, ws=ws, ws_bytes=0, check=False) == WS
     M = 1 << 20
-    assert b(p, 128, g, p, 256, D(1.0, 0, 255), p, 128, w, M=M, N=128, K=256, dW=p, ws=ws,
+    assert b(p, 128, g, p, 256, D(1.0, 0, 255), p, 128, w, M=M, N=128, K=256, dWacc=p, ws=ws,
              ws_bytes=cdl.cdl_workspace_bytes(2, M, 128, 256), check=False) == OVF
 
 

@@ -189,3 +189,28 @@ def test_resnet18_layer3_shape_sampled_compare(torch):
     # properties that hold at any size: column sums of the forward accumulators
     colsum = A.astype(np.int64).sum(axis=0) @ W.astype(np.int64)
     assert np.array_equal(acc.astype(np.int64).sum(axis=0), colsum)
+
+
+def test_long_reduction_beyond_int32_is_summed_exactly(torch):
+    # dW over M rows whose worst-case (and, for the constant operands, actual) total exceeds 2^31: the float output
+    # must equal float(int64 sum) * scale; asking for the int32 accumulators is refused.
+    M, K, N = 70001, 160, 48
+    a, g = cdl.IndexDesc(0.25, 0, 255), cdl.IndexDesc(1e-3, -127, 127)
+    for kind in ("constant", "random"):
+        if kind == "constant":
+            A = np.full((M, K), 255, dtype=np.uint8)
+            G = np.full((M, N), 127, dtype=np.int8)
+            G[:, 1::2] = -127
+        else:
+            A = inputs.uniform_indices((M, K), 0, 255, seed=11)
+            G = inputs.uniform_indices((M, N), -127, 127, seed=12)
+        ref = oracle.gemm_dw(A, G)
+        if kind == "constant":
+            assert np.abs(ref).max() >= 2 ** 31
+        out = run_bwd(torch, G, A, None, g, a, None, want=("dW",))
+        assert np.array_equal(out["dW"], scaled(ref, g.q, a.q))
+    ldg, lda = ld16(N), ld16(K)
+    nb = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K)
+    buf = torch.zeros(max(nb, M * lda), dtype=torch.uint8, device="cuda")
+    rc = cdl.cdl_qlinear_bwd(buf, ldg, g, buf, lda, a, None, ldg, None, M, N, K, None, None, buf, None, buf, nb, check=False)
+    assert rc == -5
