@@ -48,7 +48,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="cdl", choices=["cdl", "reference"])
     ap.add_argument("--workload", default="resnet18_layer3_conv",
-                    choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny"])
+                    choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny", "resnet18_b256"])
+    ap.add_argument("--batch", type=int, default=256, help="batch size of the resnet18_b256 workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
@@ -395,8 +396,111 @@ def run_gemm(args):
                       "data": "synthetic", "config": {"workload": "index_gemm"}}), flush=True)
 
 
+def run_network(args):
+    """Whole ResNet-18 (224x224) as a sequence of CDL layer steps: every conv and the FC layer with its true im2col
+    GEMM shape, 3-bit weights (step = std(w) / 3), 4-bit activations (step from the mean magnitude), window of 5.
+    Inputs are drawn on the device (seeded); each layer owns its buffers, so a step touches ~40 GB at batch 256."""
+    import torch
+
+    import paper_2501_09849_b200 as cdl
+    from paper_2501_09849_b200 import build as cdl_build
+    from paper_2501_09849_b200 import inputs
+    from paper_2501_09849_b200.layer import CALLS, CdlLayerStep
+    cdl_build.build()
+    cdl.load_library()
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device="cuda").manual_seed(4)
+    stream = torch.cuda.current_stream()
+    q_g = 4.0 * G_STD / 127.0
+    layers = []
+    for name, M, K, N, n_x in inputs.resnet18_layers(args.batch):
+        Np = (N + 15) // 16 * 16                  # index matrices need 16-byte row pitches: fc's 1000 columns -> 1008
+        w = torch.randn(K * Np, device="cuda", generator=gen) * (2.0 / K) ** 0.5
+        x = torch.randn(n_x, device="cuda", generator=gen).abs_()
+        wq = inputs.Quantizer(float(w.std()) / 3.0, -3, 3, 100.0, 0.01, 0)
+        xq = inputs.Quantizer(float(2.0 * x.mean() / 8.0 ** 0.5), 0, 15, 100.0, 0.01, 5)
+        st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g)
+        st.w.copy_(w)
+        st.x.copy_(x)
+        del w, x
+        # im2col index matrix drawn from the quantized activations' own level histogram
+        hist = torch.zeros(16, dtype=torch.int64, device="cuda")
+        cdl.cdl_quantize_hard(st.x, n_x, cdl.QuantParams(xq.q, 0, 15), None, hist)
+        cdf = torch.cumsum(hist.double() / float(n_x), 0).float()
+        rows = max(1, (1 << 26) // K)
+        for r0 in range(0, M, rows):
+            r1 = min(M, r0 + rows)
+            u = torch.rand((r1 - r0, K), device="cuda", generator=gen)
+            st.A_idx[r0:r1, :K] = torch.searchsorted(cdf, u).clamp_(max=15).to(torch.uint8)
+        st.dY.copy_(torch.randn((M, Np), device="cuda", generator=gen) * G_STD)
+        st.gx_in.copy_(torch.randn(n_x, device="cuda", generator=gen))
+        layers.append((name, M, K, N, n_x, st))
+    torch.cuda.synchronize()
+
+    def run_all(mark=None):
+        for li, (_, _, _, _, _, st) in enumerate(layers):
+            st.run(mark=(lambda nm, li=li: mark(li, nm)) if mark else None)
+
+    warm = max(3, min(args.warmup, 5))
+    steps = max(3, min(args.steps, 20))
+    for _ in range(warm):
+        run_all()
+    torch.cuda.synchronize()
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in layers] for _ in range(steps)]
+    cnt = {}
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    wall0 = time.time()
+    t0.record(stream)
+    for it in range(steps):
+        cnt.clear()
+
+        def mark(li, nm, it=it):
+            i = cnt.get(li, 0)
+            ev[it][li][i].record(stream)
+            cnt[li] = i + 1
+        run_all(mark)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop(wall0, time.time())
+    ms_step = t0.elapsed_time(t1) / steps
+    pk, pk_kind = peaks()
+    hbm = float(pk["hbm_gbs"])
+    table, tot_ops, tot_q, gemm_ms, quant_ms = [], 0.0, 0, 0.0, 0.0
+    for li, (name, M, K, N, n_x, st) in enumerate(layers):
+        per = {c: sum(ev[it][li][i].elapsed_time(ev[it][li][i + 1]) for it in range(steps)) / steps for i, c in enumerate(CALLS)}
+        g_ms = per["qlinear_fwd"] + per["qlinear_bwd_dx"] + per["qlinear_bwd_dw"]
+        q_ms = sum(v for c, v in per.items() if c.startswith("quantize"))
+        ops = 6.0 * M * K * N
+        q_el = 2 * (n_x + K * N) + M * N
+        table.append({"layer": name, "M": M, "K": K, "N": N, "ms": round(sum(per.values()), 4), "gemm_ms": round(g_ms, 4),
+                      "gemm_int8_TOPS": round(ops / (g_ms * 1e-3) / 1e12, 1), "quantizer_ms": round(q_ms, 4),
+                      "quantizer_Gelem_per_s": round(q_el / (q_ms * 1e-3) / 1e9, 1),
+                      "status": cdl.cdl_workspace_status(st.ws, check=False)})
+        tot_ops += ops
+        tot_q += q_el
+        gemm_ms += g_ms
+        quant_ms += q_ms
+    print(json.dumps({
+        "metric": METRIC, "value": tot_q / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32+s8",
+        "data": "synthetic",
+        "config": {"workload": "resnet18_b256", "batch": args.batch, "layers": len(layers), "weight_levels": 7,
+                   "activation_levels": 16, "window_x": 5, "l2": "every layer's tensors exceed the 126 MB L2"},
+        "network_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": tot_ops / (gemm_ms * 1e-3) / 1e12,
+        "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": tot_q / (quant_ms * 1e-3) / 1e9,
+        "layers": table, "clocks": clocks, "peak_hbm_gbs": hbm, "peak_source": pk_kind,
+        "e2e": None, "e2e_note": "not measured for this workload (a step's inputs are ~11 GB); see the default workload",
+        "gpu_launches": steps * len(layers) * len(CALLS)}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.workload == "resnet18_b256" and args.impl == "cdl":
+        run_network(args)
+        return
     if args.sweep:
         run_sweep(args)
         return

@@ -138,15 +138,21 @@ def resnet18_layer3_conv(seed: int = 3):
     return case, w, a
 
 
-# ResNet-18 at 224x224, batch 256: every conv and the FC layer as an im2col GEMM (M, K, N).
-RESNET18_GEMMS = (
-    [("conv1", 256 * 112 * 112, 147, 64)]
-    + [(f"layer1.{i}", 256 * 56 * 56, 576, 64) for i in range(4)]
-    + [("layer2.0", 256 * 28 * 28, 576, 128)] + [(f"layer2.{i}", 256 * 28 * 28, 1152, 128) for i in range(1, 4)]
-    + [("layer2.ds", 256 * 28 * 28, 64, 128)]
-    + [("layer3.0", 256 * 14 * 14, 1152, 256)] + [(f"layer3.{i}", 256 * 14 * 14, 2304, 256) for i in range(1, 4)]
-    + [("layer3.ds", 256 * 14 * 14, 128, 256)]
-    + [("layer4.0", 256 * 7 * 7, 2304, 512)] + [(f"layer4.{i}", 256 * 7 * 7, 4608, 512) for i in range(1, 4)]
-    + [("layer4.ds", 256 * 7 * 7, 256, 512)]
-    + [("fc", 256, 512, 1000)]
-)
+def resnet18_layers(batch: int = 256):
+    """ResNet-18 at 224x224: every conv and the FC layer as (name, M, K, N, n_x): the im2col GEMM it runs
+    (M = batch x output pixels, K = kernel area x input channels, N = output channels) and the number of elements
+    n_x of its input activation tensor (batch x input pixels x input channels, what the quantizer sees)."""
+    b = batch
+    L = [("conv1", b * 112 * 112, 147, 64, b * 224 * 224 * 3)]
+    L += [(f"layer1.{i}", b * 56 * 56, 576, 64, b * 56 * 56 * 64) for i in range(4)]
+    L += [("layer2.0", b * 28 * 28, 576, 128, b * 56 * 56 * 64)]
+    L += [(f"layer2.{i}", b * 28 * 28, 1152, 128, b * 28 * 28 * 128) for i in range(1, 4)]
+    L += [("layer2.ds", b * 28 * 28, 64, 128, b * 56 * 56 * 64)]
+    L += [("layer3.0", b * 14 * 14, 1152, 256, b * 28 * 28 * 128)]
+    L += [(f"layer3.{i}", b * 14 * 14, 2304, 256, b * 14 * 14 * 256) for i in range(1, 4)]
+    L += [("layer3.ds", b * 14 * 14, 128, 256, b * 28 * 28 * 128)]
+    L += [("layer4.0", b * 7 * 7, 2304, 512, b * 14 * 14 * 256)]
+    L += [(f"layer4.{i}", b * 7 * 7, 4608, 512, b * 7 * 7 * 512) for i in range(1, 4)]
+    L += [("layer4.ds", b * 7 * 7, 256, 512, b * 14 * 14 * 256)]
+    L += [("fc", b, 512, 1000, b * 512)]
+    return L

@@ -24,11 +24,12 @@ CALLS = ("quantize_soft_w", "entropy_w", "quantize_soft_x", "entropy_x", "qlinea
 
 
 class CdlLayerStep:
-    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda"):
+    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None):
         """wq / xq: objects with q, lo, hi, alpha, rate_weight, window (weights / activations); n_x: number of
         activation elements quantized per step (the layer's input tensor, before im2col)."""
         self.torch = torch
         self.M, self.K, self.N, self.n_x, self.n_w = M, K, N, n_x, K * N
+        self.lda = lda if lda is not None else (K + 15) // 16 * 16     # row pitch of A_idx (multiple of 16 bytes)
         self.wq, self.xq, self.q_g = wq, xq, float(q_g)
         t, dev = torch, device
         f32, i8, u8 = t.float32, t.int8, t.uint8
@@ -38,7 +39,7 @@ class CdlLayerStep:
         # inputs of a step
         self.w = t.empty(self.n_w, dtype=f32, device=dev)
         self.x = t.empty(n_x, dtype=f32, device=dev)
-        self.A_idx = t.empty((M, K), dtype=idt(xq.lo), device=dev)
+        self.A_idx = t.zeros((M, self.lda), dtype=idt(xq.lo), device=dev)
         self.dY = t.empty((M, N), dtype=f32, device=dev)
         self.gx_in = t.empty(n_x, dtype=f32, device=dev)         # dL/dQ(x) after the scatter back from dA
         # outputs
@@ -84,13 +85,13 @@ class CdlLayerStep:
         m(CALLS[1]); cdl.cdl_index_entropy(self.hist_w, nlw, s[0:1], self.prob_w, None, stream)
         m(CALLS[2]); cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, stream)
         m(CALLS[3]); cdl.cdl_index_entropy(self.hist_x, nlx, s[1:2], self.prob_x, None, stream)
-        m(CALLS[4]); cdl.cdl_qlinear_fwd(self.A_idx, K, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
+        m(CALLS[4]); cdl.cdl_qlinear_fwd(self.A_idx, self.lda, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
                                          None, self.ws, self.ws_bytes, stream)
         m(CALLS[5]); cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, stream)
         # the two backward products are issued as two calls so that each can be timed on its own
         m(CALLS[6]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
                                          M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
-        m(CALLS[7]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, K, self.da, None, N, None,
+        m(CALLS[7]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
                                          M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
         m(CALLS[8]); cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, s[4:5], s[5:6], stream)
         m(CALLS[9]); cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, s[2:3], s[3:4], stream)
