@@ -419,7 +419,7 @@ def run_network(args):
         x = torch.randn(n_x, device="cuda", generator=gen).abs_()
         wq = inputs.Quantizer(float(w.std()) / 3.0, -3, 3, 100.0, 0.01, 0)
         xq = inputs.Quantizer(float(2.0 * x.mean() / 8.0 ** 0.5), 0, 15, 100.0, 0.01, 5)
-        st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g)
+        st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g, need_dx=(name != "conv1"))   # the image needs no gradient
         st.w.copy_(w)
         st.x.copy_(x)
         del w, x
@@ -473,11 +473,12 @@ def run_network(args):
         per = {c: sum(ev[it][li][i].elapsed_time(ev[it][li][i + 1]) for it in range(steps)) / steps for i, c in enumerate(CALLS)}
         g_ms = per["qlinear_fwd"] + per["qlinear_bwd_dx"] + per["qlinear_bwd_dw"]
         q_ms = sum(v for c, v in per.items() if c.startswith("quantize"))
-        ops = 6.0 * M * K * N
+        ops = (6.0 if st.need_dx else 4.0) * M * K * N
         q_el = 2 * (n_x + K * N) + M * N
         table.append({"layer": name, "M": M, "K": K, "N": N, "ms": round(sum(per.values()), 4), "gemm_ms": round(g_ms, 4),
                       "gemm_int8_TOPS": round(ops / (g_ms * 1e-3) / 1e12, 1), "quantizer_ms": round(q_ms, 4),
                       "quantizer_Gelem_per_s": round(q_el / (q_ms * 1e-3) / 1e9, 1),
+                      "calls_us": {c: round(v * 1e3, 1) for c, v in per.items()},
                       "status": cdl.cdl_workspace_status(st.ws, check=False)})
         tot_ops += ops
         tot_q += q_el

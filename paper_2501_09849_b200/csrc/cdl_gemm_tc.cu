@@ -19,7 +19,7 @@
 // global memory sees whole 128-byte lines.  Work units are (tile, split of the reduced dimension); with more
 // than one split the staging block is added into an int32 buffer with a TMA bulk reduce-add (integer, so the
 // result does not depend on order).  Outputs whose pitch or base is not 16-byte aligned, and tiles 16 columns
-// wide, are written straight from registers instead.
+// wide, go through the same staging block and are copied out by the warps one row at a time.
 // Every wait is bounded: on expiry the kernel records CDL_ERR_TIMEOUT in the status word and winds down.
 #include <cuda.h>
 
@@ -325,7 +325,6 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int erow = quarter * 32 + lane;       // row of the tile owned by this thread
         const bool leader = threadIdx.x == 64;      // issues and tracks the bulk stores
         const uint32_t out_base = smem_base + (uint32_t)(kStages * kStageBytes);
-        const bool vec_ok = (P.J & 3) == 0;
         uint32_t tcount = 0, ocount = 0;
 
         // 32 four-byte values of this thread's row -> swizzled staging block -> TMA store or reduce-add
@@ -349,6 +348,37 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             ++ocount;
         };
 
+        // Same staging, then the warp copies its own 32 rows out itself, one row (up to 128 contiguous bytes) per
+        // instruction: for outputs TMA cannot take (row pitch or base not a multiple of 16 bytes, 16-column tiles).
+        auto stage_and_copy = [&](const uint32_t (&w)[32], int32_t *out, bool reduce, long long row_off, int tile_row0,
+                                  int col0, int ncol) {
+            const uint32_t blk = out_base + (ocount & 1u) * (uint32_t)kOutBytes;
+            if (leader) bulk_wait_read_1();
+            epi_barrier();
+            const uint32_t dst = blk + (uint32_t)erow * 128u;
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c4 ^ (erow & 7)) << 4)),
+                             "r"(w[4 * c4]), "r"(w[4 * c4 + 1]), "r"(w[4 * c4 + 2]), "r"(w[4 * c4 + 3])
+                             : "memory");
+            __syncwarp();
+            for (int rr = 0; rr < 32; ++rr) {
+                const int rl = quarter * 32 + rr;
+                const int grow = tile_row0 + rl;
+                if (grow >= P.I) break;                                    // uniform over the warp
+                uint32_t val;
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(val)
+                             : "r"(blk + (uint32_t)rl * 128u + (uint32_t)(((lane >> 2) ^ (rl & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
+                if (lane < ncol) {
+                    int32_t *q = out + (row_off + grow) * P.J + col0 + lane;
+                    if (reduce) asm volatile("red.global.add.s32 [%0], %1;" ::"l"(q), "r"(val) : "memory");
+                    else *q = (int32_t)val;
+                }
+            }
+            __syncwarp();
+            ++ocount;
+        };
+
         for (int u = blockIdx.x; u < units; u += gridDim.x, ++tcount) {
             const int tile = u / P.splits;
             const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
@@ -361,7 +391,6 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 break;
             }
             tc_fence_after();
-            const int row = ti * TM + erow;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
             for (int c0 = 0; c0 < P.TN; c0 += 32) {
                 const int col0 = tj * P.TN + c0;
@@ -370,39 +399,14 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 tc_ld32(taddr + (uint32_t)c0, v);
                 tc_wait_ld();
                 const int ncol = min(min(32, P.TN - c0), P.J - col0);
-                const long long off = (long long)row * P.J + col0;
-                const bool in_rows = row < P.I;
                 if (P.splits > 1) {
-                    if (P.tma_acc) {
-                        stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + ti * TM);
-                    } else if (in_rows) {
-                        int32_t *dst = P.acc_out + off + (long long)slab_row0 * P.J;
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (c < ncol) {
-                                if (P.slab_rows == 0)
-                                    asm volatile("red.global.add.s32 [%0], %1;" ::"l"(dst + c), "r"(v[c]) : "memory");
-                                else
-                                    dst[c] = (int)v[c];
-                            }
-                    }
+                    if (P.tma_acc) stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + ti * TM);
+                    else stage_and_copy(v, P.acc_out, P.slab_rows == 0, slab_row0, ti * TM, col0, ncol);
                     continue;
                 }
                 if (P.acc_out != nullptr) {
-                    if (P.tma_acc) {
-                        stage_and_send(v, &map_acc, false, col0, ti * TM);
-                    } else if (in_rows) {
-                        if (vec_ok && ncol == 32) {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<int4 *>(P.acc_out + off + c) =
-                                    make_int4((int)v[c], (int)v[c + 1], (int)v[c + 2], (int)v[c + 3]);
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (c < ncol) P.acc_out[off + c] = (int)v[c];
-                        }
-                    }
+                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, ti * TM);
+                    else stage_and_copy(v, P.acc_out, false, 0, ti * TM, col0, ncol);
                 }
                 if (P.f_out != nullptr) {
                     uint32_t f[32];
@@ -413,19 +417,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
                     }
-                    if (P.tma_f) {
-                        stage_and_send(f, &map_f, false, col0, ti * TM);
-                    } else if (in_rows) {
-                        if (vec_ok && ncol == 32) {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<uint4 *>(P.f_out + off + c) = make_uint4(f[c], f[c + 1], f[c + 2], f[c + 3]);
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (c < ncol) P.f_out[off + c] = __uint_as_float(f[c]);
-                        }
-                    }
+                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, ti * TM);
+                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, ti * TM, col0, ncol);
                 }
             }
             tc_fence_before();

@@ -24,11 +24,12 @@ CALLS = ("quantize_soft_w", "entropy_w", "quantize_soft_x", "entropy_x", "qlinea
 
 
 class CdlLayerStep:
-    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None):
+    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None, need_dx=True):
         """wq / xq: objects with q, lo, hi, alpha, rate_weight, window (weights / activations); n_x: number of
         activation elements quantized per step (the layer's input tensor, before im2col)."""
         self.torch = torch
         self.M, self.K, self.N, self.n_x, self.n_w = M, K, N, n_x, K * N
+        self.need_dx = need_dx      # False for the first layer of a network: its input needs no gradient
         self.lda = lda if lda is not None else (K + 15) // 16 * 16     # row pitch of A_idx (multiple of 16 bytes)
         self.wq, self.xq, self.q_g = wq, xq, float(q_g)
         t, dev = torch, device
@@ -53,7 +54,7 @@ class CdlLayerStep:
         self.prob_x = t.empty(xq.hi - xq.lo + 1, dtype=f32, device=dev)
         self.Y = t.empty((M, N), dtype=f32, device=dev)
         self.G_idx = t.empty((M, N), dtype=i8, device=dev)
-        self.dA = t.empty((M, K), dtype=f32, device=dev)
+        self.dA = t.empty((M, K), dtype=f32, device=dev) if need_dx else None
         self.dW = t.empty((K, N), dtype=f32, device=dev)
         self.dx = t.empty(n_x, dtype=f32, device=dev)
         self.dw = t.empty(self.n_w, dtype=f32, device=dev)
@@ -89,8 +90,10 @@ class CdlLayerStep:
                                          None, self.ws, self.ws_bytes, stream)
         m(CALLS[5]); cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, stream)
         # the two backward products are issued as two calls so that each can be timed on its own
-        m(CALLS[6]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
-                                         M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
+        m(CALLS[6])
+        if self.need_dx:
+            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
+                                M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
         m(CALLS[7]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
                                          M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
         m(CALLS[8]); cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, s[4:5], s[5:6], stream)
