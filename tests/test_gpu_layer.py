@@ -214,3 +214,30 @@ def test_long_reduction_beyond_int32_is_summed_exactly(torch):
     buf = torch.zeros(max(nb, M * lda), dtype=torch.uint8, device="cuda")
     rc = cdl.cdl_qlinear_bwd(buf, ldg, g, buf, lda, a, None, ldg, None, M, N, K, None, None, buf, None, buf, nb, check=False)
     assert rc == -5
+
+
+def test_resnet18_conv1_and_fc_shapes(torch):
+    # ResNet-18's first conv as an im2col GEMM at batch 16 (M = 16*112*112, K = 147 padded to a pitch of 160,
+    # N = 64) with 8-bit activation indices (first layer kept at 8 bits, Sec. VI-B.2): dW reduces over 200704 rows,
+    # beyond what int32 guarantees, so only its float output exists.  And the FC layer (256, 512, 1000 -> pitch 1008).
+    M, K, N = 16 * 112 * 112, 147, 64
+    A = inputs.uniform_indices((M, K), 0, 255, seed=21)
+    W = inputs.uniform_indices((K, N), -3, 3, seed=22)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=23)
+    a, w, g = cdl.IndexDesc(0.02, 0, 255), cdl.IndexDesc(0.05, -3, 3), cdl.IndexDesc(1e-3, -127, 127)
+    acc, y = run_fwd(torch, A, W, a, w)
+    out = run_bwd(torch, G, A, W, g, a, w, want=("dX", "dW"))
+    rng = np.random.default_rng(1)
+    rows = np.unique(np.concatenate([np.arange(0, 2), np.arange(M - 2, M), np.arange(127, 130), rng.integers(0, M, size=300)]))
+    ref_f = oracle.gemm_fwd(A[rows], W)
+    assert np.array_equal(acc[rows].astype(np.int64), ref_f) and np.array_equal(y[rows], scaled(ref_f, a.q, w.q))
+    assert np.array_equal(out["dX"][rows], scaled(oracle.gemm_dx(G[rows], W), g.q, w.q))
+    ks = np.unique(np.concatenate([[0, 1, 127, 128, 145, 146], rng.integers(0, K, size=10)]))
+    ref_w = oracle.gemm_dw(np.ascontiguousarray(A[:, ks]), G)
+    assert np.array_equal(out["dW"][ks], scaled(ref_w, g.q, a.q))
+    # FC layer
+    M, K, N = 256, 512, 1000
+    A = inputs.uniform_indices((M, K), 0, 15, seed=24)
+    W = inputs.uniform_indices((K, N), -3, 3, seed=25)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=26)
+    check_all_products(torch, A, W, G, cdl.IndexDesc(0.25, 0, 15), w, g)
