@@ -54,6 +54,13 @@ def _load():
         lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        lib.cdl_oracle_philox4x32_10.argtypes = [P, P, P]
+        lib.cdl_oracle_philox4x32_10.restype = None
+        lib.cdl_oracle_uniform.argtypes = [c.c_uint64, c.c_uint64]
+        lib.cdl_oracle_uniform.restype = c.c_double
+        lib.cdl_oracle_sample.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, c.c_uint64,
+                                          c.c_uint64, P, P, P, P]
+        lib.cdl_oracle_sample.restype = None
         for f in ("cpmf", "soft", "partials", "hard", "entropy", "backward", "gemm_fwd", "gemm_dx", "gemm_dw"):
             getattr(lib, "cdl_oracle_" + f).restype = None
         _lib = lib
@@ -186,3 +193,29 @@ def gemm_dw(A, G):
     acc = np.empty((K, N), dtype=np.int64)
     _load().cdl_oracle_gemm_dw(_ptr(A), lda, au, _ptr(G), ldg, M, N, K, _ptr(acc))
     return acc
+
+
+def philox4x32_10(ctr, key):
+    """One block of Philox4x32-10: ctr 4 x uint32, key 2 x uint32 -> 4 x uint32."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.empty(4, dtype=np.uint32)
+    _load().cdl_oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def uniform(seed, e):
+    """The uniform number in [0,1) element number e draws under `seed`."""
+    return float(_load().cdl_oracle_uniform(int(seed), int(e)))
+
+
+def sample(x, q, lo, hi, alpha, window=0, seed=0, first_index=0):
+    """Q_p(x) by inversion (Sec. IV-A, Eq. (7)).  Returns (idx int32, u, cdf_lo, cdf_hi): the sampled indices, each
+    element's uniform number and the cumulative probabilities just below / through the chosen level."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    idx = np.empty(x.shape, dtype=np.int32)
+    u, a, b = (np.empty(x.shape, dtype=np.float64) for _ in range(3))
+    _load().cdl_oracle_sample(_ptr(x), x.size, q, lo, hi, alpha, window, int(seed), int(first_index),
+                              _ptr(idx), _ptr(u), _ptr(a), _ptr(b))
+    return idx, u, a, b

@@ -179,6 +179,81 @@ void cdl_oracle_hard(const float *x, int64_t n, float q, int lo, int hi,
 }
 
 /* ---------------------------------------------------------------------------
+ * Counter-based generator Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as
+ * 1, 2, 3", SC 2011), written from its published definition: ten rounds of
+ *   (c0,c1,c2,c3) <- (hi(M1*c2) ^ c1 ^ k0, lo(M1*c2), hi(M0*c0) ^ c3 ^ k1, lo(M0*c0))
+ * with the key (k0,k1) advanced by the Weyl constants (W0,W1) between rounds.
+ * ------------------------------------------------------------------------- */
+void cdl_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += W0;
+            k1 += W1;
+        }
+        const uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0;
+        c1 = n1;
+        c2 = n2;
+        c3 = n3;
+    }
+    out[0] = c0;
+    out[1] = c1;
+    out[2] = c2;
+    out[3] = c3;
+}
+
+/* The uniform number in [0,1) that element number e of a tensor draws under `seed`: word (e mod 4) of the
+ * Philox block with counter (e div 4, 0) and key = seed, top 24 bits scaled by 2^-24. */
+double cdl_oracle_uniform(uint64_t seed, uint64_t e)
+{
+    const uint64_t blk = e >> 2;
+    const uint32_t ctr[4] = {(uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u};
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t r[4];
+    cdl_oracle_philox4x32_10(ctr, key, r);
+    return (double)(r[e & 3] >> 8) * (1.0 / 16777216.0);
+}
+
+/* ---------------------------------------------------------------------------
+ * Probabilistic quantizer Q_p of Sec. IV-A, Eq. (7): theta is mapped to level i with probability
+ * P_alpha(iq | theta).  Sampling by inversion: with u the element's uniform number, the index is the first
+ * level, in increasing order, whose cumulative probability exceeds u.  cdf_lo / cdf_hi (nullable) receive the
+ * cumulative probability just below and through the chosen level, u_out the uniform number.
+ * ------------------------------------------------------------------------- */
+void cdl_oracle_sample(const float *x, int64_t n, float q, int lo, int hi, float alpha, int window,
+                       uint64_t seed, uint64_t first_index, int32_t *idx, double *u_out,
+                       double *cdf_lo, double *cdf_hi)
+{
+    const int nlev = hi - lo + 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < n; ++e) {
+        double P[CDL_ORACLE_MAX_LEVELS];
+        cdl_oracle_cpmf((double)x[e], (double)q, lo, hi, (double)alpha, window, P);
+        const double u = cdl_oracle_uniform(seed, first_index + (uint64_t)e);
+        double cum = 0.0, below = 0.0;
+        int k = -1;
+        for (int i = 0; i < nlev; ++i) {
+            if (P[i] == 0.0) continue;
+            below = cum;
+            cum += P[i];
+            k = i;
+            if (cum > u) break;
+        }
+        idx[e] = lo + k;
+        if (u_out) u_out[e] = u;
+        if (cdf_lo) cdf_lo[e] = below;
+        if (cdf_hi) cdf_hi[e] = cum;
+    }
+}
+
+/* ---------------------------------------------------------------------------
  * Entropy of the empirical level distribution, H(P) = -sum_c P[c] log2 P[c]
  * (Sec. III-A with base 2; Sec. V-C), P[c] = hist[c] / n, 0 log 0 = 0.
  * ------------------------------------------------------------------------- */
