@@ -247,7 +247,7 @@ def run_reference(args, rank):
 def run_sweep(args):
     """Quantizer-only bandwidth sweep: fp32 tensors of 2^20 .. 2^max elements (50/50 N(0,1) / Laplace(0,1) mixture
     drawn on the device), L in {1,3,7,15,127}, alpha in {1,100,1e4}, step 4/L; hard, hard+hist, soft, soft+idx+hist,
-    backward and backward+rate timed separately with CUDA events."""
+    sampled index+hist, backward and backward+rate timed separately with CUDA events."""
     import torch
 
     import paper_2501_09849_b200 as cdl
@@ -315,10 +315,13 @@ def run_sweep(args):
                             return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, None, None)
                         if kind == "soft_idx_hist":
                             return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, ix, hist)
+                        if kind == "sample_hist":
+                            return lambda: cdl.cdl_quantize_sample(xs, n, PP, 7, o, ix, None, hist)
                         return lambda: cdl.cdl_quantize_backward(xs, gs, n, PP, ys, s[0:1], s[1:2])
                     return make
                 passes = {"hard": (5, mk("hard")), "hard_hist": (5, mk("hard_hist")), "soft": (8, mk("soft")),
-                          "soft_idx_hist": (9, mk("soft_idx_hist")), "backward": (12, mk("backward")),
+                          "soft_idx_hist": (9, mk("soft_idx_hist")), "sample_hist": (5, mk("sample_hist")),
+                          "backward": (12, mk("backward")),
                           "backward_rate": (12, mk("backward", Pr))}
                 if alpha != 1.0:
                     passes.pop("hard"), passes.pop("hard_hist")      # the hard passes do not depend on alpha

@@ -113,6 +113,20 @@ int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p,
                       float *y_soft, void *idx_out, uint64_t *hist, void *stream);
 
 /*
+ * Probabilistic quantizer Q_p of Sec. IV-A, Eq. (7) - what CDL's forward pass applies to weights and activations
+ * (Algorithm 1): element i is mapped to level k with probability P_alpha(kq | x[i]) (CPMF of Eq. (4), optionally
+ * truncated to p->window levels).  Sampling is by inversion in increasing level order: with u_i in [0,1) the
+ * element's uniform number, the index is the first level whose cumulative probability exceeds u_i.  u_i is the
+ * top 24 bits, times 2^-24, of word (e mod 4) of the Philox4x32-10 block with counter (e div 4, 0) and key `seed`,
+ * where e = first_index + i: the draw depends only on (seed, e), so any partition of a tensor into calls or
+ * ranks (each passing its own first_index) reproduces the same sample.  The cumulative sums are binary32; next to
+ * a cumulative-probability boundary (within ~1e-6) the neighbouring level may be chosen.
+ *   idx_out [dev] n index bytes, nullable;  y_out [dev] n floats idx * q, nullable;  hist: as cdl_quantize_hard.
+ */
+int cdl_quantize_sample(const float *x, int64_t n, const cdl_quant_params *p, uint64_t seed,
+                        uint64_t first_index, void *idx_out, float *y_out, uint64_t *hist, void *stream);
+
+/*
  * Backward of the quantizer with Q_d as the gradient proxy (Sec. V-B, Eqs. (18), (20)-(24)):
  *   grad_x[i]  = grad_out[i] * dQ_d/dtheta(x[i])                     Lemma 1, Eq. (9a): 2 alpha Var
  *                + rate_weight * d(n H)/dtheta_i                      (only if level_prob != NULL)

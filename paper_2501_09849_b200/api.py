@@ -11,7 +11,7 @@ from pathlib import Path
 
 __all__ = [
     "CdlError", "QuantParams", "IndexDesc", "library_path", "load_library",
-    "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward",
+    "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
@@ -90,6 +90,7 @@ def load_library():
     lib.cdl_quantize_hard.argtypes = [P, I64, P, P, P, P]
     lib.cdl_quantize_soft.argtypes = [P, I64, P, P, P, P, P]
     lib.cdl_quantize_backward.argtypes = [P, P, I64, P, P, P, P, P]
+    lib.cdl_quantize_sample.argtypes = [P, I64, P, C.c_uint64, C.c_uint64, P, P, P, P]
     lib.cdl_index_entropy.argtypes = [P, I32, P, P, P, P]
     lib.cdl_qlinear_fwd.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd.argtypes = [P, I64, P, P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, C.c_size_t, P]
@@ -97,7 +98,7 @@ def load_library():
     lib.cdl_workspace_bytes.argtypes = [I32, I32, I32, I32]
     lib.cdl_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_status.argtypes = [P, P]
-    for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_index_entropy",
+    for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample", "cdl_index_entropy",
                  "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status"):
         getattr(lib, name).restype = C.c_int
     _LIB = lib
@@ -148,6 +149,14 @@ def cdl_quantize_soft(x, n, p: QuantParams, y_soft, idx_out=None, hist=None, str
     rc = load_library().cdl_quantize_soft(_ptr(x), n, C.byref(pc), _ptr(y_soft), _ptr(idx_out), _ptr(hist),
                                           _stream(stream))
     return _check(rc, "cdl_quantize_soft", check)
+
+
+def cdl_quantize_sample(x, n, p: QuantParams, seed, first_index=0, idx_out=None, y_out=None, hist=None, stream=None,
+                        check=True):
+    pc = p._c()
+    rc = load_library().cdl_quantize_sample(_ptr(x), n, C.byref(pc), int(seed), int(first_index), _ptr(idx_out),
+                                            _ptr(y_out), _ptr(hist), _stream(stream))
+    return _check(rc, "cdl_quantize_sample", check)
 
 
 def cdl_quantize_backward(x, grad_out, n, p: QuantParams, grad_x=None, grad_q=None, grad_alpha=None, stream=None,

@@ -180,6 +180,22 @@ int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p, floa
                            nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
+int cdl_quantize_sample(const float *x, int64_t n, const cdl_quant_params *p, uint64_t seed, uint64_t first_index,
+                        void *idx_out, float *y_out, uint64_t *hist, void *stream)
+{
+    if (n < 0 || (n > 0 && x == nullptr)) return CDL_ERR_ARG;
+    if (bad_f32_ptr(x) || bad_f32_ptr(y_out) || (reinterpret_cast<uintptr_t>(hist) & 7u)) return CDL_ERR_ALIGN;
+    QuantDev qd;
+    int rc = make_quant_dev(p, true, &qd);
+    if (rc != CDL_OK) return rc;
+    qd.seed = seed;
+    qd.first_index = first_index;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    return launch_quantize(MODE_SAMPLE, x, nullptr, n, qd, y_out, idx_out,
+                           reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
+                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
 int cdl_quantize_backward(const float *x, const float *grad_out, int64_t n, const cdl_quant_params *p,
                           float *grad_x, double *grad_q, double *grad_alpha, void *stream)
 {

@@ -27,9 +27,11 @@ struct QuantDev {
     int window;       // 0 = whole index set, else an odd window smaller than nlev
     int jmax;         // levels further than jmax from the nearest one carry < 2^-40 of its weight
     const float *level_prob;  // nullptr: no rate term
+    unsigned long long seed;         // MODE_SAMPLE: generator key
+    unsigned long long first_index;  // MODE_SAMPLE: counter-space index of element 0
 };
 
-enum QuantMode { MODE_HARD = 0, MODE_SOFT = 1, MODE_BWD = 2 };
+enum QuantMode { MODE_HARD = 0, MODE_SOFT = 1, MODE_BWD = 2, MODE_SAMPLE = 3 };
 
 int check_device();   // CDL_OK, CDL_ERR_UNSUPPORTED or CDL_ERR_LAUNCH
 int sm_count();       // multiprocessors of the current device (0 on error)

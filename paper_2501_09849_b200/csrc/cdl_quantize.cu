@@ -56,6 +56,40 @@ __device__ __forceinline__ float rcp_approx(float x)
     return y;
 }
 
+// Philox4x32-10 (Salmon et al., SC 2011) from its definition: ten rounds of
+//   (c0,c1,c2,c3) <- (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)),  key += (W0, W1) between rounds.
+// Counter = (block number, 0), key = seed; the block's four words serve elements 4 b .. 4 b + 3.
+__device__ __forceinline__ uint4 philox4x32_10(unsigned long long block, unsigned long long seed)
+{
+    const unsigned int M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    unsigned int c0 = (unsigned int)block, c1 = (unsigned int)(block >> 32), c2 = 0u, c3 = 0u;
+    unsigned int k0 = (unsigned int)seed, k1 = (unsigned int)(seed >> 32);
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) {
+            k0 += W0;
+            k1 += W1;
+        }
+        const unsigned int n0 = __umulhi(M1, c2) ^ c1 ^ k0;
+        const unsigned int n1 = M1 * c2;
+        const unsigned int n2 = __umulhi(M0, c0) ^ c3 ^ k1;
+        const unsigned int n3 = M0 * c0;
+        c0 = n0;
+        c1 = n1;
+        c2 = n2;
+        c3 = n3;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+// top 24 bits of a word as a uniform number in [0, 1)
+__device__ __forceinline__ float u01(unsigned int w) { return (float)(w >> 8) * 5.9604644775390625e-8f; }
+__device__ __forceinline__ float philox_uniform(unsigned long long seed, unsigned long long e)
+{
+    const uint4 r = philox4x32_10(e >> 2, seed);
+    const unsigned int k = (unsigned int)e & 3u;
+    return u01(k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w);
+}
+
 struct ElemOut {
     int k0;       // hard index
     float y;      // Q_d
@@ -123,6 +157,15 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         float em = ex2_approx(-P.c1 * wm);
         e1 = (kn < P.fhi) ? e1 : 0.0f;
         em = (kn > P.flo) ? em : 0.0f;
+        if (MODE == MODE_SAMPLE) {
+            // inversion in increasing level order: kn-1 (em), kn (1), kn+1 (e1); g carries the uniform number
+            const float S = 1.0f + e1 + em;
+            const float tt = fminf(g * S, S * 0.99999994f);
+            const int ks = ki + ((tt >= em + 1.0f) ? 1 : 0) - ((tt < em) ? 1 : 0);
+            o.k0 = ks;
+            o.y = __fmul_rn((float)ks, q);
+            return o;
+        }
         const float rS = rcp_approx(1.0f + e1 + em);
         m1 = (e1 - em) * rS;
         o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
@@ -145,6 +188,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float j0 = stf - kn;                    // -4 .. 0
         const float B = P.c1x2 * dh;
         float T0 = 0.0f, T1 = 0.0f, T2 = 0.0f, T3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
+        float ev[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
         const float *Lp = Ltab;
         float Lc = 0.0f;
         if (RATE) {
@@ -155,6 +199,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         for (int i = 0; i < 5; ++i) {
             const float jf = j0 + (float)i;
             const float e = ex2_approx(jf * fmaf(-P.A, jf, B));
+            if (MODE == MODE_SAMPLE) ev[i] = e;
             T0 += e;
             if (i > 0) T1 = fmaf((float)i, e, T1);
             if (MODE == MODE_BWD) {
@@ -168,6 +213,20 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                     if (i > 0) R1 = fmaf((float)i, le, R1);
                 }
             }
+        }
+        if (MODE == MODE_SAMPLE) {
+            const float tt = fminf(g * T0, T0 * 0.99999994f);
+            float cum = 0.0f;
+            int cnt = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                cum += ev[i];
+                cnt += (cum <= tt) ? 1 : 0;
+            }
+            const int ks = min(max(ki - 2, P.lo), P.hi - 4) + cnt;
+            o.k0 = ks;
+            o.y = __fmul_rn((float)ks, q);
+            return o;
         }
         const float rT = rcp_approx(T0);
         const float mi = T1 * rT;                      // E I, I = level - st
@@ -212,6 +271,22 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                     R1 = fmaf(jf, le, R1);
                 }
             }
+        }
+        if (MODE == MODE_SAMPLE) {
+            // second pass over the same levels: first one whose running sum exceeds u * S
+            const float tt = fminf(g * S, S * 0.99999994f);
+            float cum = 0.0f, jj = (float)jlo;
+            int ks = ki + jhi;
+            for (int j = jlo; j <= jhi; ++j, jj += 1.0f) {
+                cum += ex2_approx(jj * fmaf(-P.A, jj, B));
+                if (cum > tt) {
+                    ks = ki + j;
+                    break;
+                }
+            }
+            o.k0 = ks;
+            o.y = __fmul_rn((float)ks, q);
+            return o;
         }
         const float rS = rcp_approx(S);
         m1 = S1 * rS;
@@ -299,6 +374,20 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     gs[2] = gv[b].z;
                     gs[3] = gv[b].w;
                 }
+                if (MODE == MODE_SAMPLE) {
+                    // the uniform numbers of elements e0 .. e0+3: one Philox block when e0 is a multiple of 4
+                    const unsigned long long e0 = P.first_index + (unsigned long long)(head + 4 * i);
+                    if ((e0 & 3ull) == 0ull) {
+                        const uint4 r = philox4x32_10(e0 >> 2, P.seed);
+                        gs[0] = u01(r.x);
+                        gs[1] = u01(r.y);
+                        gs[2] = u01(r.z);
+                        gs[3] = u01(r.w);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) gs[c] = philox_uniform(P.seed, e0 + c);
+                    }
+                }
                 float ys[4], gxs[4];
                 unsigned int packed = 0u;
 #pragma unroll
@@ -311,7 +400,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     packed |= ((unsigned int)o.k0 & 0xffu) << (8 * c);
                     if (MODE != MODE_BWD && do_hist) hist_add(hist_s, o.k0 - P.lo, lane);
                 }
-                if (MODE == MODE_SOFT) __stcs(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
+                if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) __stcs(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
                 if (MODE == MODE_BWD && gx != nullptr) __stcs(gx4 + i, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
                 if (MODE != MODE_BWD && idx != nullptr) idx4[i] = packed;
             }
@@ -327,9 +416,10 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     const int64_t nrem = head + (n - tail0);
     for (int64_t t = tid; t < nrem; t += stride) {
         const int64_t i = (t < head) ? t : (tail0 + (t - head));
-        const float gi = (MODE == MODE_BWD) ? g[i] : 0.0f;
+        const float gi = (MODE == MODE_BWD) ? g[i]
+                         : (MODE == MODE_SAMPLE) ? philox_uniform(P.seed, P.first_index + (unsigned long long)i) : 0.0f;
         const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, x[i], gi);
-        if (MODE == MODE_SOFT) y[i] = o.y;
+        if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) y[i] = o.y;
         if (MODE == MODE_BWD) {
             if (gx != nullptr) gx[i] = o.gx;
             acc_q += (double)o.tq;
@@ -422,7 +512,7 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     int64_t head = (int64_t)((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
     if (head > n) head = n;
     bool vec = true;
-    if (mode == MODE_SOFT) vec = vec && aligned_to(y + head, 16);
+    if (mode == MODE_SOFT || (mode == MODE_SAMPLE && y != nullptr)) vec = vec && aligned_to(y + head, 16);
     if (mode == MODE_BWD) {
         vec = vec && aligned_to(grad_out + head, 16);
         if (grad_x) vec = vec && aligned_to(grad_x + head, 16);
@@ -443,6 +533,10 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
             return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, false)
                  : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, false)
                                      : CDL_Q(MODE_SOFT, PATH_LOOP, false);
+        case MODE_SAMPLE:
+            return path == PATH_NEAR3 ? CDL_Q(MODE_SAMPLE, PATH_NEAR3, false)
+                 : path == PATH_WIN5 ? CDL_Q(MODE_SAMPLE, PATH_WIN5, false)
+                                     : CDL_Q(MODE_SAMPLE, PATH_LOOP, false);
         case MODE_BWD:
             if (rate)
                 return path == PATH_NEAR3 ? CDL_Q(MODE_BWD, PATH_NEAR3, true)
