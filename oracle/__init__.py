@@ -54,6 +54,8 @@ def _load():
         lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        lib.cdl_oracle_mpmf.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, P]
+        lib.cdl_oracle_mpmf.restype = None
         lib.cdl_oracle_philox4x32_10.argtypes = [P, P, P]
         lib.cdl_oracle_philox4x32_10.restype = None
         lib.cdl_oracle_uniform.argtypes = [c.c_uint64, c.c_uint64]
@@ -219,3 +221,12 @@ def sample(x, q, lo, hi, alpha, window=0, seed=0, first_index=0):
     _load().cdl_oracle_sample(_ptr(x), x.size, q, lo, hi, alpha, window, int(seed), int(first_index),
                               _ptr(idx), _ptr(u), _ptr(a), _ptr(b))
     return idx, u, a, b
+
+
+def mpmf(x, q, lo, hi, alpha, window=0):
+    """Soft histogram sum_i P(. | x[i]) (Sec. V-C, Eq. (25) times n); float64[nlev]."""
+    _check_levels(lo, hi)
+    x = _f32(x)
+    sums = np.zeros(hi - lo + 1, dtype=np.float64)
+    _load().cdl_oracle_mpmf(_ptr(x), x.size, q, lo, hi, alpha, window, _ptr(sums))
+    return sums

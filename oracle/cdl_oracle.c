@@ -179,6 +179,24 @@ void cdl_oracle_hard(const float *x, int64_t n, float q, int lo, int hi,
 }
 
 /* ---------------------------------------------------------------------------
+ * Soft histogram of Sec. V-C, Eq. (25): sums[k] = sum_i P_alpha(k q | x[i]); divided by n it is the marginal
+ * PMF of the randomly quantized tensor, whose entropy is the average number of bits per entry.
+ * ------------------------------------------------------------------------- */
+void cdl_oracle_mpmf(const float *x, int64_t n, float q, int lo, int hi, float alpha, int window, double *sums)
+{
+    const int nlev = hi - lo + 1;
+    double acc[CDL_ORACLE_MAX_LEVELS];
+    for (int k = 0; k < CDL_ORACLE_MAX_LEVELS; ++k) acc[k] = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : acc[:CDL_ORACLE_MAX_LEVELS])
+    for (int64_t e = 0; e < n; ++e) {
+        double P[CDL_ORACLE_MAX_LEVELS];
+        cdl_oracle_cpmf((double)x[e], (double)q, lo, hi, (double)alpha, window, P);
+        for (int k = 0; k < nlev; ++k) acc[k] += P[k];
+    }
+    for (int k = 0; k < nlev; ++k) sums[k] = acc[k];
+}
+
+/* ---------------------------------------------------------------------------
  * Counter-based generator Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as
  * 1, 2, 3", SC 2011), written from its published definition: ten rounds of
  *   (c0,c1,c2,c3) <- (hi(M1*c2) ^ c1 ^ k0, lo(M1*c2), hi(M0*c0) ^ c3 ^ k1, lo(M0*c0))

@@ -373,3 +373,27 @@ def test_one_hot_index_matrix_selects_rows():
     A = np.zeros((K, K), dtype=np.uint8)
     A[np.arange(K), np.arange(K)[::-1]] = 1
     assert np.array_equal(oracle.gemm_fwd(A, W), W[::-1].astype(np.int64))
+
+
+# ------------------------------------------------------------------ soft histogram / marginal PMF (Sec. V-C, Eq. (25))
+def test_soft_histogram_is_the_sum_of_cpmfs_and_tends_to_the_count_histogram():
+    x = inputs.normal((3001,), 0.2, seed=31)
+    q, lo, hi = f32(0.1), -4, 3
+    for window in (0, 5):
+        s = oracle.mpmf(x, q, lo, hi, f32(40.0), window)
+        assert s.sum() == pytest.approx(x.size, rel=1e-12)               # every CPMF sums to 1
+        byhand = np.sum([oracle.cpmf(float(t), float(q), lo, hi, float(f32(40.0)), window) for t in x[:200]], axis=0)
+        np.testing.assert_allclose(oracle.mpmf(x[:200], q, lo, hi, f32(40.0), window), byhand, rtol=1e-12)
+    # Remark of Sec. IV-A: for large alpha all the mass sits on the nearest level -> the count histogram
+    u = x.astype(np.float64) / float(q)
+    away = np.abs(u - np.floor(u) - 0.5) > 0.02
+    _, hist = oracle.hard(x[away], q, lo, hi)
+    np.testing.assert_allclose(oracle.mpmf(x[away], q, lo, hi, f32(1e7)), hist.astype(np.float64), rtol=0, atol=1e-6)
+
+
+def test_soft_histogram_two_levels_closed_form():
+    q, alpha = f32(0.5), f32(6.0)
+    x = inputs.normal((500,), 0.5, seed=32)
+    s = oracle.mpmf(x, q, 0, 1, alpha)
+    sig = 1.0 / (1.0 + np.exp(-float(alpha) * float(q) * (2.0 * x.astype(np.float64) - float(q))))
+    assert s[1] == pytest.approx(sig.sum(), rel=1e-12) and s[0] == pytest.approx((1 - sig).sum(), rel=1e-12)
