@@ -105,12 +105,18 @@ int cdl_quantize_hard(const float *x, int64_t n, const cdl_quant_params *p,
 /*
  * Soft deterministic quantizer Q_d(x) = sum_i P_alpha(iq | x) iq of Sec. IV-B, Eq. (8), with the
  * CPMF of Eq. (4) (optionally truncated to p->window levels), and, in the same pass over x,
- * optionally the hard index and the histogram exactly as cdl_quantize_hard writes them.
- *   y_soft   [dev] n floats, required.   idx_out, hist: nullable.
+ * optionally the hard index and the histogram exactly as cdl_quantize_hard writes them, and the soft
+ * histogram of Sec. V-C, Eq. (25): the marginal PMF of the randomly quantized tensor is
+ * (1/n) sum_i P_alpha(. | x[i]), whose entropy is the bits-per-entry the objective constrains.
+ *   y_soft    [dev] n floats, required.   idx_out, hist: nullable.
+ *   soft_hist [dev] nlev uint64, nullable: sum_i P_alpha(kq | x[i]) per level k in fixed point, units of 2^-32
+ *             (integer sums: exact and independent of the order of accumulation).  Cleared first unless
+ *             CDL_HIST_ACCUMULATE.  cdl_index_entropy accepts it in place of a count histogram (it only uses
+ *             ratios): H_bits is then the entropy of the marginal PMF and level_prob that PMF.
  * x must be finite for y_soft to be meaningful (NaN and infinities give NaN).
  */
 int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p,
-                      float *y_soft, void *idx_out, uint64_t *hist, void *stream);
+                      float *y_soft, void *idx_out, uint64_t *hist, uint64_t *soft_hist, void *stream);
 
 /*
  * Probabilistic quantizer Q_p of Sec. IV-A, Eq. (7) - what CDL's forward pass applies to weights and activations

@@ -88,7 +88,7 @@ def load_library():
     lib.cdl_strerror.restype = C.c_char_p
     lib.cdl_strerror.argtypes = [C.c_int]
     lib.cdl_quantize_hard.argtypes = [P, I64, P, P, P, P]
-    lib.cdl_quantize_soft.argtypes = [P, I64, P, P, P, P, P]
+    lib.cdl_quantize_soft.argtypes = [P, I64, P, P, P, P, P, P]
     lib.cdl_quantize_backward.argtypes = [P, P, I64, P, P, P, P, P]
     lib.cdl_quantize_sample.argtypes = [P, I64, P, C.c_uint64, C.c_uint64, P, P, P, P]
     lib.cdl_index_entropy.argtypes = [P, I32, P, P, P, P]
@@ -144,9 +144,9 @@ def cdl_quantize_hard(x, n, p: QuantParams, idx_out=None, hist=None, stream=None
     return _check(rc, "cdl_quantize_hard", check)
 
 
-def cdl_quantize_soft(x, n, p: QuantParams, y_soft, idx_out=None, hist=None, stream=None, check=True):
+def cdl_quantize_soft(x, n, p: QuantParams, y_soft, idx_out=None, hist=None, stream=None, check=True, soft_hist=None):
     pc = p._c()
-    rc = load_library().cdl_quantize_soft(_ptr(x), n, C.byref(pc), _ptr(y_soft), _ptr(idx_out), _ptr(hist),
+    rc = load_library().cdl_quantize_soft(_ptr(x), n, C.byref(pc), _ptr(y_soft), _ptr(idx_out), _ptr(hist), _ptr(soft_hist),
                                           _stream(stream))
     return _check(rc, "cdl_quantize_soft", check)
 

@@ -163,21 +163,24 @@ int cdl_quantize_hard(const float *x, int64_t n, const cdl_quant_params *p, void
     if ((rc = check_device()) != CDL_OK) return rc;
     return launch_quantize(MODE_HARD, x, nullptr, n, qd, nullptr, idx_out,
                            reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
-                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+                           nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int cdl_quantize_soft(const float *x, int64_t n, const cdl_quant_params *p, float *y_soft, void *idx_out,
-                      uint64_t *hist, void *stream)
+                      uint64_t *hist, uint64_t *soft_hist, void *stream)
 {
     if (n < 0 || (n > 0 && (x == nullptr || y_soft == nullptr))) return CDL_ERR_ARG;
-    if (bad_f32_ptr(x) || bad_f32_ptr(y_soft) || (reinterpret_cast<uintptr_t>(hist) & 7u)) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(x) || bad_f32_ptr(y_soft) || (reinterpret_cast<uintptr_t>(hist) & 7u) ||
+        (reinterpret_cast<uintptr_t>(soft_hist) & 7u))
+        return CDL_ERR_ALIGN;
     QuantDev qd;
     int rc = make_quant_dev(p, true, &qd);
     if (rc != CDL_OK) return rc;
     if ((rc = check_device()) != CDL_OK) return rc;
     return launch_quantize(MODE_SOFT, x, nullptr, n, qd, y_soft, idx_out,
                            reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
-                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+                           nullptr, nullptr, nullptr, reinterpret_cast<unsigned long long *>(soft_hist),
+                           static_cast<cudaStream_t>(stream));
 }
 
 int cdl_quantize_sample(const float *x, int64_t n, const cdl_quant_params *p, uint64_t seed, uint64_t first_index,
@@ -193,7 +196,7 @@ int cdl_quantize_sample(const float *x, int64_t n, const cdl_quant_params *p, ui
     if ((rc = check_device()) != CDL_OK) return rc;
     return launch_quantize(MODE_SAMPLE, x, nullptr, n, qd, y_out, idx_out,
                            reinterpret_cast<unsigned long long *>(hist), (p->flags & CDL_HIST_ACCUMULATE) != 0,
-                           nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+                           nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int cdl_quantize_backward(const float *x, const float *grad_out, int64_t n, const cdl_quant_params *p,
@@ -208,7 +211,7 @@ int cdl_quantize_backward(const float *x, const float *grad_out, int64_t n, cons
     if (bad_f32_ptr(qd.level_prob)) return CDL_ERR_ALIGN;
     if ((rc = check_device()) != CDL_OK) return rc;
     return launch_quantize(MODE_BWD, x, grad_out, n, qd, nullptr, nullptr, nullptr, false, grad_x, grad_q,
-                           grad_alpha, static_cast<cudaStream_t>(stream));
+                           grad_alpha, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits, float *level_prob, uint64_t *n_out,

@@ -39,7 +39,8 @@ int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out);
 
 int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, const QuantDev &qd,
                     float *y, void *idx, unsigned long long *hist, bool hist_accumulate,
-                    float *grad_x, double *grad_q, double *grad_alpha, cudaStream_t stream);
+                    float *grad_x, double *grad_q, double *grad_alpha, unsigned long long *soft_hist,
+                    cudaStream_t stream);
 int launch_entropy(const unsigned long long *hist, int nlev, double *H, float *prob,
                    unsigned long long *n_out, cudaStream_t stream);
 

@@ -90,6 +90,13 @@ __device__ __forceinline__ float philox_uniform(unsigned long long seed, unsigne
     return u01(k == 0 ? r.x : k == 1 ? r.y : k == 2 ? r.z : r.w);
 }
 
+// Adds P (a CPMF entry in [0,1]) to the soft-histogram bin of `level` in units of 2^-32: integer sums are exact and
+// independent of the order in which elements arrive.
+__device__ __forceinline__ void mp_add(unsigned long long *mp_s, int bin, int lane, float P)
+{
+    atomicAdd(&mp_s[bin * 32 + lane], (unsigned long long)__float2uint_rn(P * 4294967296.0f));
+}
+
 struct ElemOut {
     int k0;       // hard index
     float y;      // Q_d
@@ -123,7 +130,8 @@ __device__ __noinline__ void nearest_fixup(const QuantDev &P, float &kn, int &ki
 }
 
 template <int MODE, int PATH, bool RATE>
-__device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__restrict__ Ltab, float x, float g)
+__device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__restrict__ Ltab, float x, float g,
+                                              unsigned long long *mp_s = nullptr, int lane = 0)
 {
     ElemOut o;
     const float q = P.q;
@@ -169,6 +177,11 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rS = rcp_approx(1.0f + e1 + em);
         m1 = (e1 - em) * rS;
         o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
+        if (MODE == MODE_SOFT && mp_s != nullptr) {
+            mp_add(mp_s, ki - P.lo, lane, rS);
+            if (e1 > 0.0f) mp_add(mp_s, ki + 1 - P.lo, lane, e1 * rS);
+            if (em > 0.0f) mp_add(mp_s, ki - 1 - P.lo, lane, em * rS);
+        }
         if (MODE == MODE_BWD) {
             const float m2 = (e1 + em) * rS;         // E J^2; E J^3 = E J
             varj = fmaf(-m1, m1, m2);
@@ -199,7 +212,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         for (int i = 0; i < 5; ++i) {
             const float jf = j0 + (float)i;
             const float e = ex2_approx(jf * fmaf(-P.A, jf, B));
-            if (MODE == MODE_SAMPLE) ev[i] = e;
+            if (MODE == MODE_SAMPLE || MODE == MODE_SOFT) ev[i] = e;
             T0 += e;
             if (i > 0) T1 = fmaf((float)i, e, T1);
             if (MODE == MODE_BWD) {
@@ -231,6 +244,11 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rT = rcp_approx(T0);
         const float mi = T1 * rT;                      // E I, I = level - st
         o.y = __fmaf_rn(stf, q, __fmul_rn(q, mi));
+        if (MODE == MODE_SOFT && mp_s != nullptr) {
+            const int b0 = min(max(ki - 2, P.lo), P.hi - 4) - P.lo;
+#pragma unroll
+            for (int i = 0; i < 5; ++i) mp_add(mp_s, b0 + i, lane, ev[i] * rT);
+        }
         m1 = mi + j0;
         if (MODE == MODE_BWD) {
             const float m2i = T2 * rT, m3i = T3 * rT;
@@ -291,6 +309,11 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rS = rcp_approx(S);
         m1 = S1 * rS;
         o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
+        if (MODE == MODE_SOFT && mp_s != nullptr) {
+            float jj = (float)jlo;
+            for (int j = jlo; j <= jhi; ++j, jj += 1.0f)
+                mp_add(mp_s, ki + j - P.lo, lane, ex2_approx(jj * fmaf(-P.A, jj, B)) * rS);
+        }
         if (MODE == MODE_BWD) {
             const float m2 = S2 * rS, m3 = S3 * rS;
             varj = fmaf(-m1, m1, m2);
@@ -323,13 +346,20 @@ __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__restrict__ g, int64_t n,
                 int64_t head, int64_t n4, float *__restrict__ y, unsigned char *__restrict__ idx,
                 unsigned long long *__restrict__ hist, float *__restrict__ gx,
-                double *__restrict__ gq, double *__restrict__ ga)
+                double *__restrict__ gq, double *__restrict__ ga, unsigned long long *__restrict__ mp)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *Ltab = reinterpret_cast<float *>(smem_raw);                       // CDL_MAX_LEVELS floats
     unsigned int *hist_s = reinterpret_cast<unsigned int *>(smem_raw + CDL_MAX_LEVELS * sizeof(float));
     const int lane = threadIdx.x & 31;
     const bool do_hist = hist != nullptr;
+    // soft histogram (sum of CPMFs per level, fixed point): bins behind the index histogram's, only when asked for
+    unsigned long long *mp_s = nullptr;
+    if (MODE == MODE_SOFT && mp != nullptr) {
+        mp_s = reinterpret_cast<unsigned long long *>(smem_raw + CDL_MAX_LEVELS * sizeof(float) +
+                                                      (do_hist ? (size_t)P.nlev * 32 * sizeof(unsigned int) : 0));
+        for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) mp_s[k] = 0ull;
+    }
 
     if (RATE) {
         for (int k = threadIdx.x; k < P.nlev; k += kThreads) {
@@ -339,7 +369,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     }
     if (do_hist)
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) hist_s[k] = 0u;
-    if (RATE || do_hist) __syncthreads();
+    if (RATE || do_hist || mp_s != nullptr) __syncthreads();
 
     double acc_q = 0.0, acc_a = 0.0;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
@@ -392,7 +422,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 unsigned int packed = 0u;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c]);
+                    const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
                     ys[c] = o.y;
                     gxs[c] = o.gx;
                     part_q += o.tq;
@@ -418,7 +448,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         const int64_t i = (t < head) ? t : (tail0 + (t - head));
         const float gi = (MODE == MODE_BWD) ? g[i]
                          : (MODE == MODE_SAMPLE) ? philox_uniform(P.seed, P.first_index + (unsigned long long)i) : 0.0f;
-        const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, x[i], gi);
+        const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, x[i], gi, mp_s, lane);
         if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) y[i] = o.y;
         if (MODE == MODE_BWD) {
             if (gx != nullptr) gx[i] = o.gx;
@@ -430,6 +460,16 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         }
     }
 
+    if (MODE == MODE_SOFT && mp_s != nullptr) {
+        __syncthreads();
+        const int warp = threadIdx.x >> 5;
+        for (int b = warp; b < P.nlev; b += kThreads / 32) {
+            unsigned long long c = mp_s[b * 32 + lane];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) c += __shfl_down_sync(0xffffffffu, c, off);
+            if (lane == 0 && c != 0ull) atomicAdd(&mp[b], c);
+        }
+    }
     if (MODE != MODE_BWD && do_hist) {
         __syncthreads();
         const int warp = threadIdx.x >> 5;
@@ -466,10 +506,16 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
 template <int MODE, int PATH, bool RATE>
 int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int64_t head, int64_t n4,
              float *y, unsigned char *idx, unsigned long long *hist, float *gx, double *gq, double *ga,
-             cudaStream_t stream)
+             unsigned long long *mp, cudaStream_t stream)
 {
-    const size_t smem = CDL_MAX_LEVELS * sizeof(float) + (hist ? (size_t)qd.nlev * 32 * sizeof(unsigned int) : 0);
+    const size_t smem = CDL_MAX_LEVELS * sizeof(float) + (hist ? (size_t)qd.nlev * 32 * sizeof(unsigned int) : 0) +
+                        (mp ? (size_t)qd.nlev * 32 * sizeof(unsigned long long) : 0);
     auto kern = quantize_kernel<MODE, PATH, RATE>;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem) != cudaSuccess || per_sm < 1) {
         (void)cudaGetLastError();
@@ -483,7 +529,7 @@ int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int6
     const int64_t cap = (int64_t)sms * per_sm;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    kern<<<(unsigned int)blocks, kThreads, smem, stream>>>(qd, x, g, n, head, n4, y, idx, hist, gx, gq, ga);
+    kern<<<(unsigned int)blocks, kThreads, smem, stream>>>(qd, x, g, n, head, n4, y, idx, hist, gx, gq, ga, mp);
     return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
 }
 
@@ -493,8 +539,15 @@ inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintp
 
 int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, const QuantDev &qd,
                     float *y, void *idx, unsigned long long *hist, bool hist_accumulate,
-                    float *grad_x, double *grad_q, double *grad_alpha, cudaStream_t stream)
+                    float *grad_x, double *grad_q, double *grad_alpha, unsigned long long *soft_hist,
+                    cudaStream_t stream)
 {
+    if (soft_hist != nullptr && !hist_accumulate) {
+        if (cudaMemsetAsync(soft_hist, 0, (size_t)qd.nlev * sizeof(unsigned long long), stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+    }
     if (hist != nullptr && !hist_accumulate) {
         if (cudaMemsetAsync(hist, 0, (size_t)qd.nlev * sizeof(unsigned long long), stream) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -525,7 +578,7 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     const int path = qd.near3 ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
     const bool rate = (mode == MODE_BWD) && qd.level_prob != nullptr && qd.rate_c != 0.0f;
 #define CDL_Q(M, PTH, RT) \
-    launch_t<M, PTH, RT>(qd, x, grad_out, n, head, n4, y, ib, hist, grad_x, grad_q, grad_alpha, stream)
+    launch_t<M, PTH, RT>(qd, x, grad_out, n, head, n4, y, ib, hist, grad_x, grad_q, grad_alpha, soft_hist, stream)
     switch (mode) {
         case MODE_HARD:
             return CDL_Q(MODE_HARD, PATH_LOOP, false);

@@ -303,3 +303,39 @@ def test_mismatched_alignments_take_the_scalar_path(torch):
     assert_backward_close(yb[1:].cpu().numpy(), float(sc[0]), float(sc[1]), ref, g, P.q, P.alpha)
     cdl.cdl_quantize_backward(xd, gd, n, P, None, s[0:1], None)       # optional outputs
     assert abs(float(s.cpu()[0]) - ref["grad_q"]) <= RTOL * ref["abs_q"] + 1e-6 * ref["mag_q"]
+
+
+@pytest.mark.parametrize("q,lo,hi,alpha,window", [
+    (0.1, -4, 3, 100.0, 0), (0.1, -4, 3, 5000.0, 0), (0.25, 0, 15, 50.0, 5), (0.56, 0, 15, 100.0, 5),
+    (0.02, -7, 7, 50.0, 0), (0.05, -128, 127, 40.0, 0), (0.3, 2, 2, 10.0, 0)])
+def test_soft_histogram_and_its_entropy(torch, q, lo, hi, alpha, window):
+    # Sec. V-C, Eq. (25): sum of CPMFs per level in 2^-32 fixed point, entropy of the marginal PMF via cdl_index_entropy
+    n = 300007
+    centre = 0.5 * (lo + hi) * q
+    x = (inputs.normal((n,), max(hi - lo, 2) * q / 4.0, seed=lo + hi + 3) + f32(centre)).astype(f32)
+    if lo == 0:
+        x = np.abs(x)
+    P = cdl.QuantParams(q, lo, hi, alpha, window=window)
+    xd = dev(torch, x)
+    y = torch.empty(n, dtype=torch.float32, device="cuda")
+    sh = torch.full((P.nlev,), 77, dtype=torch.int64, device="cuda")
+    hist = torch.empty(P.nlev, dtype=torch.int64, device="cuda")
+    cdl.cdl_quantize_soft(xd, n, P, y, None, hist, soft_hist=sh)
+    ref = oracle.mpmf(x, f32(q), lo, hi, f32(alpha), window)
+    got = sh.cpu().numpy().view(np.uint64).astype(np.float64) / 2.0 ** 32
+    assert np.all(np.abs(got - ref) <= 5e-6 * ref + 1e-9 * n + 1e-6), np.max(np.abs(got - ref))
+    assert abs(got.sum() - n) <= 2e-6 * n
+    # the soft value and the count histogram of the same call are unchanged by the extra output
+    assert_soft_close(y.cpu().numpy(), oracle.soft(x, f32(q), lo, hi, f32(alpha), window), q)
+    assert np.array_equal(hist.cpu().numpy().view(np.uint64), oracle.hard(x, f32(q), lo, hi)[1])
+    H = torch.zeros(1, dtype=torch.float64, device="cuda")
+    lp = torch.zeros(P.nlev, dtype=torch.float32, device="cuda")
+    cdl.cdl_index_entropy(sh, P.nlev, H, lp)
+    p = ref / ref.sum()
+    refH = float(-np.sum(p[p > 0] * np.log2(p[p > 0])))
+    assert abs(float(H.cpu()[0]) - refH) <= 2e-5
+    np.testing.assert_allclose(lp.cpu().numpy(), p, rtol=1e-5, atol=1e-9)
+    # determinism: integer accumulation gives the same bits on a second run
+    sh2 = torch.zeros(P.nlev, dtype=torch.int64, device="cuda")
+    cdl.cdl_quantize_soft(xd, n, P, y, None, None, soft_hist=sh2)
+    assert torch.equal(sh, sh2)
