@@ -33,8 +33,25 @@
 namespace cdl {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kBatch = 4;  // float4 loads in flight per thread
+// Launch shape (overridable at build time for tuning runs)
+#ifndef CDL_Q_THREADS
+#define CDL_Q_THREADS 256
+#endif
+#ifndef CDL_Q_BATCH
+#define CDL_Q_BATCH 4
+#endif
+#ifndef CDL_Q_MINBLOCKS
+#define CDL_Q_MINBLOCKS 1
+#endif
+#ifdef CDL_Q_PLAIN_LDST
+#define CDL_LD(p) (*(p))
+#define CDL_ST(p, v) (*(p) = (v))
+#else
+#define CDL_LD(p) __ldcs(p)
+#define CDL_ST(p, v) __stcs(p, v)
+#endif
+constexpr int kThreads = CDL_Q_THREADS;
+constexpr int kBatch = CDL_Q_BATCH;  // float4 loads in flight per thread
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
 // |quotient - nearest integer| above this may be a rounding tie once the 3-ulp error of the reciprocal product is
@@ -133,6 +150,9 @@ template <int MODE, int PATH, bool RATE>
 __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__restrict__ Ltab, float x, float g,
                                               unsigned long long *mp_s = nullptr, int lane = 0)
 {
+    // the third template flag means "rate term" in the backward pass and "soft histogram" in the soft pass
+    constexpr bool kRate = RATE && MODE == MODE_BWD;
+    constexpr bool kSoftHist = RATE && MODE == MODE_SOFT;
     ElemOut o;
     const float q = P.q;
     // ---- hard index: rint(clamp(RN(x / q))), a NaN quotient clamps to lo.  x * RN(1/q) is within 3 ulp of the
@@ -177,7 +197,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rS = rcp_approx(1.0f + e1 + em);
         m1 = (e1 - em) * rS;
         o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
-        if (MODE == MODE_SOFT && mp_s != nullptr) {
+        if (kSoftHist) {
             mp_add(mp_s, ki - P.lo, lane, rS);
             if (e1 > 0.0f) mp_add(mp_s, ki + 1 - P.lo, lane, e1 * rS);
             if (em > 0.0f) mp_add(mp_s, ki - 1 - P.lo, lane, em * rS);
@@ -186,7 +206,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
             const float m2 = (e1 + em) * rS;         // E J^2; E J^3 = E J
             varj = fmaf(-m1, m1, m2);
             covj = m1 - m1 * m2;
-            if (RATE) {
+            if (kRate) {
                 const float Lc = Ltab[ki - P.lo];
                 const float l1 = (Ltab[min(ki + 1, P.hi) - P.lo] - Lc) * e1;
                 const float lm = (Ltab[max(ki - 1, P.lo) - P.lo] - Lc) * em;
@@ -204,7 +224,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         float ev[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
         const float *Lp = Ltab;
         float Lc = 0.0f;
-        if (RATE) {
+        if (kRate) {
             Lc = Ltab[ki - P.lo];
             Lp = Ltab + (min(max(ki - 2, P.lo), P.hi - 4) - P.lo);
         }
@@ -212,7 +232,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         for (int i = 0; i < 5; ++i) {
             const float jf = j0 + (float)i;
             const float e = ex2_approx(jf * fmaf(-P.A, jf, B));
-            if (MODE == MODE_SAMPLE || MODE == MODE_SOFT) ev[i] = e;
+            if (MODE == MODE_SAMPLE || kSoftHist) ev[i] = e;
             T0 += e;
             if (i > 0) T1 = fmaf((float)i, e, T1);
             if (MODE == MODE_BWD) {
@@ -220,7 +240,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                     T2 = fmaf((float)(i * i), e, T2);
                     T3 = fmaf((float)(i * i * i), e, T3);
                 }
-                if (RATE) {
+                if (kRate) {
                     const float le = (Lp[i] - Lc) * e;
                     R0 += le;
                     if (i > 0) R1 = fmaf((float)i, le, R1);
@@ -244,7 +264,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rT = rcp_approx(T0);
         const float mi = T1 * rT;                      // E I, I = level - st
         o.y = __fmaf_rn(stf, q, __fmul_rn(q, mi));
-        if (MODE == MODE_SOFT && mp_s != nullptr) {
+        if (kSoftHist) {
             const int b0 = min(max(ki - 2, P.lo), P.hi - 4) - P.lo;
 #pragma unroll
             for (int i = 0; i < 5; ++i) mp_add(mp_s, b0 + i, lane, ev[i] * rT);
@@ -254,7 +274,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
             const float m2i = T2 * rT, m3i = T3 * rT;
             varj = fmaf(-mi, mi, m2i);
             covj = fmaf(-mi, m2i, m3i) + 2.0f * j0 * varj;   // Cov(J, J^2) with J = I + j0
-            if (RATE) rate = (R1 - mi * R0) * rT;
+            if (kRate) rate = (R1 - mi * R0) * rT;
         }
     } else {
         int jlo, jhi;
@@ -272,7 +292,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         }
         const float B = P.c1x2 * dh;
         float S = 0.0f, S1 = 0.0f, S2 = 0.0f, S3 = 0.0f, R0 = 0.0f, R1 = 0.0f;
-        const float Lc = RATE ? Ltab[ki - P.lo] : 0.0f;
+        const float Lc = kRate ? Ltab[ki - P.lo] : 0.0f;
         const float *Lp = Ltab + (ki - P.lo);
         float jf = (float)jlo;
         for (int j = jlo; j <= jhi; ++j, jf += 1.0f) {
@@ -283,7 +303,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
                 const float j2 = jf * jf;
                 S2 = fmaf(j2, e, S2);
                 S3 = fmaf(j2 * jf, e, S3);
-                if (RATE) {
+                if (kRate) {
                     const float le = (Lp[j] - Lc) * e;
                     R0 += le;
                     R1 = fmaf(jf, le, R1);
@@ -309,7 +329,7 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
         const float rS = rcp_approx(S);
         m1 = S1 * rS;
         o.y = __fmaf_rn(kn, q, __fmul_rn(q, m1));
-        if (MODE == MODE_SOFT && mp_s != nullptr) {
+        if (kSoftHist) {
             float jj = (float)jlo;
             for (int j = jlo; j <= jhi; ++j, jj += 1.0f)
                 mp_add(mp_s, ki + j - P.lo, lane, ex2_approx(jj * fmaf(-P.A, jj, B)) * rS);
@@ -318,12 +338,12 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
             const float m2 = S2 * rS, m3 = S3 * rS;
             varj = fmaf(-m1, m1, m2);
             covj = fmaf(-m1, m2, m3);
-            if (RATE) rate = (R1 - m1 * R0) * rS;
+            if (kRate) rate = (R1 - m1 * R0) * rS;
         }
     }
     if (MODE == MODE_BWD) {
         float gx = g * (P.a2 * varj);
-        if (RATE) gx = fmaf(P.rate_c, rate, gx);
+        if (kRate) gx = fmaf(P.rate_c, rate, gx);
         o.gx = gx;
         const float dmk = fmaf(-kn, q, dh);            // d - kn q
         const float dq = (kn + m1) + P.two_aq * (dmk * varj - q * covj);
@@ -342,7 +362,7 @@ __device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane
 // Vector region: elements [head, head + 4 n4); the remaining head + tail elements are done one by one.
 // When the pointers do not allow 128-bit access the host passes n4 = 0 and everything is scalar.
 template <int MODE, int PATH, bool RATE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, CDL_Q_MINBLOCKS)
 quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__restrict__ g, int64_t n,
                 int64_t head, int64_t n4, float *__restrict__ y, unsigned char *__restrict__ idx,
                 unsigned long long *__restrict__ hist, float *__restrict__ gx,
@@ -355,13 +375,13 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     const bool do_hist = hist != nullptr;
     // soft histogram (sum of CPMFs per level, fixed point): bins behind the index histogram's, only when asked for
     unsigned long long *mp_s = nullptr;
-    if (MODE == MODE_SOFT && mp != nullptr) {
+    if (MODE == MODE_SOFT && RATE) {
         mp_s = reinterpret_cast<unsigned long long *>(smem_raw + CDL_MAX_LEVELS * sizeof(float) +
                                                       (do_hist ? (size_t)P.nlev * 32 * sizeof(unsigned int) : 0));
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) mp_s[k] = 0ull;
     }
 
-    if (RATE) {
+    if (MODE == MODE_BWD && RATE) {
         for (int k = threadIdx.x; k < P.nlev; k += kThreads) {
             const float p = P.level_prob[k];
             Ltab[k] = (p < 9.31322574615478515625e-10f) ? -30.0f : log2f(p);   // 2^-30
@@ -369,7 +389,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     }
     if (do_hist)
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) hist_s[k] = 0u;
-    if (RATE || do_hist || mp_s != nullptr) __syncthreads();
+    if (RATE || do_hist) __syncthreads();
 
     double acc_q = 0.0, acc_a = 0.0;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
@@ -387,8 +407,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         for (int b = 0; b < kBatch; ++b) {
             const int64_t i = base + b * stride;
             if (i < n4) {
-                xv[b] = __ldcs(x4 + i);
-                if (MODE == MODE_BWD) gv[b] = __ldcs(g4 + i);
+                xv[b] = CDL_LD(x4 + i);
+                if (MODE == MODE_BWD) gv[b] = CDL_LD(g4 + i);
             }
         }
         float part_q = 0.0f, part_a = 0.0f;
@@ -430,8 +450,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     packed |= ((unsigned int)o.k0 & 0xffu) << (8 * c);
                     if (MODE != MODE_BWD && do_hist) hist_add(hist_s, o.k0 - P.lo, lane);
                 }
-                if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) __stcs(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
-                if (MODE == MODE_BWD && gx != nullptr) __stcs(gx4 + i, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
+                if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) CDL_ST(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
+                if (MODE == MODE_BWD && gx != nullptr) CDL_ST(gx4 + i, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
                 if (MODE != MODE_BWD && idx != nullptr) idx4[i] = packed;
             }
         }
@@ -460,7 +480,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         }
     }
 
-    if (MODE == MODE_SOFT && mp_s != nullptr) {
+    if (MODE == MODE_SOFT && RATE) {   // RATE doubles as "soft histogram requested" in the soft pass
         __syncthreads();
         const int warp = threadIdx.x >> 5;
         for (int b = warp; b < P.nlev; b += kThreads / 32) {
@@ -583,6 +603,10 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
         case MODE_HARD:
             return CDL_Q(MODE_HARD, PATH_LOOP, false);
         case MODE_SOFT:
+            if (soft_hist != nullptr)
+                return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, true)
+                     : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, true)
+                                         : CDL_Q(MODE_SOFT, PATH_LOOP, true);
             return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, false)
                  : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, false)
                                      : CDL_Q(MODE_SOFT, PATH_LOOP, false);
