@@ -243,9 +243,11 @@ int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_d
  * 256-byte status block at its start.  0 for an unknown op or non-positive sizes. */
 size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K);
 
-/* Synchronises `stream`, reads the status block at the start of a GEMM workspace and returns CDL_OK
- * or CDL_ERR_TIMEOUT (a device-side wait gave up; the outputs of that call are then undefined). */
-int cdl_workspace_status(const void *ws, void *stream);
+/* Synchronises `stream` and reports whether a bounded device-side wait of a GEMM call that used this workspace
+ * gave up: CDL_ERR_TIMEOUT (the outputs of that call are then undefined; the record is cleared by this call) or
+ * CDL_OK.  The GEMM calls never touch the first word of a workspace unless a wait expires, in which case they
+ * store CDL_ERR_TIMEOUT there and it stays until read here; any other content (a fresh allocation) reads as OK. */
+int cdl_workspace_status(void *ws, void *stream);
 
 /* Static, NUL-terminated description of a status code. */
 const char *cdl_strerror(int status);

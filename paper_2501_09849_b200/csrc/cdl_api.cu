@@ -241,7 +241,7 @@ size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
     }
 }
 
-int cdl_workspace_status(const void *ws, void *stream)
+int cdl_workspace_status(void *ws, void *stream)
 {
     if (ws == nullptr) return CDL_ERR_WORKSPACE;
     int32_t word = 0;
@@ -251,7 +251,9 @@ int cdl_workspace_status(const void *ws, void *stream)
         (void)cudaGetLastError();
         return CDL_ERR_LAUNCH;
     }
-    return word == 0 ? CDL_OK : CDL_ERR_TIMEOUT;
+    if (word != CDL_ERR_TIMEOUT) return CDL_OK;     // kernels write nothing but this code into the word
+    if (cudaMemsetAsync(ws, 0, sizeof word, st) != cudaSuccess) (void)cudaGetLastError();
+    return CDL_ERR_TIMEOUT;
 }
 
 int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, const void *W_idx, int64_t ldw,
@@ -274,10 +276,6 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, con
     if (acc_out != nullptr && overflow_risk(K, ra, rw)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return CDL_ERR_LAUNCH;
-    }
     const float scale = (a->q * w->q);
     GemmOperand X{A_idx, lda, 1, ra.is_unsigned, (int)ra.absmax};
     GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
@@ -315,10 +313,6 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
     if (dWacc != nullptr && overflow_risk(M, ra, rg)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return CDL_ERR_LAUNCH;
-    }
     if (want_dx) {
         // dX[m,k] = sum_n G[m,n] W[k,n]
         GemmOperand X{G_idx, ldg, 1, false, (int)rg.absmax};

@@ -575,8 +575,12 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
         }
     }
     if (mode == MODE_BWD) {
-        if (grad_q && cudaMemsetAsync(grad_q, 0, sizeof(double), stream) != cudaSuccess) return CDL_ERR_LAUNCH;
-        if (grad_alpha && cudaMemsetAsync(grad_alpha, 0, sizeof(double), stream) != cudaSuccess) return CDL_ERR_LAUNCH;
+        if (grad_q != nullptr && grad_alpha == grad_q + 1) {       // adjacent scalars: one clear
+            if (cudaMemsetAsync(grad_q, 0, 2 * sizeof(double), stream) != cudaSuccess) return CDL_ERR_LAUNCH;
+        } else {
+            if (grad_q && cudaMemsetAsync(grad_q, 0, sizeof(double), stream) != cudaSuccess) return CDL_ERR_LAUNCH;
+            if (grad_alpha && cudaMemsetAsync(grad_alpha, 0, sizeof(double), stream) != cudaSuccess) return CDL_ERR_LAUNCH;
+        }
     }
     if (n == 0) return CDL_OK;
 
