@@ -497,7 +497,7 @@ def run_network(args):
         "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": tot_q / (quant_ms * 1e-3) / 1e9,
         "layers": table, "clocks": clocks, "peak_hbm_gbs": hbm, "peak_source": pk_kind,
         "e2e": None, "e2e_note": "not measured for this workload (a step's inputs are ~11 GB); see the default workload",
-        "gpu_launches": steps * len(layers) * len(CALLS)}), flush=True)
+        "gpu_launches": steps * sum(st.kernels_per_step() for *_, st in layers)}), flush=True)
 
 
 def main():
@@ -666,7 +666,7 @@ def main():
             "kernels": kernels, "roofline": roof, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e_steps},
-            "gpu_launches": args.steps * len(CALLS), "device_status": status,
+            "gpu_launches": args.steps * step.kernels_per_step(), "device_status": status,
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle

@@ -72,6 +72,12 @@ class CdlLayerStep:
         self.dw_desc = cdl.IndexDesc(wq.q, wq.lo, wq.hi)
         self.dg = cdl.IndexDesc(self.q_g, -127, 127)
 
+    def kernels_per_step(self):
+        """Kernels of this library one step launches: one per call, plus the small kernel that turns the split
+        weight-gradient reduction into floats when the reduction over M is split across SMs."""
+        split_dw = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, self.M, self.N, self.K) > 256
+        return len(CALLS) - (0 if self.need_dx else 1) + (1 if split_dw else 0)
+
     def input_tensors(self):
         return {"w": self.w, "x": self.x, "A_idx": self.A_idx, "dY": self.dY, "gx_in": self.gx_in}
 
