@@ -29,12 +29,15 @@ namespace cdl {
 namespace {
 
 constexpr int kThreadsTC = 192;
-constexpr int kStages = 4;
+constexpr int kStagesSingle = 4;        // one CTA per tile: 16 KB of X + up to 32 KB of Y per stage
+constexpr int kStagesPair = 6;          // CTA pair per 256-row tile: 16 KB of X + 16 KB of Y per stage and CTA
+constexpr int kStagesMax = 6;
 constexpr int TM = 128;                 // output rows per tile = UMMA M
 constexpr int BR = 128;                 // bytes (= elements) of the reduced dimension per stage
 constexpr int kABytes = TM * BR;        // 16 KB
 constexpr int kBBytesMax = 256 * BR;    // 32 KB
-constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kStageBytesSingle = kABytes + kBBytesMax;
+constexpr int kStageBytesPair = kABytes + 128 * BR;
 constexpr int kOutBytes = TM * 128;     // epilogue staging block: 128 rows x 32 four-byte columns
 // The whole 227 KB opt-in window is requested (stages need 193 KB): operand descriptors then address
 // allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
@@ -114,6 +117,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// Load issued by either CTA of a pair into its own shared memory; the bytes are counted on the barrier at offset
+// `bar` of CTA 0 (no multicast: each CTA fetches its own box).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .b32 rb;\n\t"
+        "mapa.shared::cluster.u32 rb, %4, 0;\n\t"
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3}], [rb];\n\t}"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int c0, int c1, uint32_t src)
 {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
@@ -146,6 +161,43 @@ __device__ __forceinline__ bool epi_all(bool v)
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// ---- CTA-pair helpers (cluster of two CTAs, cta_group::2)
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank)
+{
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank)
+        : "memory");
+}
+// both CTAs of the pair get the arrival (same barrier offset in each)
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
 
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
@@ -190,13 +242,21 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
+// PAIR = false: one CTA per 128 x TN tile.  PAIR = true (TN = 256): a cluster of two CTAs per 256 x 256 tile with
+// tcgen05.mma.cta_group::2: CTA r of the pair stages rows [128 r, 128 r + 128) of X and columns [128 r, 128 r + 128)
+// of Y, the MMA issued by CTA 0 reads both halves from both shared memories and each CTA's TMEM receives its 128
+// rows of the 256 x 256 accumulator.  A byte staged by either CTA then feeds twice as many multiply-adds, which is
+// what the shared-memory-capacity x latency product of one SM cannot otherwise sustain.  Hand-shake in pair mode:
+// the TMA loads of both CTAs count their bytes on CTA 0's "stage full" barrier; tcgen05.commit multicasts "stage
+// free" and "accumulator full" to both CTAs; the epilogues of both CTAs arrive on CTA 0's "accumulator free" barrier.
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreadsTC, 1)
 index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_f, const __grid_constant__ CUtensorMap map_acc,
                      const TcParams P)
 {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) unsigned long long bars[2 * kStages + 4];
+    __shared__ __align__(8) unsigned long long bars[2 * kStagesMax + 4];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -205,10 +265,17 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const int lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
 
+    constexpr int kStages = PAIR ? kStagesPair : kStagesSingle;
+    constexpr int kStageBytes = PAIR ? kStageBytesPair : kStageBytesSingle;
+    constexpr int TMU = PAIR ? 2 * TM : TM;                   // rows of a work unit's tile
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // CTA 0 of a pair issues the MMAs
+    const int cta_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int cta_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+
     auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
-    auto empty_bar = [&](int s) { return smem_u32(&bars[kStages + s]); };
-    auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * kStages + b]); };
-    auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * kStages + 2 + b]); };
+    auto empty_bar = [&](int s) { return smem_u32(&bars[kStagesMax + s]); };
+    auto tfull_bar = [&](int b) { return smem_u32(&bars[2 * kStagesMax + b]); };
+    auto tempty_bar = [&](int b) { return smem_u32(&bars[2 * kStagesMax + 2 + b]); };
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -218,23 +285,32 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), 4);
+            mbar_init(tempty_bar(b), PAIR ? 8 : 4);       // one arrival per epilogue warp (of both CTAs in pair mode)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();       // both CTAs' barriers exist before any remote arrive or multicast commit
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
     const int units = P.tiles_i * P.tiles_j * P.splits;
-    const int b_blocks = (P.TN + 127) / 128;                              // 128-wide blocks of an MN-major B tile
-    const uint32_t b_bytes = P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR);
+    const int b_blocks = PAIR ? 1 : (P.TN + 127) / 128;                   // 128-wide blocks of an MN-major B tile
+    const uint32_t b_bytes = PAIR ? (uint32_t)(128 * BR)
+                                  : (P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR));
+    const int brow = PAIR ? (int)rank * 128 : 0;                          // this CTA's share of the Y tile
     const uint32_t stage_tx = (uint32_t)kABytes + b_bytes;
     bool failed = false;
 
@@ -242,7 +318,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // ------------------------------------------------------------ TMA producer (one lane)
         if (lane == 0) {
             uint32_t it = 0;
-            for (int u = blockIdx.x; u < units && !failed; u += gridDim.x) {
+            for (int u = cta_first; u < units && !failed; u += cta_step) {
                 const int split = u % P.splits;
                 const int tile = u / P.splits;
                 const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
@@ -257,9 +333,19 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     }
                     const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
                     const uint32_t sb = sa + kABytes;
+                    const int arow = ti * TMU + (int)rank * TM;
+                    if (PAIR) {
+                        // both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
+                        if (rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_tx);
+                        if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
+                        else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
+                        if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, tj * P.TN + brow, rb * BR, full_bar(s));
+                        else tma_load_2d_pair(sb, &map_b, rb * BR, tj * P.TN + brow, full_bar(s));
+                        continue;
+                    }
                     mbar_expect_tx(full_bar(s), stage_tx);
-                    if (P.a_mn_major) tma_load_2d(sa, &map_a, ti * TM, rb * BR, full_bar(s));   // {i (inner), r}
-                    else tma_load_2d(sa, &map_a, rb * BR, ti * TM, full_bar(s));                 // {r (inner), i}
+                    if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
+                    else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
                     if (P.b_mn_major) {
                         for (int bb = 0; bb < b_blocks; ++bb)
                             tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, tj * P.TN + bb * 128, rb * BR, full_bar(s));
@@ -274,10 +360,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer (one lane)
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (one lane; CTA 0 in pair mode)
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0, tcount = 0;
-            for (int u = blockIdx.x; u < units && !failed; u += gridDim.x, ++tcount) {
+            for (int u = cta_first; u < units && !failed; u += cta_step, ++tcount) {
                 const int split = u % P.splits;
                 const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
                 const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
@@ -307,12 +393,19 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
                     const uint32_t b_step = P.b_mn_major ? (4096u >> 4) : (32u >> 4);
 #pragma unroll
-                    for (int k = 0; k < BR / 32; ++k)
-                        tc_mma_i8(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc,
-                                  (rb > rb0 || k > 0) ? 1u : 0u);
-                    tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
+                    for (int k = 0; k < BR / 32; ++k) {
+                        const uint32_t acc = (rb > rb0 || k > 0) ? 1u : 0u;
+                        if (PAIR) tc_mma_i8_pair(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc, acc);
+                        else tc_mma_i8(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc, acc);
+                    }
+                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                    if (PAIR) tc_commit_pair(empty_bar(s));
+                    else tc_commit(empty_bar(s));
                 }
-                if (!failed) tc_commit(tfull_bar(buf));  // accumulator complete
+                if (!failed) {                               // accumulator complete
+                    if (PAIR) tc_commit_pair(tfull_bar(buf));
+                    else tc_commit(tfull_bar(buf));
+                }
             }
             if (failed) {
                 abort_s = 1;
@@ -379,7 +472,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             ++ocount;
         };
 
-        for (int u = blockIdx.x; u < units; u += gridDim.x, ++tcount) {
+        for (int u = cta_first; u < units; u += cta_step, ++tcount) {
             const int tile = u / P.splits;
             const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
             const int slab_row0 = (u % P.splits) * P.slab_rows;     // 0 unless partial tiles go to per-split slabs
@@ -391,22 +484,23 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 break;
             }
             tc_fence_after();
+            const int trow0 = ti * TMU + (int)rank * TM;     // first output row of this CTA's part of the tile
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
             for (int c0 = 0; c0 < P.TN; c0 += 32) {
                 const int col0 = tj * P.TN + c0;
-                if (col0 >= P.J) break;             // uniform over the CTA
+                if (col0 >= P.J || trow0 >= P.I) break;             // uniform over the CTA
                 uint32_t v[32];
                 tc_ld32(taddr + (uint32_t)c0, v);
                 tc_wait_ld();
                 const int ncol = min(min(32, P.TN - c0), P.J - col0);
                 if (P.splits > 1) {
-                    if (P.tma_acc) stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + ti * TM);
-                    else stage_and_copy(v, P.acc_out, P.slab_rows == 0, slab_row0, ti * TM, col0, ncol);
+                    if (P.tma_acc) stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + trow0);
+                    else stage_and_copy(v, P.acc_out, P.slab_rows == 0, slab_row0, trow0, col0, ncol);
                     continue;
                 }
                 if (P.acc_out != nullptr) {
-                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, ti * TM);
-                    else stage_and_copy(v, P.acc_out, false, 0, ti * TM, col0, ncol);
+                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, trow0);
+                    else stage_and_copy(v, P.acc_out, false, 0, trow0, col0, ncol);
                 }
                 if (P.f_out != nullptr) {
                     uint32_t f[32];
@@ -417,13 +511,16 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
                     }
-                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, ti * TM);
-                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, ti * TM, col0, ncol);
+                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, trow0);
+                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, trow0, col0, ncol);
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_remote(tempty_bar(buf), 0u);
+                else mbar_arrive(tempty_bar(buf));
+            }
         }
         if (leader) bulk_wait_all();                // staged blocks are out before shared memory goes away
         if (failed && lane == 0) {
@@ -435,9 +532,11 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();       // neither CTA leaves while its partner may still touch its shared memory / TMEM
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
 
@@ -512,7 +611,7 @@ bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t out
     const cuuint32_t box[2] = {128u, box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -521,22 +620,32 @@ bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t out
 namespace {
 // Split of the reduced dimension: when the tiles alone cannot occupy half of the device, and always into at
 // least min_splits parts (the caller's bound that keeps every part's int32 partial sums exact).
-void plan(int I, int J, int R, int min_splits, int *TN_out, int *splits_out)
+struct Plan {
+    int TN;         // output columns per tile
+    int splits;     // parts of the reduced dimension
+    int pair;       // 1: CTA pairs on 256-row tiles
+    int tile_rows;  // output rows per work unit (128, or 256 for a pair)
+};
+
+Plan plan(int I, int J, int R, int min_splits)
 {
-    int TN = 256;
-    while (TN > 16 && TN / 2 >= J) TN /= 2;
-    const long long tiles = (long long)((I + TM - 1) / TM) * ((J + TN - 1) / TN);
+    Plan p;
+    p.TN = 256;
+    while (p.TN > 16 && p.TN / 2 >= J) p.TN /= 2;
+    p.pair = (p.TN == 256 && I > TM) ? 1 : 0;
+    p.tile_rows = p.pair ? 2 * TM : TM;
+    const int slots = p.pair ? kPlanSMs / 2 : kPlanSMs;      // work units that run at once
+    const long long tiles = (long long)((I + p.tile_rows - 1) / p.tile_rows) * ((J + p.TN - 1) / p.TN);
     const int rblocks = (R + BR - 1) / BR;
-    int splits = 1;
-    if (tiles * 2 <= kPlanSMs) {
-        splits = (int)(kPlanSMs / tiles);
+    p.splits = 1;
+    if (tiles * 2 <= slots) {
+        p.splits = (int)(slots / tiles);
         const int max_splits = (rblocks + 3) / 4;      // keep at least four stages of work per unit
-        if (splits > max_splits) splits = max_splits;
-        if (splits < 1) splits = 1;
+        if (p.splits > max_splits) p.splits = max_splits;
+        if (p.splits < 1) p.splits = 1;
     }
-    if (splits < min_splits) splits = min_splits;
-    *TN_out = TN;
-    *splits_out = splits;
+    if (p.splits < min_splits) p.splits = min_splits;
+    return p;
 }
 
 // Parts the reduced dimension must be cut into so that a part's sum of |x| * |y| stays below 2^31 (whole r-blocks).
@@ -555,14 +664,13 @@ int min_exact_splits(int R, long long xmax, long long ymax)
 // is long enough that its int32 total could overflow for byte operands of the widest range, the per-split slabs.
 size_t tc_gemm_scratch_bytes(int I, int J, int R)
 {
-    int TN, splits;
-    plan(I, J, R, 1, &TN, &splits);
+    Plan p = plan(I, J, R, 1);
     size_t need = 0;
-    if (splits > 1) need = (size_t)I * (size_t)J * sizeof(int32_t);
+    if (p.splits > 1) need = (size_t)I * (size_t)J * sizeof(int32_t);
     if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
-        plan(I, J, R, min_exact_splits(R, 255, 128), &TN, &splits);
-        const size_t slab = (size_t)((I + TM - 1) / TM) * TM * (size_t)J * sizeof(int32_t);
-        if (slab * splits > need) need = slab * splits;
+        p = plan(I, J, R, min_exact_splits(R, 255, 128));
+        const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
+        if (slab * p.splits > need) need = slab * p.splits;
     }
     return (need + 255u) & ~(size_t)255u;
 }
@@ -585,11 +693,12 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     // keeps its own slab, and the slabs are summed in int64 (float output only).
     const bool wide = (long long)R * X.absmax * Y.absmax >= ((long long)1 << 31);
     if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
-    int TN, splits;
-    plan(I, J, R, wide ? min_exact_splits(R, X.absmax, Y.absmax) : 1, &TN, &splits);
+    const Plan pl = plan(I, J, R, wide ? min_exact_splits(R, X.absmax, Y.absmax) : 1);
+    const int TN = pl.TN, splits = pl.splits;
+    const bool pair = pl.pair != 0;
     P.TN = TN;
-    P.slab_rows = wide ? ((I + TM - 1) / TM) * TM : 0;
-    P.tiles_i = (I + TM - 1) / TM;
+    P.tiles_i = (I + pl.tile_rows - 1) / pl.tile_rows;
+    P.slab_rows = wide ? P.tiles_i * pl.tile_rows : 0;
     P.tiles_j = (J + TN - 1) / TN;
     P.rblocks = (R + BR - 1) / BR;
     const int sms = sm_count();
@@ -600,7 +709,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.a_mn_major = a_mn ? 1 : 0;
     P.b_mn_major = b_mn ? 1 : 0;
     P.idesc = (2u << 4) | ((X.is_unsigned ? 0u : 1u) << 7) | ((Y.is_unsigned ? 0u : 1u) << 10) |
-              ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+              ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(pl.tile_rows >> 4) << 24);
     P.scale = scale;
     P.bias = bias;
     P.status = status;
@@ -625,7 +734,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
     else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
-    else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, (uint32_t)TN);
+    else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
     // outputs through shared memory + TMA when their pitch and base allow it and the tile is at least one box wide
     CUtensorMap map_f = map_a, map_acc = map_a;      // placeholders when unused
     const bool out_ok = TN >= 32 && (J & 3) == 0;
@@ -643,18 +752,58 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     if (!ok) return CDL_ERR_LAUNCH;
 
     static bool attr_set[64];
+    static int pair_slots[64];         // CTA pairs the device runs at once
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(index_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+    if (dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(index_gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(index_gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return CDL_ERR_LAUNCH;
         }
+        cudaLaunchConfig_t qc = {};
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = 2;
+        qa[0].val.clusterDim.y = 1;
+        qa[0].val.clusterDim.z = 1;
+        qc.gridDim = dim3(2 * (sms / 2));
+        qc.blockDim = dim3(kThreadsTC);
+        qc.dynamicSmemBytes = kSmemBytes;
+        qc.attrs = qa;
+        qc.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, index_gemm_tc_kernel<true>, &qc) != cudaSuccess || nclusters < 1) {
+            (void)cudaGetLastError();
+            nclusters = sms / 2;
+        }
+        pair_slots[dev] = nclusters < sms / 2 ? nclusters : sms / 2;
         attr_set[dev] = true;
     }
     const long long units = tiles * splits;
-    const int grid = (int)(units < sms ? units : sms);
-    index_gemm_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+    if (pair) {
+        const int slots = pair_slots[dev];
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3(2u * (unsigned)(units < slots ? units : slots));
+        cfg.blockDim = dim3(kThreadsTC);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = stream;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true>, map_a, map_b, map_f, map_acc, P) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+    } else {
+        const int grid = (int)(units < sms ? units : sms);
+        index_gemm_tc_kernel<false><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+    }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (f_out != nullptr && (splits > 1 || wide)) {
         const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
