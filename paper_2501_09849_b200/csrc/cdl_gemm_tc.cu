@@ -12,11 +12,12 @@
 // pipeline stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is
 // [rows][128 bytes] with the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or
 // columns outside the matrix are zero-filled by TMA, which makes ragged edges and R tails exact.
-// Warp roles (192 threads): warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2-5 run the
+// Warp roles (320 threads): warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2-9 run the
 // epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
-// Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to a
-// swizzled 128 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that
-// global memory sees whole 128-byte lines.  Work units are (tile, split of the reduced dimension); with more
+// Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to the warp's
+// swizzled 32 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that
+// global memory sees whole 128-byte lines.  The per-chunk chain (TMEM load, convert, stage, proxy fence, store)
+// is a string of latencies, so two warps share each TMEM lane quarter and take alternate chunks.  Work units are (tile, split of the reduced dimension); with more
 // than one split the staging block is added into an int32 buffer with a TMA bulk reduce-add (integer, so the
 // result does not depend on order).  Outputs whose pitch or base is not 16-byte aligned, and tiles 16 columns
 // wide, go through the same staging block and are copied out by the warps one row at a time.
@@ -28,9 +29,14 @@
 namespace cdl {
 namespace {
 
-constexpr int kThreadsTC = 192;
-constexpr int kStagesSingle = 4;        // one CTA per tile: 16 KB of X + up to 32 KB of Y per stage
-constexpr int kStagesPair = 6;          // CTA pair per 256-row tile: 16 KB of X + 16 KB of Y per stage and CTA
+constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each taking every other 32-column chunk
+constexpr int kThreadsTC = 64 + 32 * kEpiWarps;
+// Shared memory is divided between operand stages and epilogue staging blocks (4 KB each, per epilogue warp).
+// Which of the two needs the bytes in flight depends on the shape: a long reduced dimension loads much more than
+// it stores, a short one (two stages per 128 KB of output) the opposite.
+//                                          load-heavy           store-heavy
+//   one CTA per tile  (48 KB stages)       4 stages + 1 block   3 stages + 2 blocks
+//   CTA pair per tile (32 KB stages)       6 stages + 1 block   4 stages + 3 blocks
 constexpr int kStagesMax = 6;
 constexpr int TM = 128;                 // output rows per tile = UMMA M
 constexpr int BR = 128;                 // bytes (= elements) of the reduced dimension per stage
@@ -38,7 +44,7 @@ constexpr int kABytes = TM * BR;        // 16 KB
 constexpr int kBBytesMax = 256 * BR;    // 32 KB
 constexpr int kStageBytesSingle = kABytes + kBBytesMax;
 constexpr int kStageBytesPair = kABytes + 128 * BR;
-constexpr int kOutBytes = TM * 128;     // epilogue staging block: 128 rows x 32 four-byte columns
+constexpr int kOutWarpBytes = 32 * 128;  // epilogue staging block of one warp: 32 rows x 32 four-byte columns
 // The whole 227 KB opt-in window is requested (stages need 193 KB): operand descriptors then address
 // allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
 constexpr int kSmemBytes = 232448 - 1024;
@@ -140,21 +146,21 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int c0
                  ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// AND over the 128 epilogue threads (named barrier 1)
+// AND over the epilogue threads (named barrier 1)
 __device__ __forceinline__ bool epi_all(bool v)
 {
     uint32_t out;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(out)
-        : "r"((uint32_t)v)
+        : "r"((uint32_t)v), "n"(32 * kEpiWarps)
         : "memory");
     return out != 0;
 }
@@ -227,7 +233,21 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Wait for the TMEM loads in flight and tie the loaded registers to the wait, so that no use of them is scheduled
+// ahead of it.
+__device__ __forceinline__ void tc_wait_ld_pin(uint32_t (&v)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :
+                 : "memory");
+    asm volatile(""
+                 : "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                   "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :
+                 : "memory");
+}
 
 // Shared-memory operand descriptor (sm_100 format): start address, leading / stride byte offsets in 16-byte
 // units, version 1, 128-byte swizzle.
@@ -249,7 +269,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // what the shared-memory-capacity x latency product of one SM cannot otherwise sustain.  Hand-shake in pair mode:
 // the TMA loads of both CTAs count their bytes on CTA 0's "stage full" barrier; tcgen05.commit multicasts "stage
 // free" and "accumulator full" to both CTAs; the epilogues of both CTAs arrive on CTA 0's "accumulator free" barrier.
-template <bool PAIR>
+template <bool PAIR, bool STORE_HEAVY>
 __global__ void __launch_bounds__(kThreadsTC, 1)
 index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_f, const __grid_constant__ CUtensorMap map_acc,
@@ -265,8 +285,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const int lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
 
-    constexpr int kStages = PAIR ? kStagesPair : kStagesSingle;
+    constexpr int kStages = PAIR ? (STORE_HEAVY ? 4 : 6) : (STORE_HEAVY ? 3 : 4);
     constexpr int kStageBytes = PAIR ? kStageBytesPair : kStageBytesSingle;
+    constexpr int kOutBlocks = PAIR ? (STORE_HEAVY ? 3 : 1) : (STORE_HEAVY ? 2 : 1);      // per epilogue warp
+    static_assert(kStages * kStageBytes + kEpiWarps * kOutBlocks * kOutWarpBytes + 1024 <= kSmemBytes, "shared memory");
     constexpr int TMU = PAIR ? 2 * TM : TM;                   // rows of a work unit's tile
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // CTA 0 of a pair issues the MMAs
     const int cta_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -285,7 +307,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), PAIR ? 8 : 4);       // one arrival per epilogue warp (of both CTAs in pair mode)
+            mbar_init(tempty_bar(b), PAIR ? 2 * kEpiWarps : kEpiWarps);       // one arrival per epilogue warp (of both CTAs in pair mode)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -413,55 +435,52 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue warps 2..5
+        // ------------------------------------------------------------ epilogue warps 2..9
+        // Each warp works on its own: it reads its 32 TMEM lanes (= 32 output rows), stages 32 columns of them in a
+        // 4 KB block of its own and sends that block with its own TMA store, so the warps never wait for one
+        // another inside a tile; the TMEM load of the next 32 columns is in flight while the current ones are sent.
         const int quarter = warp & 3;               // TMEM lanes this warp may read: 32 * (warp % 4) ..
-        const int erow = quarter * 32 + lane;       // row of the tile owned by this thread
-        const bool leader = threadIdx.x == 64;      // issues and tracks the bulk stores
-        const uint32_t out_base = smem_base + (uint32_t)(kStages * kStageBytes);
+        const int half = (warp - 2) >> 2;           // which of the two warps of this quarter: chunks half, half + 2, ..
+        const uint32_t wbuf = smem_base + (uint32_t)(kStages * kStageBytes) + (uint32_t)((warp - 2) * kOutBlocks * kOutWarpBytes);
         uint32_t tcount = 0, ocount = 0;
 
-        // 32 four-byte values of this thread's row -> swizzled staging block -> TMA store or reduce-add
-        auto stage_and_send = [&](const uint32_t (&w)[32], const CUtensorMap *map, bool reduce, int col0, int row0) {
-            const uint32_t blk = out_base + (ocount & 1u) * (uint32_t)kOutBytes;
-            if (leader) bulk_wait_read_1();         // the block used two sends ago has been read out
-            epi_barrier();
-            const uint32_t dst = blk + (uint32_t)erow * 128u;
+        // 32 four-byte values of this thread's row -> this warp's swizzled staging block (its blocks in turn)
+        auto stage = [&](const uint32_t (&w)[32]) -> uint32_t {
+            const uint32_t blk = wbuf + ocount * (uint32_t)kOutWarpBytes;
+            if (lane == 0) bulk_wait_read<kOutBlocks - 1>();      // the send that last used this block has read it
+            __syncwarp();
+            const uint32_t dst = blk + (uint32_t)lane * 128u;
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4)
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c4 ^ (erow & 7)) << 4)),
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c4 ^ (lane & 7)) << 4)),
                              "r"(w[4 * c4]), "r"(w[4 * c4 + 1]), "r"(w[4 * c4 + 2]), "r"(w[4 * c4 + 3])
                              : "memory");
+            return blk;
+        };
+        // staged block -> TMA store or reduce-add of a {32 columns, 32 rows} box at (col0, row0)
+        auto stage_and_send = [&](const uint32_t (&w)[32], const CUtensorMap *map, bool reduce, int col0, int row0, int row_end) {
+            const uint32_t blk = stage(w);
             fence_async_smem();
-            epi_barrier();
-            if (leader) {
+            __syncwarp();
+            if (lane == 0 && row0 < row_end) {
                 if (reduce) tma_reduce_add_2d(map, col0, row0, blk);
                 else tma_store_2d(map, col0, row0, blk);
                 bulk_commit();
             }
-            ++ocount;
+            ocount = ocount + 1 == (uint32_t)kOutBlocks ? 0u : ocount + 1;      // next block; one copied out by the warp itself is reused at once
         };
-
-        // Same staging, then the warp copies its own 32 rows out itself, one row (up to 128 contiguous bytes) per
+        // Same staging, then the warp copies its 32 rows out itself, one row (up to 128 contiguous bytes) per
         // instruction: for outputs TMA cannot take (row pitch or base not a multiple of 16 bytes, 16-column tiles).
-        auto stage_and_copy = [&](const uint32_t (&w)[32], int32_t *out, bool reduce, long long row_off, int tile_row0,
+        auto stage_and_copy = [&](const uint32_t (&w)[32], int32_t *out, bool reduce, long long row_off, int row0,
                                   int col0, int ncol) {
-            const uint32_t blk = out_base + (ocount & 1u) * (uint32_t)kOutBytes;
-            if (leader) bulk_wait_read_1();
-            epi_barrier();
-            const uint32_t dst = blk + (uint32_t)erow * 128u;
-#pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4)
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((c4 ^ (erow & 7)) << 4)),
-                             "r"(w[4 * c4]), "r"(w[4 * c4 + 1]), "r"(w[4 * c4 + 2]), "r"(w[4 * c4 + 3])
-                             : "memory");
+            const uint32_t blk = stage(w);
             __syncwarp();
             for (int rr = 0; rr < 32; ++rr) {
-                const int rl = quarter * 32 + rr;
-                const int grow = tile_row0 + rl;
+                const int grow = row0 + rr;
                 if (grow >= P.I) break;                                    // uniform over the warp
                 uint32_t val;
                 asm volatile("ld.shared.b32 %0, [%1];" : "=r"(val)
-                             : "r"(blk + (uint32_t)rl * 128u + (uint32_t)(((lane >> 2) ^ (rl & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
+                             : "r"(blk + (uint32_t)rr * 128u + (uint32_t)(((lane >> 2) ^ (rr & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
                 if (lane < ncol) {
                     int32_t *q = out + (row_off + grow) * P.J + col0 + lane;
                     if (reduce) asm volatile("red.global.add.s32 [%0], %1;" ::"l"(q), "r"(val) : "memory");
@@ -469,7 +488,6 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 }
             }
             __syncwarp();
-            ++ocount;
         };
 
         for (int u = cta_first; u < units; u += cta_step, ++tcount) {
@@ -478,29 +496,30 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const int slab_row0 = (u % P.splits) * P.slab_rows;     // 0 unless partial tiles go to per-split slabs
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
-            // the four warps must agree on the outcome: the staging code below uses CTA-level named barriers
+            // the epilogue warps agree on the outcome, so that either all of them or none release the accumulator
             if (!epi_all(mbar_wait(tfull_bar(buf), tph, abort_flag))) {
                 failed = true;
                 break;
             }
             tc_fence_after();
-            const int trow0 = ti * TMU + (int)rank * TM;     // first output row of this CTA's part of the tile
+            const int wrow0 = ti * TMU + (int)rank * TM + quarter * 32;     // first output row of this warp
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
-            for (int c0 = 0; c0 < P.TN; c0 += 32) {
+            const int tile_cols = min(P.TN, P.J - tj * P.TN);
+            const int nchunks = wrow0 < P.I ? (tile_cols + 31) / 32 : 0;   // uniform over the warp
+
+            // one chunk = 32 columns of the warp's 32 rows
+            auto emit = [&](const uint32_t (&v)[32], int ch) {
+                const int c0 = ch * 32;
                 const int col0 = tj * P.TN + c0;
-                if (col0 >= P.J || trow0 >= P.I) break;             // uniform over the CTA
-                uint32_t v[32];
-                tc_ld32(taddr + (uint32_t)c0, v);
-                tc_wait_ld();
                 const int ncol = min(min(32, P.TN - c0), P.J - col0);
                 if (P.splits > 1) {
-                    if (P.tma_acc) stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + trow0);
-                    else stage_and_copy(v, P.acc_out, P.slab_rows == 0, slab_row0, trow0, col0, ncol);
-                    continue;
+                    if (P.tma_acc) stage_and_send(v, &map_acc, P.slab_rows == 0, col0, slab_row0 + wrow0, 0x7fffffff);
+                    else stage_and_copy(v, P.acc_out, P.slab_rows == 0, slab_row0, wrow0, col0, ncol);
+                    return;
                 }
                 if (P.acc_out != nullptr) {
-                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, trow0);
-                    else stage_and_copy(v, P.acc_out, false, 0, trow0, col0, ncol);
+                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, wrow0, P.I);
+                    else stage_and_copy(v, P.acc_out, false, 0, wrow0, col0, ncol);
                 }
                 if (P.f_out != nullptr) {
                     uint32_t f[32];
@@ -511,8 +530,24 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
                     }
-                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, trow0);
-                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, trow0, col0, ncol);
+                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, wrow0, P.I);
+                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, wrow0, col0, ncol);
+                }
+            };
+
+            uint32_t va[32], vb[32];
+            int ch = half;
+            if (ch < nchunks) tc_ld32(taddr + (uint32_t)(ch * 32), va);
+            while (ch < nchunks) {
+                tc_wait_ld_pin(va);
+                if (ch + 2 < nchunks) tc_ld32(taddr + (uint32_t)((ch + 2) * 32), vb);
+                emit(va, ch);
+                ch += 2;
+                if (ch < nchunks) {
+                    tc_wait_ld_pin(vb);
+                    if (ch + 2 < nchunks) tc_ld32(taddr + (uint32_t)((ch + 2) * 32), va);
+                    emit(vb, ch);
+                    ch += 2;
                 }
             }
             tc_fence_before();
@@ -522,7 +557,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 else mbar_arrive(tempty_bar(buf));
             }
         }
-        if (leader) bulk_wait_all();                // staged blocks are out before shared memory goes away
+        if (lane == 0) bulk_wait_all();             // staged blocks are out before shared memory goes away
         if (failed && lane == 0) {
             abort_s = 1;
             atomicExch(P.status, CDL_ERR_TIMEOUT);
@@ -587,14 +622,15 @@ EncodeTiledFn get_encode()
     return fn;
 }
 
-// Output matrix [rows][cols] of 4-byte elements, row pitch cols * 4; box = {32 columns (128 bytes), 128 rows}.
+// Output matrix [rows][cols] of 4-byte elements, row pitch cols * 4; box = {32 columns (128 bytes), 32 rows}: one
+// epilogue warp's staging block.
 bool encode_out_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows, bool is_float)
 {
     EncodeTiledFn fn = get_encode();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 4};
-    const cuuint32_t box[2] = {32u, (cuuint32_t)TM};
+    const cuuint32_t box[2] = {32u, 32u};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(map, is_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_INT32, 2, const_cast<void *>(base),
               dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -757,8 +793,10 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(index_gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(index_gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(index_gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(index_gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(index_gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(index_gemm_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return CDL_ERR_LAUNCH;
         }
@@ -774,7 +812,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         qc.attrs = qa;
         qc.numAttrs = 1;
         int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, index_gemm_tc_kernel<true>, &qc) != cudaSuccess || nclusters < 1) {
+        if (cudaOccupancyMaxActiveClusters(&nclusters, index_gemm_tc_kernel<true, false>, &qc) != cudaSuccess || nclusters < 1) {
             (void)cudaGetLastError();
             nclusters = sms / 2;
         }
@@ -782,6 +820,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         attr_set[dev] = true;
     }
     const long long units = tiles * splits;
+    // bytes a CTA loads per work unit against the bytes it stores (4-byte outputs of a 128 x TN tile)
+    const long long unit_load = (long long)((P.rblocks + splits - 1) / splits) * (kABytes + (pair ? 128 : TN) * BR);
+    const bool store_heavy = unit_load <= 2ll * TM * TN * 4;
     if (pair) {
         const int slots = pair_slots[dev];
         cudaLaunchConfig_t cfg = {};
@@ -796,13 +837,16 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         cfg.stream = stream;
         cfg.attrs = at;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true>, map_a, map_b, map_f, map_acc, P) != cudaSuccess) {
+        const cudaError_t le = store_heavy ? cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true, true>, map_a, map_b, map_f, map_acc, P)
+                                           : cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true, false>, map_a, map_b, map_f, map_acc, P);
+        if (le != cudaSuccess) {
             (void)cudaGetLastError();
             return CDL_ERR_LAUNCH;
         }
     } else {
         const int grid = (int)(units < sms ? units : sms);
-        index_gemm_tc_kernel<false><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        if (store_heavy) index_gemm_tc_kernel<false, true><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        else index_gemm_tc_kernel<false, false><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (f_out != nullptr && (splits > 1 || wide)) {
