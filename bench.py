@@ -44,13 +44,14 @@ NCU_TRAFFIC_BYTES = {
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=3000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="cdl", choices=["cdl", "reference"])
     ap.add_argument("--workload", default="resnet18_layer3_conv",
                     choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny", "resnet18_b256"])
     ap.add_argument("--batch", type=int, default=256, help="batch size of the resnet18_b256 workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step one by one instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
     ap.add_argument("--sweep-max-log2n", type=int, default=28)
@@ -566,8 +567,10 @@ def main():
         exchange()
     torch.cuda.synchronize()
 
-    # ---- timed region: device-resident inputs
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(args.steps)]
+    # ---- timed region: device-resident inputs, the step replayed from a CUDA graph (launch gaps between the ten
+    # short kernels of a step are a tenth of its time when they are launched one by one)
+    graph = step.capture() if not args.no_graph else None
+    torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -575,8 +578,10 @@ def main():
     wall0 = time.time()
     t_start.record(stream)
     for it in range(args.steps):
-        ev = iter(events[it])
-        step.run(mark=lambda name: next(ev).record(stream))
+        if graph is not None:
+            graph.replay()
+        else:
+            step.run()
         exchange()
     t_end.record(stream)
     torch.cuda.synchronize()
@@ -585,7 +590,16 @@ def main():
         dist.barrier()
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
-    per_call_ms = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(args.steps)) / args.steps
+
+    # ---- per-call times: a second pass over the same steps, launched call by call with an event between calls
+    k_steps = min(args.steps, 500)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(k_steps)]
+    for it in range(k_steps):
+        ev = iter(events[it])
+        step.run(mark=lambda name: next(ev).record(stream))
+        exchange()
+    torch.cuda.synchronize()
+    per_call_ms = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(k_steps)) / k_steps
                    for i, name in enumerate(CALLS)}
     status = cdl.cdl_workspace_status(step.ws, check=False)
 
@@ -603,7 +617,10 @@ def main():
     for _ in range(e_steps):
         for k, t in dev_in.items():
             t.copy_(pinned[k].view(t.shape), non_blocking=True)
-        step.run()
+        if graph is not None:
+            graph.replay()
+        else:
+            step.run()
         exchange()
         out_host["scalars"].copy_(step.scalars, non_blocking=True)
         out_host["dw"].copy_(step.dw, non_blocking=True)
@@ -667,6 +684,8 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e_steps},
             "gpu_launches": args.steps * step.kernels_per_step(), "device_status": status,
+            "launch": "stream launches" if graph is None else "CUDA graph replay of one step",
+            "kernel_timing": f"second pass of {k_steps} steps launched call by call, one CUDA event between calls",
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle

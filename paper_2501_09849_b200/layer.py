@@ -78,6 +78,23 @@ class CdlLayerStep:
         split_dw = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, self.M, self.N, self.K) > 256
         return len(CALLS) - (0 if self.need_dx else 1) + (1 if split_dw else 0)
 
+    def capture(self):
+        """Record one step into a CUDA graph and return it (``graph.replay()`` enqueues the step on the current
+        stream).  All buffers of a step are owned by this object and never reallocated, so the recorded pointers
+        stay valid.  One step runs eagerly first: the library's one-time set-up per device must not fall into the
+        capture."""
+        t = self.torch
+        graph = t.cuda.CUDAGraph()
+        side = t.cuda.Stream()
+        side.wait_stream(t.cuda.current_stream())
+        with t.cuda.stream(side):
+            self.run()
+            side.synchronize()
+            with t.cuda.graph(graph, stream=side):
+                self.run()
+        t.cuda.current_stream().wait_stream(side)
+        return graph
+
     def input_tensors(self):
         return {"w": self.w, "x": self.x, "A_idx": self.A_idx, "dY": self.dY, "gx_in": self.gx_in}
 

@@ -241,3 +241,47 @@ def test_resnet18_conv1_and_fc_shapes(torch):
     W = inputs.uniform_indices((K, N), -3, 3, seed=25)
     G = inputs.uniform_indices((M, N), -127, 127, seed=26)
     check_all_products(torch, A, W, G, cdl.IndexDesc(0.25, 0, 15), w, g)
+
+
+def test_step_replayed_from_a_cuda_graph_equals_the_step_launched_call_by_call(torch):
+    # the recorded step must write exactly what the eager step writes (same kernels, same launch shapes); the
+    # products themselves are checked against the oracle above
+    from paper_2501_09849_b200.layer import CdlLayerStep
+    case, wt, at = inputs.tiny_layer(seed=4)
+    M, K, N = case.M, case.K, case.N
+    step = CdlLayerStep(torch, M, K, N, at.size, case.wq, case.aq, q_g=1e-3)
+    step.w.copy_(dev(torch, wt).reshape(-1))
+    step.x.copy_(dev(torch, at).reshape(-1))
+    ai, _ = oracle.hard(at, f32(case.aq.q), case.aq.lo, case.aq.hi)
+    step.A_idx[:, :K].copy_(dev(torch, ai.astype(np.uint8).reshape(M, K)))
+    step.dY.copy_(dev(torch, inputs.normal((M, N), 3e-2, seed=4, stream=7)))
+    step.gx_in.copy_(dev(torch, inputs.normal((at.size,), 1e-2, seed=4, stream=8)))
+    outs = ("w_soft", "W_idx", "x_soft", "X_idx", "hist_w", "hist_x", "prob_w", "prob_x", "Y", "G_idx", "dA", "dW",
+            "dx", "dw")
+
+    def snapshot():
+        torch.cuda.synchronize()
+        return {k: getattr(step, k).clone() for k in outs}
+
+    def clear():
+        step.hist_w.zero_()
+        step.hist_x.zero_()
+        step.scalars.zero_()
+
+    clear()
+    step.run()
+    eager = snapshot()
+    eager_scalars = step.scalars.clone()
+    graph = step.capture()
+    for _ in range(2):
+        for k in outs:
+            getattr(step, k).zero_()
+        clear()
+        graph.replay()
+        got = snapshot()
+        for k in outs:
+            assert torch.equal(got[k], eager[k]), k
+        # entropies are pure functions of the histograms; the four gradient scalars are sums of float64 atomics
+        assert torch.equal(step.scalars[:2], eager_scalars[:2])
+        assert torch.allclose(step.scalars[2:], eager_scalars[2:], rtol=1e-9, atol=1e-12)
+    assert cdl.cdl_workspace_status(step.ws, check=False) == 0
