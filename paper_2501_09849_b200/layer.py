@@ -78,11 +78,12 @@ class CdlLayerStep:
         split_dw = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, self.M, self.N, self.K) > 256
         return len(CALLS) - (0 if self.need_dx else 1) + (1 if split_dw else 0)
 
-    def capture(self):
+    def capture(self, concurrent=True):
         """Record one step into a CUDA graph and return it (``graph.replay()`` enqueues the step on the current
         stream).  All buffers of a step are owned by this object and never reallocated, so the recorded pointers
         stay valid.  One step runs eagerly first: the library's one-time set-up per device must not fall into the
-        capture."""
+        capture.  With concurrent=True the calls are recorded on three streams along the data dependencies of the
+        step (see run_forked), so that the short kernels run beside the long ones."""
         t = self.torch
         graph = t.cuda.CUDAGraph()
         side = t.cuda.Stream()
@@ -91,9 +92,61 @@ class CdlLayerStep:
             self.run()
             side.synchronize()
             with t.cuda.graph(graph, stream=side):
-                self.run()
+                if concurrent:
+                    self.run_forked()
+                else:
+                    self.run()
         t.cuda.current_stream().wait_stream(side)
         return graph
+
+    def run_forked(self):
+        """The same ten calls as run(), issued on the current stream and two helper streams along the step's data
+        dependencies:
+            current:  quantize w -> forward -> dA -> dW -> quantizer backward on w
+            second:   quantize x -> entropy of x -> quantizer backward on x
+            third:    quantize dL/dY ;  entropy of w
+        The forward product needs W_idx; dA needs G_idx and W_idx; dW needs G_idx; the backward pass on w needs dW
+        and the level probabilities of w.  All helper work is joined back into the current stream at the end."""
+        t = self.torch
+        if not hasattr(self, "_helpers"):
+            self._helpers = (t.cuda.Stream(), t.cuda.Stream())
+        s0 = t.cuda.current_stream()
+        s1, s2 = self._helpers
+        sc = self.scalars
+        M, K, N = self.M, self.K, self.N
+        nlw, nlx = self.Pw.nlev, self.Px.nlev
+
+        def after(stream):
+            e = t.cuda.Event()
+            e.record(stream)
+            return e
+        fork = after(s0)
+        s1.wait_event(fork)
+        s2.wait_event(fork)
+        # second stream: everything on the activation tensor
+        cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, s1)
+        cdl.cdl_index_entropy(self.hist_x, nlx, sc[1:2], self.prob_x, None, s1)
+        cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
+        # third stream: gradient indices
+        cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, s2)
+        g_ready = after(s2)
+        # current stream: weights, then the three products
+        cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, s0)
+        w_ready = after(s0)
+        s2.wait_event(w_ready)
+        cdl.cdl_index_entropy(self.hist_w, nlw, sc[0:1], self.prob_w, None, s2)
+        pw_ready = after(s2)
+        cdl.cdl_qlinear_fwd(self.A_idx, self.lda, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
+                            None, self.ws, self.ws_bytes, s0)
+        s0.wait_event(g_ready)
+        if self.need_dx:
+            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
+                                M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, s0)
+        cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
+                            M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, s0)
+        s0.wait_event(pw_ready)
+        cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, sc[2:3], sc[3:4], s0)
+        s0.wait_event(after(s1))
 
     def input_tensors(self):
         return {"w": self.w, "x": self.x, "A_idx": self.A_idx, "dY": self.dY, "gx_in": self.gx_in}
