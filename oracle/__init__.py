@@ -54,6 +54,11 @@ def _load():
         lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
+        lib.cdl_oracle_conv_fwd.argtypes = [P, c.c_int, P, c.c_int64] + [c.c_int] * 9 + [P]
+        lib.cdl_oracle_conv_dx.argtypes = [P, P, c.c_int64] + [c.c_int] * 9 + [P]
+        lib.cdl_oracle_conv_dw.argtypes = [P, c.c_int, P] + [c.c_int] * 9 + [P]
+        for f in (lib.cdl_oracle_conv_fwd, lib.cdl_oracle_conv_dx, lib.cdl_oracle_conv_dw):
+            f.restype = None
         lib.cdl_oracle_mpmf.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, P]
         lib.cdl_oracle_mpmf.restype = None
         lib.cdl_oracle_philox4x32_10.argtypes = [P, P, P]
@@ -194,6 +199,54 @@ def gemm_dw(A, G):
     N = G.shape[1]
     acc = np.empty((K, N), dtype=np.int64)
     _load().cdl_oracle_gemm_dw(_ptr(A), lda, au, _ptr(G), ldg, M, N, K, _ptr(acc))
+    return acc
+
+
+def _conv_dims(X, Wt, R, S):
+    X = np.ascontiguousarray(X)
+    if X.dtype not in (np.int8, np.uint8) or X.ndim != 4:
+        raise TypeError("X is an int8 or uint8 [N,H,W,C] index tensor")
+    Wt, ldw, wu = _idx_bytes(Wt)
+    N, H, W, C = X.shape
+    assert not wu and Wt.shape[0] == R * S * C
+    return X, Wt, ldw, (N, H, W, C), Wt.shape[1]
+
+
+def conv_fwd(X, Wt, R, S, pad_h, pad_w):
+    """Stride-1 cross-correlation with zero padding on indices, int64: X [N,H,W,C] int8|uint8, Wt [(r*S+s)*C+c, CO]
+    int8 -> [N,P,Q,CO]."""
+    X, Wt, ldw, (N, H, W, C), CO = _conv_dims(X, Wt, R, S)
+    P, Q = H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1
+    acc = np.empty((N, P, Q, CO), dtype=np.int64)
+    _load().cdl_oracle_conv_fwd(_ptr(X), int(X.dtype == np.uint8), _ptr(Wt), ldw, N, H, W, C, R, S, pad_h, pad_w, CO,
+                                _ptr(acc))
+    return acc
+
+
+def conv_dx(G, Wt, x_shape, R, S, pad_h, pad_w):
+    """Adjoint of conv_fwd in X: G [N,P,Q,CO] int8, Wt as in conv_fwd -> [N,H,W,C] int64."""
+    N, H, W, C = x_shape
+    G = np.ascontiguousarray(G)
+    Wt, ldw, wu = _idx_bytes(Wt)
+    CO = Wt.shape[1]
+    assert G.dtype == np.int8 and not wu and Wt.shape[0] == R * S * C
+    assert G.shape == (N, H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1, CO)
+    acc = np.empty((N, H, W, C), dtype=np.int64)
+    _load().cdl_oracle_conv_dx(_ptr(G), _ptr(Wt), ldw, N, H, W, C, R, S, pad_h, pad_w, CO, _ptr(acc))
+    return acc
+
+
+def conv_dw(X, G, R, S, pad_h, pad_w):
+    """Adjoint of conv_fwd in Wt: X [N,H,W,C] int8|uint8, G [N,P,Q,CO] int8 -> [(r*S+s)*C+c, CO] int64."""
+    X = np.ascontiguousarray(X)
+    G = np.ascontiguousarray(G)
+    N, H, W, C = X.shape
+    CO = G.shape[3]
+    assert X.dtype in (np.int8, np.uint8) and G.dtype == np.int8
+    assert G.shape == (N, H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1, CO)
+    acc = np.empty((R * S * C, CO), dtype=np.int64)
+    _load().cdl_oracle_conv_dw(_ptr(X), int(X.dtype == np.uint8), _ptr(G), N, H, W, C, R, S, pad_h, pad_w, CO,
+                               _ptr(acc))
     return acc
 
 
