@@ -236,6 +236,43 @@ int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_d
                                const void *A_idx, int64_t lda, const cdl_index_desc *a,
                                int32_t M, int32_t N, int32_t K, float *dW, void *stream);
 
+/*
+ * The same three layer products for a convolutional layer (the layers of the paper's networks, Sec. VI-C and
+ * VI-D, are convolutions; Algorithm 1, forward and backward pass), computed straight from the NHWC index
+ * tensors: the patch matrix whose rows cdl_qlinear_* takes as A_idx is never written to memory, its tiles are
+ * gathered by the loads of the kernel, with zero (= index 0 = level 0) outside the image.
+ * Stride 1, filter R x S with R and S odd, padding (R-1)/2 and (S-1)/2: the output has the spatial size of the
+ * input (3 x 3 and 1 x 1 layers of a ResNet).  C and C_out multiples of 128 (else CDL_ERR_ARG: form the patch
+ * matrix and call cdl_qlinear_*).
+ *   X_idx [dev] N x H x W x C index bytes (signedness from x);  G_idx [dev] N x H x W x C_out int8;
+ *   W_idx [dev] (R*S*C) x C_out int8, row (r*S + s)*C + c, leading dimension ldw (multiple of 16);
+ *   all three 16-byte aligned.
+ *   forward   ACC[n,p,q,co] = sum_{r,s,c} X_idx[n, p-(R-1)/2+r, q-(S-1)/2+s, c] * W_idx[(r*S+s)*C+c, co]
+ *             Y = (float)ACC * (x->q * w->q) + bias[co]            acc_out, y_out: N x H x W x C_out, nullable
+ *   backward  dXACC[n,h,w,c] = sum_{r,s,co} G_idx[n, h+(R-1)/2-r, w+(S-1)/2-s, co] * W_idx[(r*S+s)*C+c, co]
+ *             dX = (float)dXACC * (g->q * w->q)                     dXacc, dX: N x H x W x C, nullable
+ *             dWACC[(r*S+s)*C+c, co] = sum_{n,p,q} X_idx[n, p-(R-1)/2+r, q-(S-1)/2+s, c] * G_idx[n,p,q,co]
+ *             dW = (float)dWACC * (g->q * x->q)                     dWacc, dW: (R*S*C) x C_out (ld C_out), nullable
+ *   X_idx may be NULL when no dW output is wanted, W_idx when no dX output is.
+ *   ws [dev]: cdl_qconv_workspace_bytes(shape, C_out) bytes, 256-byte aligned.
+ * Overflow rule and the int64 summation of long reductions as for cdl_qlinear_*.
+ */
+typedef struct {
+    int32_t N, H, W, C;   /* the layer's input tensor */
+    int32_t R, S;         /* filter height and width */
+} cdl_conv_shape;
+
+int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                  const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out, const float *bias,
+                  void *ws, size_t ws_bytes, void *stream);
+
+int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
+                  const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
+                  int32_t *dXacc, float *dX, int32_t *dWacc, float *dW, void *ws, size_t ws_bytes, void *stream);
+
+/* Bytes of device workspace cdl_qconv_fwd / cdl_qconv_bwd need; 0 for an unsupported shape. */
+size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out);
+
 #define CDL_OP_QLINEAR_FWD 1
 #define CDL_OP_QLINEAR_BWD 2
 

@@ -14,6 +14,7 @@ __all__ = [
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
+    "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
 
@@ -95,11 +96,16 @@ def load_library():
     lib.cdl_qlinear_fwd.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd.argtypes = [P, I64, P, P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd_dw_noalloc.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P]
+    lib.cdl_qconv_fwd.argtypes = [P, P, P, I64, P, P, I32, P, P, P, P, C.c_size_t, P]
+    lib.cdl_qconv_bwd.argtypes = [P, P, P, P, P, I64, P, P, I32, P, P, P, P, P, C.c_size_t, P]
+    lib.cdl_qconv_workspace_bytes.argtypes = [P, I32]
+    lib.cdl_qconv_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_bytes.argtypes = [I32, I32, I32, I32]
     lib.cdl_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_status.argtypes = [P, P]
     for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample", "cdl_index_entropy",
-                 "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status"):
+                 "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status",
+                 "cdl_qconv_fwd", "cdl_qconv_bwd"):
         getattr(lib, name).restype = C.c_int
     _LIB = lib
     return lib
@@ -200,6 +206,45 @@ def cdl_qlinear_bwd(G_idx, ldg, g: IndexDesc, A_idx, lda, a, W_idx, ldw, w, M, N
                                         C.byref(wc) if wc is not None else None, M, N, K, _ptr(dXacc), _ptr(dX),
                                         _ptr(dWacc), _ptr(dW), _ptr(ws), ws_bytes, _stream(stream))
     return _check(rc, "cdl_qlinear_bwd", check)
+
+
+class _ConvShapeC(C.Structure):
+    _fields_ = [("N", C.c_int32), ("H", C.c_int32), ("W", C.c_int32), ("C", C.c_int32), ("R", C.c_int32), ("S", C.c_int32)]
+
+
+class ConvShape:
+    """cdl_conv_shape: input tensor N x H x W x C, filter R x S (stride 1, padding (R-1)/2, (S-1)/2)."""
+
+    def __init__(self, N, H, W, C, R, S):
+        self.N, self.H, self.W, self.C, self.R, self.S = int(N), int(H), int(W), int(C), int(R), int(S)
+
+    def _c(self):
+        return _ConvShapeC(self.N, self.H, self.W, self.C, self.R, self.S)
+
+
+def cdl_qconv_workspace_bytes(shape: ConvShape, C_out):
+    sc = shape._c()
+    return int(load_library().cdl_qconv_workspace_bytes(C.byref(sc), C_out))
+
+
+def cdl_qconv_fwd(X_idx, x: IndexDesc, W_idx, ldw, w: IndexDesc, shape: ConvShape, C_out, acc_out=None, y_out=None,
+                  bias=None, ws=None, ws_bytes=0, stream=None, check=True):
+    xc, wc, sc = x._c(), w._c(), shape._c()
+    rc = load_library().cdl_qconv_fwd(_ptr(X_idx), C.byref(xc), _ptr(W_idx), ldw, C.byref(wc), C.byref(sc), C_out,
+                                      _ptr(acc_out), _ptr(y_out), _ptr(bias), _ptr(ws), ws_bytes, _stream(stream))
+    return _check(rc, "cdl_qconv_fwd", check)
+
+
+def cdl_qconv_bwd(G_idx, g: IndexDesc, X_idx, x, W_idx, ldw, w, shape: ConvShape, C_out, dXacc=None, dX=None,
+                  dWacc=None, dW=None, ws=None, ws_bytes=0, stream=None, check=True):
+    gc, sc = g._c(), shape._c()
+    xc = x._c() if x is not None else None
+    wc = w._c() if w is not None else None
+    rc = load_library().cdl_qconv_bwd(_ptr(G_idx), C.byref(gc), _ptr(X_idx), C.byref(xc) if xc is not None else None,
+                                      _ptr(W_idx), ldw, C.byref(wc) if wc is not None else None, C.byref(sc), C_out,
+                                      _ptr(dXacc), _ptr(dX), _ptr(dWacc), _ptr(dW), _ptr(ws), ws_bytes,
+                                      _stream(stream))
+    return _check(rc, "cdl_qconv_bwd", check)
 
 
 def cdl_qlinear_bwd_dw_noalloc(G_idx, ldg, g: IndexDesc, A_idx, lda, a: IndexDesc, M, N, K, dW, stream=None, check=True):

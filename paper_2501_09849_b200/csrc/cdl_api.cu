@@ -332,4 +332,114 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
     return CDL_OK;
 }
 
+namespace {
+// pixels, taps and patch length of a supported convolution shape; false when the shape is not supported
+bool conv_dims(const cdl_conv_shape *s, int32_t C_out, int64_t *M, int *taps)
+{
+    if (s == nullptr || s->N <= 0 || s->H <= 0 || s->W <= 0 || s->C <= 0 || C_out <= 0) return false;
+    if (s->R <= 0 || s->S <= 0 || (s->R & 1) == 0 || (s->S & 1) == 0 || s->R > 127 || s->S > 127) return false;
+    if ((s->C % 128) != 0 || (C_out % 128) != 0) return false;
+    *M = (int64_t)s->N * s->H * s->W;
+    *taps = s->R * s->S;
+    if (*M > 0x7fffff00ll || (int64_t)*taps * s->C > 0x7fffff00ll || (int64_t)*taps * C_out > 0x7fffff00ll) return false;
+    return true;
+}
+}  // namespace
+
+size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
+{
+    int64_t M;
+    int taps;
+    if (!conv_dims(shape, C_out, &M, &taps)) return 0;
+    const size_t f = tc_gemm_scratch_bytes((int)M, C_out, taps * shape->C);
+    const size_t dx = tc_gemm_scratch_bytes((int)M, shape->C, taps * C_out);
+    const size_t dw = tc_gemm_scratch_bytes(taps * shape->C, C_out, (int)M);
+    size_t m = f > dx ? f : dx;
+    if (dw > m) m = dw;
+    return kStatusBytes + m;
+}
+
+int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                  const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out, const float *bias,
+                  void *ws, size_t ws_bytes, void *stream)
+{
+    int64_t M;
+    int taps;
+    if (X_idx == nullptr || W_idx == nullptr || !conv_dims(shape, C_out, &M, &taps)) return CDL_ERR_ARG;
+    if (acc_out == nullptr && y_out == nullptr) return CDL_ERR_ARG;
+    if (ldw < C_out) return CDL_ERR_ARG;
+    IndexRange rx, rw;
+    int rc;
+    if ((rc = index_range(x, &rx)) != CDL_OK) return rc;
+    if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+    if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+    if ((ldw & 15) || (reinterpret_cast<uintptr_t>(X_idx) & 15u) || (reinterpret_cast<uintptr_t>(W_idx) & 15u)) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(acc_out) || bad_f32_ptr(y_out) || bad_f32_ptr(bias)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_workspace_bytes(shape, C_out))
+        return CDL_ERR_WORKSPACE;
+    const int K = taps * shape->C;
+    if (acc_out != nullptr && overflow_risk(K, rx, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    // Y[pixel, co] = sum_{tap, c} patch(pixel; tap, c) * W[tap * C + c, co]
+    ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 0, 0};
+    GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
+    GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
+    return launch_index_gemm_tc(X, Y, (int)M, C_out, K, acc_out, y_out, (x->q * w->q), bias,
+                                static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws),
+                                static_cast<cudaStream_t>(stream), &cg);
+}
+
+int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
+                  const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
+                  int32_t *dXacc, float *dX, int32_t *dWacc, float *dW, void *ws, size_t ws_bytes, void *stream)
+{
+    const bool want_dx = dXacc != nullptr || dX != nullptr;
+    const bool want_dw = dWacc != nullptr || dW != nullptr;
+    int64_t M;
+    int taps;
+    if (G_idx == nullptr || !conv_dims(shape, C_out, &M, &taps)) return CDL_ERR_ARG;
+    if (!want_dx && !want_dw) return CDL_ERR_ARG;
+    if ((want_dx && W_idx == nullptr) || (want_dw && X_idx == nullptr)) return CDL_ERR_ARG;
+    if (want_dx && ldw < C_out) return CDL_ERR_ARG;
+    IndexRange rg, rx{false, 0}, rw{false, 0};
+    int rc;
+    if ((rc = index_range(g, &rg)) != CDL_OK) return rc;
+    if (rg.is_unsigned && g->hi > 127) return CDL_ERR_RANGE;
+    if (want_dw && (rc = index_range(x, &rx)) != CDL_OK) return rc;
+    if (want_dx) {
+        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+    }
+    if (reinterpret_cast<uintptr_t>(G_idx) & 15u) return CDL_ERR_ALIGN;
+    if (want_dw && (reinterpret_cast<uintptr_t>(X_idx) & 15u)) return CDL_ERR_ALIGN;
+    if (want_dx && ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_workspace_bytes(shape, C_out))
+        return CDL_ERR_WORKSPACE;
+    if (dXacc != nullptr && overflow_risk((int64_t)taps * C_out, rg, rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (dWacc != nullptr && overflow_risk(M, rx, rg)) return CDL_ERR_OVERFLOW_RISK;
+    if ((rc = check_device()) != CDL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (want_dx) {
+        // dX[pixel, c] = sum_{tap', co} patchG(pixel; tap', co) * W[(taps-1-tap') * C + c, co]: the patches of the
+        // gradient tensor (same padding) against the filter taps in mirrored order
+        ConvGather cg{shape->N, shape->H, shape->W, C_out, shape->R, shape->S, 0, shape->C};
+        GemmOperand X{G_idx, 0, 0, false, (int)rg.absmax};
+        GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
+        rc = launch_index_gemm_tc(X, Y, (int)M, shape->C, taps * C_out, dXacc, dX, (g->q * w->q), nullptr,
+                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg);
+        if (rc != CDL_OK) return rc;
+    }
+    if (want_dw) {
+        // dW[tap * C + c, co] = sum_pixel patch(pixel; tap, c) * G[pixel, co]
+        ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 1, 0};
+        GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
+        GemmOperand Y{G_idx, 1, C_out, false, (int)rg.absmax};
+        rc = launch_index_gemm_tc(X, Y, taps * shape->C, C_out, (int)M, dWacc, dW, (g->q * x->q), nullptr,
+                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg);
+        if (rc != CDL_OK) return rc;
+    }
+    return CDL_OK;
+}
+
 }  // extern "C"

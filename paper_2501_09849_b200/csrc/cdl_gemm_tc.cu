@@ -65,6 +65,14 @@ struct TcParams {
     const float *bias;
     int *status;
     int tma_f, tma_acc;     // the float / int32 output goes through shared memory and TMA
+    // Implicit patch matrix (convolution): the X operand is gathered by TMA im2col loads from an [N,H,W,C] index
+    // tensor instead of being read from a stored matrix.
+    int conv;               // 0: stored matrix; 1: X(i = pixel, r = tap * C + c); 2: X(i = tap * C + c, r = pixel)
+    int cH, cW, cC, cS;     // image height and width, channels, filter width
+    int cblocks;            // 128-channel blocks per tap (C / 128)
+    int pad_h, pad_w;
+    int taps;               // R * S
+    int y_tap_rows;         // > 0: the Y block of tap t starts at row (taps - 1 - t) * y_tap_rows of the stored matrix
     int slab_rows;          // 0: splits add into one I x J buffer.  > 0: split s stores its partial tile into rows
                             // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
 };
@@ -120,6 +128,27 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+
+// im2col load: 128 consecutive pixels (w fastest, then h, then n) x 128 channel bytes starting at pixel (w, h, n)
+// shifted by the filter tap (off_w, off_h); positions outside the tensor read as zero
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, int c, int w, int h, int n,
+                                                int off_w, int off_h, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+        ::"r"(dst), "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"((unsigned short)off_w), "h"((unsigned short)off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_pair(uint32_t dst, const CUtensorMap *map, int c, int w, int h, int n,
+                                                     int off_w, int off_h, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .b32 rb;\n\t"
+        "mapa.shared::cluster.u32 rb, %6, 0;\n\t"
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3, %4, %5}], [rb], {%7, %8};\n\t}"
+        ::"r"(dst), "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"((unsigned short)off_w), "h"((unsigned short)off_h)
         : "memory");
 }
 
@@ -356,23 +385,42 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
                     const uint32_t sb = sa + kABytes;
                     const int arow = ti * TMU + (int)rank * TM;
+                    // patch gather: which pixel block, channel block and filter tap this stage holds
+                    int g_c = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, b_row = tj * P.TN + brow;
+                    if (P.conv != 0) {
+                        // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
+                        const int i0 = arow < P.I ? arow : 0;
+                        const int tap = P.conv == 1 ? rb / P.cblocks : i0 / P.cC;
+                        const int pix = P.conv == 1 ? i0 : rb * BR;
+                        g_c = P.conv == 1 ? (rb % P.cblocks) * BR : i0 % P.cC;
+                        g_n = pix / (P.cH * P.cW);
+                        const int rem = pix - g_n * (P.cH * P.cW);
+                        g_h = rem / P.cW - P.pad_h;
+                        g_w = rem % P.cW - P.pad_w;
+                        g_oh = tap / P.cS;
+                        g_ow = tap % P.cS;
+                        if (P.y_tap_rows > 0) b_row += (P.taps - 1 - tap) * P.y_tap_rows;
+                    }
+                    const int b_red = P.y_tap_rows > 0 ? (rb % P.cblocks) * BR : rb * BR;   // Y coordinate along r
                     if (PAIR) {
                         // both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_tx);
-                        if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
+                        if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, g_w, g_h, g_n, g_ow, g_oh, full_bar(s));
+                        else if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
                         else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
-                        if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, tj * P.TN + brow, rb * BR, full_bar(s));
-                        else tma_load_2d_pair(sb, &map_b, rb * BR, tj * P.TN + brow, full_bar(s));
+                        if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, b_row, b_red, full_bar(s));
+                        else tma_load_2d_pair(sb, &map_b, b_red, b_row, full_bar(s));
                         continue;
                     }
                     mbar_expect_tx(full_bar(s), stage_tx);
-                    if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
+                    if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, g_w, g_h, g_n, g_ow, g_oh, full_bar(s));
+                    else if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
                     else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
                     if (P.b_mn_major) {
                         for (int bb = 0; bb < b_blocks; ++bb)
-                            tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, tj * P.TN + bb * 128, rb * BR, full_bar(s));
+                            tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, b_row + bb * 128, b_red, full_bar(s));
                     } else {
-                        tma_load_2d(sb, &map_b, rb * BR, tj * P.TN, full_bar(s));
+                        tma_load_2d(sb, &map_b, b_red, b_row, full_bar(s));
                     }
                 }
             }
@@ -651,6 +699,37 @@ bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t out
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+// [N,H,W,C] byte tensor read in im2col mode: one load fetches 128 consecutive base pixels x 128 channel bytes,
+// the base pixels running over the input shifted by the padding, the filter tap given per load as an offset.
+bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g)
+{
+    static EncodeIm2colFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return false;
+        }
+        fn = reinterpret_cast<EncodeIm2colFn>(p);
+    }
+    const int pad_h = (g.R - 1) / 2, pad_w = (g.S - 1) / 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)g.C, (cuuint64_t)g.C * g.W, (cuuint64_t)g.C * g.W * g.H};
+    const int lower[2] = {-pad_w, -pad_h};                          // {w, h}: first base pixel
+    const int upper[2] = {pad_w - (g.S - 1), pad_h - (g.R - 1)};    // last base pixel relative to the far corner
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, 128u, 128u,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 namespace {
@@ -716,9 +795,9 @@ size_t tc_gemm_scratch_bytes(int I, int J, int R)
 // bytes, used only when the reduced dimension is split and no int32 output was requested.
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream)
+                         cudaStream_t stream, const ConvGather *conv)
 {
-    const bool a_mn = X.stride_outer == 1 && X.stride_red != 1;
+    const bool a_mn = conv != nullptr ? conv->transposed != 0 : (X.stride_outer == 1 && X.stride_red != 1);
     const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
     TcParams P;
     P.I = I;
@@ -746,6 +825,21 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.b_mn_major = b_mn ? 1 : 0;
     P.idesc = (2u << 4) | ((X.is_unsigned ? 0u : 1u) << 7) | ((Y.is_unsigned ? 0u : 1u) << 10) |
               ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(pl.tile_rows >> 4) << 24);
+    P.conv = 0;
+    P.cH = P.cW = P.cC = P.cS = P.cblocks = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
+    if (conv != nullptr) {
+        if (conv->C % BR != 0 || (conv->R & 1) == 0 || (conv->S & 1) == 0) return CDL_ERR_ARG;
+        P.conv = conv->transposed ? 2 : 1;
+        P.cH = conv->H;
+        P.cW = conv->W;
+        P.cC = conv->C;
+        P.cS = conv->S;
+        P.cblocks = conv->C / BR;
+        P.pad_h = (conv->R - 1) / 2;
+        P.pad_w = (conv->S - 1) / 2;
+        P.taps = conv->R * conv->S;
+        P.y_tap_rows = conv->y_tap_rows;
+    }
     P.scale = scale;
     P.bias = bias;
     P.status = status;
@@ -767,9 +861,13 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     CUtensorMap map_a, map_b;
     bool ok;
     // K-major operand: stored [outer][r], r contiguous -> inner = r.  MN-major: stored [r][outer] -> inner = outer.
-    if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
+    if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv);
+    else if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
     else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
+    else if (conv != nullptr && conv->y_tap_rows > 0)   // all taps' row blocks of the stored matrix, conv->C reduced columns each
+        ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->R * conv->S * conv->y_tap_rows,
+                              (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
     else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
     // outputs through shared memory + TMA when their pitch and base allow it and the tile is at least one box wide
     CUtensorMap map_f = map_a, map_acc = map_a;      // placeholders when unused

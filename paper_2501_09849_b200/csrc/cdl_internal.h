@@ -53,10 +53,21 @@ struct GemmOperand {
     int absmax;             // bound on |entry| (from the operand's declared index range)
 };
 
+// The X operand as an implicit patch matrix of a convolution (stride 1, zero padding, output the size of the
+// input): X.ptr then is an [N,H,W,C] tensor of index bytes, C a multiple of 128, and the rows / columns of the
+// patch matrix are gathered by TMA im2col loads, never stored.
+struct ConvGather {
+    int N, H, W, C;         // the gathered tensor
+    int R, S;               // filter height and width (odd); padding is (R-1)/2, (S-1)/2
+    int transposed;         // 0: X(i = pixel, r = tap * C + c);  1: X(i = tap * C + c, r = pixel)
+    int y_tap_rows;         // > 0: Y is stored as [taps * y_tap_rows][C] (r contiguous) and the block of tap t is the
+                            //      one of the mirrored tap, rows (taps - 1 - t) * y_tap_rows ..  (backward-data product)
+};
+
 // Tensor-core index GEMM (TMA + tcgen05 + TMEM); operands need 16-byte aligned bases and pitches.
 size_t tc_gemm_scratch_bytes(int I, int J, int R);
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream);
+                         cudaStream_t stream, const ConvGather *conv = nullptr);
 
 }  // namespace cdl

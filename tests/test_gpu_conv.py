@@ -1,0 +1,112 @@
+"""GPU parity of the convolution products computed from the NHWC index tensors (patch matrix never stored)
+against the CPU oracle's direct convolution: int32 accumulators bit-exact, float outputs equal to the accumulator
+times the binary32 product of the steps."""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2501_09849_b200 as cdl
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    cdl.load_library()
+    return torch
+
+
+def dev(torch, a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def scaled(acc, qa, qb, bias=None):
+    y = acc.astype(f32) * f32(f32(qa) * f32(qb))
+    if bias is not None:
+        y = (y + bias.astype(f32)).astype(f32)
+    return y
+
+
+def make(seed, N, H, W, C, CO, R, S, unsigned=True):
+    rng = np.random.default_rng(seed)
+    # activations: 4-bit indices with many zeros (post-ReLU); weights 15 levels; gradients 8-bit
+    X = (rng.integers(0, 16, (N, H, W, C)) * (rng.random((N, H, W, C)) < 0.6)).astype(np.uint8) if unsigned \
+        else rng.integers(-8, 8, (N, H, W, C)).astype(np.int8)
+    Wt = rng.integers(-7, 8, (R * S * C, CO)).astype(np.int8)
+    G = rng.integers(-127, 128, (N, H, W, CO)).astype(np.int8)
+    return X, Wt, G
+
+
+def run_all(torch, X, Wt, G, R, S, unsigned=True, bias=None):
+    N, H, W, C = X.shape
+    CO = Wt.shape[1]
+    shape = cdl.ConvShape(N, H, W, C, R, S)
+    x = cdl.IndexDesc(0.25, 0, 15) if unsigned else cdl.IndexDesc(0.25, -8, 7)
+    w, g = cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    nb = cdl.cdl_qconv_workspace_bytes(shape, CO)
+    assert nb >= 256
+    ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    Xd, Wd, Gd = dev(torch, X), dev(torch, Wt), dev(torch, G)
+    acc = torch.empty((N, H, W, CO), dtype=torch.int32, device="cuda")
+    y = torch.empty((N, H, W, CO), dtype=torch.float32, device="cuda")
+    bd = dev(torch, bias) if bias is not None else None
+    cdl.cdl_qconv_fwd(Xd, x, Wd, CO, w, shape, CO, acc, y, bd, ws, nb)
+    dxa = torch.empty((N, H, W, C), dtype=torch.int32, device="cuda")
+    dx = torch.empty((N, H, W, C), dtype=torch.float32, device="cuda")
+    dwa = torch.empty((R * S * C, CO), dtype=torch.int32, device="cuda")
+    dw = torch.empty((R * S * C, CO), dtype=torch.float32, device="cuda")
+    cdl.cdl_qconv_bwd(Gd, g, Xd, x, Wd, CO, w, shape, CO, dxa, dx, dwa, dw, ws, nb)
+    torch.cuda.synchronize()
+    assert cdl.cdl_workspace_status(ws, check=False) == 0
+    ph, pw = (R - 1) // 2, (S - 1) // 2
+    ref = oracle.conv_fwd(X, Wt, R, S, ph, pw)
+    assert np.array_equal(acc.cpu().numpy(), ref.astype(np.int32))
+    assert np.array_equal(y.cpu().numpy(), scaled(ref, x.q, w.q, bias))
+    ref_dx = oracle.conv_dx(G, Wt, X.shape, R, S, ph, pw)
+    assert np.array_equal(dxa.cpu().numpy(), ref_dx.astype(np.int32))
+    assert np.array_equal(dx.cpu().numpy(), scaled(ref_dx, g.q, w.q))
+    ref_dw = oracle.conv_dw(X, G, R, S, ph, pw)
+    assert np.array_equal(dwa.cpu().numpy(), ref_dw.astype(np.int32))
+    assert np.array_equal(dw.cpu().numpy(), scaled(ref_dw, g.q, x.q))
+
+
+def test_one_tile_3x3(torch):
+    # 128 pixels = one tile; every pixel row of the patch matrix crosses an image border somewhere
+    X, Wt, G = make(1, 2, 8, 8, 128, 128, 3, 3)
+    run_all(torch, X, Wt, G, 3, 3)
+
+
+def test_cta_pair_tiles_3x3_exact_and_ragged(torch):
+    X, Wt, G = make(2, 4, 8, 8, 128, 256, 3, 3)              # 256 pixels: one pair tile
+    run_all(torch, X, Wt, G, 3, 3)
+    X, Wt, G = make(3, 3, 10, 9, 256, 256, 3, 3)             # 270 pixels: ragged second tile, blocks straddle images
+    run_all(torch, X, Wt, G, 3, 3, bias=np.linspace(-1, 1, 256).astype(f32))
+
+
+def test_signed_activations_one_by_one_and_wide_filters(torch):
+    X, Wt, G = make(4, 2, 7, 5, 128, 256, 1, 1, unsigned=False)
+    run_all(torch, X, Wt, G, 1, 1, unsigned=False)
+    X, Wt, G = make(5, 1, 9, 11, 128, 128, 5, 3)
+    run_all(torch, X, Wt, G, 5, 3)
+    X, Wt, G = make(6, 2, 6, 20, 128, 128, 3, 7)             # padding 3 along w: whole rows of zeros at the border
+    run_all(torch, X, Wt, G, 3, 7)
+
+
+def test_resnet_layer_geometry_14x14(torch):
+    # the 14 x 14 images of the ResNet-18 layer this library is benchmarked on (fewer images): 128-pixel blocks
+    # never line up with image rows, every block mixes several rows and images
+    X, Wt, G = make(7, 6, 14, 14, 256, 256, 3, 3)
+    run_all(torch, X, Wt, G, 3, 3)
+
+
+def test_unsupported_shapes_are_refused(torch):
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    t = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    y = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
+    x, w = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7)
+    for shape, co in ((cdl.ConvShape(1, 4, 4, 64, 3, 3), 128), (cdl.ConvShape(1, 4, 4, 128, 2, 2), 128),
+                      (cdl.ConvShape(1, 4, 4, 128, 3, 3), 64)):
+        assert cdl.cdl_qconv_workspace_bytes(shape, co) == 0
+        assert cdl.cdl_qconv_fwd(t, x, t, co, w, shape, co, None, y, None, ws, 1 << 20, check=False) == -1
