@@ -51,6 +51,7 @@ def parse_args():
                     choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny", "resnet18_b256"])
     ap.add_argument("--batch", type=int, default=256, help="batch size of the resnet18_b256 workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-implicit", action="store_true", help="skip the extra measurement of the layer in convolution form")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step one by one instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
@@ -107,6 +108,70 @@ def call_model(case, n_x):
         "quantize_backward_x": {"bytes": n_x * 12, "elems": n_x},
         "quantize_backward_w": {"bytes": n_w * 12, "elems": n_w},
     }
+
+
+def conv_call_model(case, n_x):
+    """call_model for the convolution form: the products read the NHWC index tensor (n_x bytes) instead of the
+    M x K patch matrix and dX is written in the layout of x."""
+    M, K, N = case.M, case.K, case.N
+    m = call_model(case, n_x)
+    m["qlinear_fwd"]["bytes"] = n_x + K * N + 4 * M * N
+    m["qlinear_bwd_dx"]["bytes"] = M * N + K * N + 4 * n_x
+    m["qlinear_bwd_dw"]["bytes"] = n_x + M * N + 4 * K * N
+    return m
+
+
+def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, peaks_hbm, int8_tops):
+    """The same layer as a convolution computed straight from the NHWC index tensor (cdl_qconv_*): same w, x and
+    dL/dY, the data gradient feeds the activation quantizer's backward pass directly.  Returns a dict of times."""
+    n_img, H, W, C = case.a_shape
+    taps = case.K // C
+    R = S = int(round(taps ** 0.5))
+    assert R * S * C == case.K and n_img * H * W == case.M
+    shape = cdl.ConvShape(n_img, H, W, C, R, S)
+    cs = CdlLayerStep(torch, case.M, case.K, case.N, step.n_x, case.wq, case.aq, q_g, conv=shape)
+    cs.w.copy_(step.w)
+    cs.x.copy_(step.x)
+    cs.dY.copy_(step.dY)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        cs.run()
+    graph = cs.capture()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    k_steps = min(steps, 200)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(k_steps)]
+    for it in range(k_steps):
+        ev = iter(events[it])
+        cs.run(mark=lambda name: next(ev).record(stream))
+    torch.cuda.synchronize()
+    per = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(k_steps)) / k_steps
+           for i, name in enumerate(CALLS)}
+    model = conv_call_model(case, step.n_x)
+    kern = {}
+    for name in CALLS:
+        m, t = model[name], per[name]
+        k = {"ms": round(t, 5), "GBps": round(m["bytes"] / (t * 1e-3) / 1e9, 1)}
+        if "ops" in m:
+            k["int8_TOPS"] = round(m["ops"] / (t * 1e-3) / 1e12, 1)
+            t_tensor, t_hbm = m["ops"] / (int8_tops * 1e12), m["bytes"] / (peaks_hbm * 1e9)
+            k["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
+            k["roofline_frac"] = round(max(t_tensor, t_hbm) / (t * 1e-3), 4)
+        kern[name] = k
+    quant_elems = sum(m["elems"] for m in model.values())
+    status = cdl.cdl_workspace_status(cs.ws, check=False)
+    return {"ms_per_step": ms, "value": quant_elems / (ms * 1e-3) / 1e9, "unit": UNIT, "steps": steps,
+            "h2d_bytes_per_step_if_e2e": sum(t.numel() * t.element_size() for t in cs.input_tensors().values()),
+            "gpu_launches": steps * cs.kernels_per_step(), "device_status": status, "kernels": kern,
+            "note": "same layer through cdl_qconv_fwd/bwd: no stored patch matrix, dX in the layout of x"}
 
 
 class ClockSampler:
@@ -687,6 +752,8 @@ def main():
             "launch": "stream launches" if graph is None else "CUDA graph replay of one step",
             "kernel_timing": f"second pass of {k_steps} steps launched call by call, one CUDA event between calls",
         }
+        if world == 1 and args.workload == "resnet18_layer3_conv" and not args.no_implicit:
+            line["implicit_conv"] = run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, args.steps, hbm, int8_tops)
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()

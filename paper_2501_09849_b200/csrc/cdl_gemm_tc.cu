@@ -375,6 +375,25 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
                 const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
                 const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
+                const int arow = ti * TMU + (int)rank * TM;
+                // Patch gather: pixel block, channel block and filter tap of the first stage of this unit, kept up
+                // to date with additions only inside the loop (this one thread feeds the whole pipeline).
+                int g_cb = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, g_tap = 0, g_c0 = 0;
+                if (P.conv != 0) {
+                    // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
+                    const int i0 = arow < P.I ? arow : 0;
+                    g_tap = P.conv == 1 ? rb0 / P.cblocks : i0 / P.cC;
+                    g_cb = P.conv == 1 ? rb0 % P.cblocks : 0;
+                    g_c0 = P.conv == 1 ? 0 : i0 % P.cC;
+                    const int pix = P.conv == 1 ? i0 : rb0 * BR;
+                    g_n = pix / (P.cH * P.cW);
+                    const int rem = pix - g_n * (P.cH * P.cW);
+                    g_h = rem / P.cW;
+                    g_w = rem % P.cW;
+                    g_oh = g_tap / P.cS;
+                    g_ow = g_tap % P.cS;
+                }
+                const int pix_dh = BR / (P.cW > 0 ? P.cW : 1), pix_dw = BR % (P.cW > 0 ? P.cW : 1);   // 128 pixels further on
                 for (int rb = rb0; rb < rb1; ++rb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
@@ -384,28 +403,36 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     }
                     const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
                     const uint32_t sb = sa + kABytes;
-                    const int arow = ti * TMU + (int)rank * TM;
-                    // patch gather: which pixel block, channel block and filter tap this stage holds
-                    int g_c = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, b_row = tj * P.TN + brow;
-                    if (P.conv != 0) {
-                        // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
-                        const int i0 = arow < P.I ? arow : 0;
-                        const int tap = P.conv == 1 ? rb / P.cblocks : i0 / P.cC;
-                        const int pix = P.conv == 1 ? i0 : rb * BR;
-                        g_c = P.conv == 1 ? (rb % P.cblocks) * BR : i0 % P.cC;
-                        g_n = pix / (P.cH * P.cW);
-                        const int rem = pix - g_n * (P.cH * P.cW);
-                        g_h = rem / P.cW - P.pad_h;
-                        g_w = rem % P.cW - P.pad_w;
-                        g_oh = tap / P.cS;
-                        g_ow = tap % P.cS;
-                        if (P.y_tap_rows > 0) b_row += (P.taps - 1 - tap) * P.y_tap_rows;
+                    int b_row = tj * P.TN + brow;
+                    if (P.y_tap_rows > 0) b_row += (P.taps - 1 - g_tap) * P.y_tap_rows;
+                    const int b_red = P.y_tap_rows > 0 ? g_cb * BR : rb * BR;   // Y coordinate along r
+                    const int g_c = P.conv == 1 ? g_cb * BR : g_c0;
+                    const int c_w = g_w - P.pad_w, c_h = g_h - P.pad_h, c_n = g_n, c_ow = g_ow, c_oh = g_oh;
+                    if (P.conv == 1) {            // next stage: next channel block, then next tap
+                        if (++g_cb == P.cblocks) {
+                            g_cb = 0;
+                            ++g_tap;
+                            if (++g_ow == P.cS) {
+                                g_ow = 0;
+                                ++g_oh;
+                            }
+                        }
+                    } else if (P.conv == 2) {     // next stage: 128 pixels further on
+                        g_w += pix_dw;
+                        g_h += pix_dh;
+                        if (g_w >= P.cW) {
+                            g_w -= P.cW;
+                            ++g_h;
+                        }
+                        while (g_h >= P.cH) {
+                            g_h -= P.cH;
+                            ++g_n;
+                        }
                     }
-                    const int b_red = P.y_tap_rows > 0 ? (rb % P.cblocks) * BR : rb * BR;   // Y coordinate along r
                     if (PAIR) {
                         // both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_tx);
-                        if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, g_w, g_h, g_n, g_ow, g_oh, full_bar(s));
+                        if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
                         else if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
                         else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
                         if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, b_row, b_red, full_bar(s));
@@ -413,7 +440,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         continue;
                     }
                     mbar_expect_tx(full_bar(s), stage_tx);
-                    if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, g_w, g_h, g_n, g_ow, g_oh, full_bar(s));
+                    if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
                     else if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
                     else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
                     if (P.b_mn_major) {

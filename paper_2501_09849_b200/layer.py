@@ -14,6 +14,10 @@ Step (names follow the paper: w weights, x activations, q / s step sizes, alpha 
    9  quantizer backward on w with grad_out = dW: dL/dw, dL/dq, dL/dalpha (+ lambda * rate term)
 The im2col gather / scatter between the activation tensor and the GEMM operand is outside the library:
 A_idx and the gradient arriving at the quantized activations are inputs of the step.
+
+With conv=ConvShape(...) the layer is a stride-1 convolution computed straight from the NHWC index tensor
+(cdl_qconv_fwd / cdl_qconv_bwd): steps 5 and 7 read X_idx itself, dA becomes dL/dQ(x) in the layout of x, and step 8
+takes it as its incoming gradient, so the only inputs of a step are w, x and dL/dY.
 """
 from __future__ import annotations
 
@@ -24,10 +28,14 @@ CALLS = ("quantize_soft_w", "entropy_w", "quantize_soft_x", "entropy_x", "qlinea
 
 
 class CdlLayerStep:
-    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None, need_dx=True):
+    def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None, need_dx=True, conv=None):
         """wq / xq: objects with q, lo, hi, alpha, rate_weight, window (weights / activations); n_x: number of
-        activation elements quantized per step (the layer's input tensor, before im2col)."""
+        activation elements quantized per step (the layer's input tensor, before im2col); conv: a ConvShape for
+        the convolution form (then M = N*H*W pixels, K = R*S*C, n_x = M*C)."""
         self.torch = torch
+        self.conv = conv
+        if conv is not None:
+            assert M == conv.N * conv.H * conv.W and K == conv.R * conv.S * conv.C and n_x == M * conv.C
         self.M, self.K, self.N, self.n_x, self.n_w = M, K, N, n_x, K * N
         self.need_dx = need_dx      # False for the first layer of a network: its input needs no gradient
         self.lda = lda if lda is not None else (K + 15) // 16 * 16     # row pitch of A_idx (multiple of 16 bytes)
@@ -40,9 +48,10 @@ class CdlLayerStep:
         # inputs of a step
         self.w = t.empty(self.n_w, dtype=f32, device=dev)
         self.x = t.empty(n_x, dtype=f32, device=dev)
-        self.A_idx = t.zeros((M, self.lda), dtype=idt(xq.lo), device=dev)
+        self.A_idx = t.zeros((M, self.lda), dtype=idt(xq.lo), device=dev) if conv is None else None
         self.dY = t.empty((M, N), dtype=f32, device=dev)
-        self.gx_in = t.empty(n_x, dtype=f32, device=dev)         # dL/dQ(x) after the scatter back from dA
+        # dL/dQ(x): an input after the scatter back from dA, or the convolution's own data gradient
+        self.gx_in = t.empty(n_x, dtype=f32, device=dev)
         # outputs
         self.w_soft = t.empty(self.n_w, dtype=f32, device=dev)
         self.W_idx = t.empty((K, N), dtype=idt(wq.lo), device=dev)
@@ -54,14 +63,18 @@ class CdlLayerStep:
         self.prob_x = t.empty(xq.hi - xq.lo + 1, dtype=f32, device=dev)
         self.Y = t.empty((M, N), dtype=f32, device=dev)
         self.G_idx = t.empty((M, N), dtype=i8, device=dev)
-        self.dA = t.empty((M, K), dtype=f32, device=dev) if need_dx else None
+        self.dA = (t.empty((M, K), dtype=f32, device=dev) if need_dx else None) if conv is None else self.gx_in
         self.dW = t.empty((K, N), dtype=f32, device=dev)
         self.dx = t.empty(n_x, dtype=f32, device=dev)
         self.dw = t.empty(self.n_w, dtype=f32, device=dev)
         # scalars: H(w), H(x) | dq, dalpha, ds, dbeta
         self.scalars = t.zeros(6, dtype=t.float64, device=dev)
-        self.ws_bytes = max(cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_FWD, M, N, K),
-                            cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K))
+        if conv is None:
+            self.ws_bytes = max(cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_FWD, M, N, K),
+                                cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K))
+        else:
+            self.ws_bytes = cdl.cdl_qconv_workspace_bytes(conv, N)
+            assert self.ws_bytes > 0, "convolution shape not supported by cdl_qconv_*"
         self.ws = t.empty(self.ws_bytes, dtype=u8, device=dev)
         self.Pw = cdl.QuantParams(wq.q, wq.lo, wq.hi, wq.alpha, wq.rate_weight, None, wq.window)
         self.Px = cdl.QuantParams(xq.q, xq.lo, xq.hi, xq.alpha, xq.rate_weight, None, xq.window)
@@ -75,7 +88,7 @@ class CdlLayerStep:
     def kernels_per_step(self):
         """Kernels of this library one step launches: one per call, plus the small kernel that turns the split
         weight-gradient reduction into floats when the reduction over M is split across SMs."""
-        split_dw = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, self.M, self.N, self.K) > 256
+        split_dw = self.ws_bytes > 256
         return len(CALLS) - (0 if self.need_dx else 1) + (1 if split_dw else 0)
 
     def capture(self, concurrent=True):
@@ -123,10 +136,13 @@ class CdlLayerStep:
         fork = after(s0)
         s1.wait_event(fork)
         s2.wait_event(fork)
-        # second stream: everything on the activation tensor
+        # second stream: everything on the activation tensor (in the convolution form its backward pass waits
+        # for the data gradient, see below)
         cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, s1)
+        x_ready = after(s1)
         cdl.cdl_index_entropy(self.hist_x, nlx, sc[1:2], self.prob_x, None, s1)
-        cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
+        if self.conv is None:
+            cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
         # third stream: gradient indices
         cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, s2)
         g_ready = after(s2)
@@ -136,20 +152,53 @@ class CdlLayerStep:
         s2.wait_event(w_ready)
         cdl.cdl_index_entropy(self.hist_w, nlw, sc[0:1], self.prob_w, None, s2)
         pw_ready = after(s2)
-        cdl.cdl_qlinear_fwd(self.A_idx, self.lda, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
-                            None, self.ws, self.ws_bytes, s0)
+        if self.conv is not None:
+            s0.wait_event(x_ready)
+        self._fwd(s0)
         s0.wait_event(g_ready)
-        if self.need_dx:
-            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
-                                M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, s0)
-        cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
-                            M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, s0)
+        self._bwd_dx(s0)
+        if self.conv is not None:
+            s1.wait_event(after(s0))
+            cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
+        self._bwd_dw(s0)
         s0.wait_event(pw_ready)
         cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, sc[2:3], sc[3:4], s0)
         s0.wait_event(after(s1))
 
     def input_tensors(self):
+        if self.conv is not None:
+            return {"w": self.w, "x": self.x, "dY": self.dY}
         return {"w": self.w, "x": self.x, "A_idx": self.A_idx, "dY": self.dY, "gx_in": self.gx_in}
+
+    # the three products, in either form
+    def _fwd(self, stream):
+        M, K, N = self.M, self.K, self.N
+        if self.conv is None:
+            cdl.cdl_qlinear_fwd(self.A_idx, self.lda, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
+                                None, self.ws, self.ws_bytes, stream)
+        else:
+            cdl.cdl_qconv_fwd(self.X_idx, self.da, self.W_idx, N, self.dw_desc, self.conv, N, None, self.Y, None,
+                              self.ws, self.ws_bytes, stream)
+
+    def _bwd_dx(self, stream):
+        M, K, N = self.M, self.K, self.N
+        if not self.need_dx:
+            return
+        if self.conv is None:
+            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
+                                M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
+        else:
+            cdl.cdl_qconv_bwd(self.G_idx, self.dg, None, None, self.W_idx, N, self.dw_desc, self.conv, N,
+                              None, self.dA, None, None, self.ws, self.ws_bytes, stream)
+
+    def _bwd_dw(self, stream):
+        M, K, N = self.M, self.K, self.N
+        if self.conv is None:
+            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
+                                M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
+        else:
+            cdl.cdl_qconv_bwd(self.G_idx, self.dg, self.X_idx, self.da, None, N, None, self.conv, N,
+                              None, None, None, self.dW, self.ws, self.ws_bytes, stream)
 
     def run(self, stream=None, mark=None):
         """Enqueue one step.  mark(name), if given, is called before each ABI call and once at the end
@@ -162,16 +211,11 @@ class CdlLayerStep:
         m(CALLS[1]); cdl.cdl_index_entropy(self.hist_w, nlw, s[0:1], self.prob_w, None, stream)
         m(CALLS[2]); cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, stream)
         m(CALLS[3]); cdl.cdl_index_entropy(self.hist_x, nlx, s[1:2], self.prob_x, None, stream)
-        m(CALLS[4]); cdl.cdl_qlinear_fwd(self.A_idx, self.lda, self.da, self.W_idx, N, self.dw_desc, M, N, K, None, self.Y,
-                                         None, self.ws, self.ws_bytes, stream)
+        m(CALLS[4]); self._fwd(stream)
         m(CALLS[5]); cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, stream)
         # the two backward products are issued as two calls so that each can be timed on its own
-        m(CALLS[6])
-        if self.need_dx:
-            cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, None, K, None, self.W_idx, N, self.dw_desc,
-                                M, N, K, None, self.dA, None, None, self.ws, self.ws_bytes, stream)
-        m(CALLS[7]); cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
-                                         M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
+        m(CALLS[6]); self._bwd_dx(stream)
+        m(CALLS[7]); self._bwd_dw(stream)
         m(CALLS[8]); cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, s[4:5], s[5:6], stream)
         m(CALLS[9]); cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, s[2:3], s[3:4], stream)
         m("end")

@@ -110,3 +110,35 @@ def test_unsupported_shapes_are_refused(torch):
                       (cdl.ConvShape(1, 4, 4, 128, 3, 3), 64)):
         assert cdl.cdl_qconv_workspace_bytes(shape, co) == 0
         assert cdl.cdl_qconv_fwd(t, x, t, co, w, shape, co, None, y, None, ws, 1 << 20, check=False) == -1
+
+
+def test_resnet18_layer3_full_size_sampled(torch):
+    # the benchmarked geometry, 256 images of 14 x 14 x 256 -> 256 channels, in the launch configuration bench.py
+    # times; the oracle computes whole images (forward, dX) and whole rows of dW chosen across taps and channels
+    N, H, W, C, CO, R, S = 256, 14, 14, 256, 256, 3, 3
+    X, Wt, G = make(8, N, H, W, C, CO, R, S)
+    shape = cdl.ConvShape(N, H, W, C, R, S)
+    x, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    nb = cdl.cdl_qconv_workspace_bytes(shape, CO)
+    ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    Xd, Wd, Gd = dev(torch, X), dev(torch, Wt), dev(torch, G)
+    y = torch.empty((N, H, W, CO), dtype=torch.float32, device="cuda")
+    dx = torch.empty((N, H, W, C), dtype=torch.float32, device="cuda")
+    dw = torch.empty((R * S * C, CO), dtype=torch.float32, device="cuda")
+    cdl.cdl_qconv_fwd(Xd, x, Wd, CO, w, shape, CO, None, y, None, ws, nb)
+    cdl.cdl_qconv_bwd(Gd, g, Xd, x, Wd, CO, w, shape, CO, None, dx, None, dw, ws, nb)
+    torch.cuda.synchronize()
+    assert cdl.cdl_workspace_status(ws, check=False) == 0
+    yh, dxh, dwh = y.cpu().numpy(), dx.cpu().numpy(), dw.cpu().numpy()
+    for n in (0, 131, 255):
+        assert np.array_equal(yh[n:n + 1], scaled(oracle.conv_fwd(X[n:n + 1], Wt, R, S, 1, 1), x.q, w.q))
+        assert np.array_equal(dxh[n:n + 1], scaled(oracle.conv_dx(G[n:n + 1], Wt, (1, H, W, C), R, S, 1, 1), g.q, w.q))
+    # rows k = (r*S + s)*C + c of dW: column k of the patch matrix is X shifted by the tap, zero outside
+    ks = [0, 255, 256 + 17, 4 * 256 + 100, 5 * 256 + 255, 8 * 256, 8 * 256 + 255, 2 * 256 + 128]
+    Xp = np.zeros((N, H + 2, W + 2, C), dtype=X.dtype)
+    Xp[:, 1:H + 1, 1:W + 1, :] = X
+    cols = np.stack([Xp[:, (k // C) // S:(k // C) // S + H, (k // C) % S:(k // C) % S + W, k % C].reshape(-1) for k in ks], axis=1)
+    ref = oracle.gemm_dw(np.ascontiguousarray(cols), G.reshape(-1, CO))
+    assert np.array_equal(dwh[ks], scaled(ref, g.q, x.q))
+    # every entry of the three outputs was written (nothing left of the poison below would survive a re-run)
+    assert np.isfinite(yh).all() and np.isfinite(dxh).all() and np.isfinite(dwh).all()
