@@ -354,6 +354,86 @@ __device__ __forceinline__ ElemOut quant_elem(const QuantDev &P, const float *__
     return o;
 }
 
+// ---- two elements at a time on the NEAR3 path, with the packed binary32 instructions of sm_100 (one issue slot
+// per pair of multiplies, adds or fused multiply-adds).  The passes are issue-bound before they are HBM-bound, and
+// three quarters of an element's arithmetic is of that kind.  Every packed operation rounds exactly like the scalar
+// one it replaces, and the sequence is the scalar path's, so both give the same bits.
+struct PairOut {
+    int k0[2];
+    float2 y, gx, tq, ta;
+};
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }   // a - b, one rounding
+
+template <int MODE, bool RATE>
+__device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const float *__restrict__ Ltab, float2 x, float2 g)
+{
+    constexpr bool kRate = RATE && MODE == MODE_BWD;
+    PairOut o;
+    const float q = P.q;
+    // hard index (see quant_elem): reciprocal product, clamp, magic-number rounding, exact quotient near ties
+    float2 c = __fmul2_rn(x, f2(P.rq));
+    if (!P.fast_div) c = make_float2(__fdiv_rn(x.x, q), __fdiv_rn(x.y, q));
+    c.x = fminf(fmaxf(c.x, P.flo), P.fhi);
+    c.y = fminf(fmaxf(c.y, P.flo), P.fhi);
+    float2 t = __fadd2_rn(c, f2(kMagic));
+    float2 kn = __fadd2_rn(t, f2(-kMagic));
+    if (P.fast_div) {
+        const float2 df = sub2(c, kn);
+        if (fabsf(df.x) > kTieGuard || fabsf(df.y) > kTieGuard) {
+            c.x = fminf(fmaxf(__fdiv_rn(x.x, q), P.flo), P.fhi);
+            c.y = fminf(fmaxf(__fdiv_rn(x.y, q), P.flo), P.fhi);
+            t = __fadd2_rn(c, f2(kMagic));
+            kn = __fadd2_rn(t, f2(-kMagic));
+        }
+    }
+    const int k0 = __float_as_int(t.x) - kMagicBits, k1 = __float_as_int(t.y) - kMagicBits;
+    o.k0[0] = k0;
+    o.k0[1] = k1;
+    // d = x - kn q as dh + dl
+    const float2 nph = __fmul2_rn(kn, f2(-q));            // -(kn q) rounded
+    const float2 pl = __ffma2_rn(kn, f2(q), nph);         // kn q - RN(kn q), exact
+    const float2 sx = __fadd2_rn(x, nph);
+    const float2 dh = sub2(sx, pl);
+    const float2 dl = sub2(sub2(sx, dh), pl);
+    // logits of the two neighbours relative to the nearest level: -alpha q (q -+ 2 d)
+    const float2 w1 = __ffma2_rn(dl, f2(-2.0f), __ffma2_rn(dh, f2(-2.0f), f2(q)));
+    const float2 wm = __ffma2_rn(dl, f2(2.0f), __ffma2_rn(dh, f2(2.0f), f2(q)));
+    const float2 a1 = __fmul2_rn(w1, f2(-P.c1)), am = __fmul2_rn(wm, f2(-P.c1));
+    float2 e1 = make_float2(ex2_approx(a1.x), ex2_approx(a1.y));
+    float2 em = make_float2(ex2_approx(am.x), ex2_approx(am.y));
+    e1.x = (kn.x < P.fhi) ? e1.x : 0.0f;
+    e1.y = (kn.y < P.fhi) ? e1.y : 0.0f;
+    em.x = (kn.x > P.flo) ? em.x : 0.0f;
+    em.y = (kn.y > P.flo) ? em.y : 0.0f;
+    const float2 S = __fadd2_rn(__fadd2_rn(f2(1.0f), e1), em);
+    const float2 rS = make_float2(rcp_approx(S.x), rcp_approx(S.y));
+    const float2 m1 = __fmul2_rn(sub2(e1, em), rS);
+    o.y = __ffma2_rn(kn, f2(q), __fmul2_rn(f2(q), m1));
+    o.gx = o.tq = o.ta = f2(0.0f);
+    if (MODE == MODE_BWD) {
+        const float2 m2 = __fmul2_rn(__fadd2_rn(e1, em), rS);          // E J^2; E J^3 = E J
+        const float2 varj = __ffma2_rn(__fmul2_rn(m1, f2(-1.0f)), m1, m2);
+        const float2 covj = sub2(m1, __fmul2_rn(m1, m2));
+        float2 gx = __fmul2_rn(g, __fmul2_rn(f2(P.a2), varj));
+        if (kRate) {
+            const float Lc0 = Ltab[k0 - P.lo], Lc1 = Ltab[k1 - P.lo];
+            const float2 l1 = __fmul2_rn(make_float2(Ltab[min(k0 + 1, P.hi) - P.lo] - Lc0, Ltab[min(k1 + 1, P.hi) - P.lo] - Lc1), e1);
+            const float2 lm = __fmul2_rn(make_float2(Ltab[max(k0 - 1, P.lo) - P.lo] - Lc0, Ltab[max(k1 - 1, P.lo) - P.lo] - Lc1), em);
+            const float2 rate = __fmul2_rn(sub2(sub2(l1, lm), __fmul2_rn(m1, __fadd2_rn(l1, lm))), rS);
+            gx = __ffma2_rn(f2(P.rate_c), rate, gx);
+        }
+        o.gx = gx;
+        const float2 qc = __fmul2_rn(f2(q), covj);
+        const float2 dmk = __ffma2_rn(kn, f2(-q), dh);                 // d - kn q
+        const float2 dq = __ffma2_rn(f2(P.two_aq), sub2(__fmul2_rn(dmk, varj), qc), __fadd2_rn(kn, m1));
+        const float2 da = __fmul2_rn(f2(P.q2), sub2(__fmul2_rn(__fmul2_rn(f2(2.0f), dh), varj), qc));
+        o.tq = __fmul2_rn(g, dq);
+        o.ta = __fmul2_rn(g, da);
+    }
+    return o;
+}
+
 __device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane)
 {
     atomicAdd(&hist_s[bin * 32 + lane], 1u);
@@ -440,8 +520,27 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 }
                 float ys[4], gxs[4];
                 unsigned int packed = 0u;
+                constexpr bool kPairs = PATH == PATH_NEAR3 && (MODE == MODE_BWD || (MODE == MODE_SOFT && !RATE));
+                if (kPairs) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                    for (int h = 0; h < 2; ++h) {
+                        const PairOut o = quant_pair_near3<MODE, RATE>(P, Ltab, make_float2(xs[2 * h], xs[2 * h + 1]),
+                                                                       make_float2(gs[2 * h], gs[2 * h + 1]));
+                        ys[2 * h] = o.y.x;
+                        ys[2 * h + 1] = o.y.y;
+                        gxs[2 * h] = o.gx.x;
+                        gxs[2 * h + 1] = o.gx.y;
+                        part_q += o.tq.x + o.tq.y;
+                        part_a += o.ta.x + o.ta.y;
+                        packed |= (((unsigned int)o.k0[0] & 0xffu) | (((unsigned int)o.k0[1] & 0xffu) << 8)) << (16 * h);
+                        if (MODE != MODE_BWD && do_hist) {
+                            hist_add(hist_s, o.k0[0] - P.lo, lane);
+                            hist_add(hist_s, o.k0[1] - P.lo, lane);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < (kPairs ? 0 : 4); ++c) {
                     const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
                     ys[c] = o.y;
                     gxs[c] = o.gx;
