@@ -38,7 +38,7 @@ namespace {
 #define CDL_Q_THREADS 256
 #endif
 #ifndef CDL_Q_BATCH
-#define CDL_Q_BATCH 4
+#define CDL_Q_BATCH 2
 #endif
 #ifndef CDL_Q_MINBLOCKS
 #define CDL_Q_MINBLOCKS 1
