@@ -250,6 +250,31 @@ def conv_dw(X, G, R, S, pad_h, pad_w):
     return acc
 
 
+def huffman_lengths(hist):
+    """Code lengths of a Huffman code for the symbols with a non-zero count (Sec. VI-B: the average number of bits per
+    weight / activation is measured with Huffman coding), by the textbook construction: repeatedly merge the two
+    lightest subtrees.  Unused symbols get length 0; a single used symbol gets one bit.  Returns (lengths, total bits
+    sum_k hist[k] * length[k]); the lengths depend on how ties are broken, the total does not."""
+    import heapq
+    h = [int(v) for v in np.asarray(hist).reshape(-1)]
+    lengths = [0] * len(h)
+    used = [k for k, c in enumerate(h) if c > 0]
+    if len(used) == 1:
+        lengths[used[0]] = 1
+    elif len(used) > 1:
+        heap = [(h[k], k, (k,)) for k in used]          # (weight, tie-break, symbols below this subtree)
+        heapq.heapify(heap)
+        nxt = len(h)
+        while len(heap) > 1:
+            w0, _, s0 = heapq.heappop(heap)
+            w1, _, s1 = heapq.heappop(heap)
+            for k in s0 + s1:
+                lengths[k] += 1
+            heapq.heappush(heap, (w0 + w1, nxt, s0 + s1))
+            nxt += 1
+    return np.array(lengths, dtype=np.int64), sum(c * l for c, l in zip(h, lengths))
+
+
 def philox4x32_10(ctr, key):
     """One block of Philox4x32-10: ctr 4 x uint32, key 2 x uint32 -> 4 x uint32."""
     c = np.ascontiguousarray(ctr, dtype=np.uint32)
