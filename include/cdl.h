@@ -163,6 +163,20 @@ int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits,
                       float *level_prob, uint64_t *n_out, void *stream);
 
 /*
+ * Huffman code lengths for the levels of a tensor, from its histogram (Sec. VI-B: the average numbers of bits per
+ * weight and per activation that the paper reports are those of a Huffman code of the quantized tensor).
+ *   hist       [dev] nlev uint64 counters (a count histogram of cdl_quantize_hard / _soft / _sample).
+ *   lengths    [dev] nlev bytes, nullable: code length of each level; 0 for a level that does not occur; when only one
+ *              level occurs its length is 1 (a reading: the paper does not treat the one-symbol case).
+ *   total_bits [dev] one uint64, nullable: sum_k hist[k] * lengths[k], the size of the coded tensor without the table.
+ *   avg_bits   [dev] one double, nullable: total_bits / n, 0 when the histogram is empty.
+ * The individual lengths depend on how equal weights are paired (any optimal prefix code is a valid answer); the
+ * total does not.  At least one output is required.
+ */
+int cdl_huffman_lengths(const uint64_t *hist, int32_t nlev, uint8_t *lengths, uint64_t *total_bits, double *avg_bits,
+                        void *stream);
+
+/*
  * Forward layer product over the indices (Sec. V-A; Algorithm 1, forward pass) with the
  * q_a * q_w rescale in the epilogue:
  *   ACC[m,n] = sum_k A_idx[m,k] * W_idx[k,n]   (int32, exact)

@@ -14,7 +14,7 @@ __all__ = [
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
-    "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
+    "cdl_huffman_lengths", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
 
@@ -96,6 +96,8 @@ def load_library():
     lib.cdl_qlinear_fwd.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd.argtypes = [P, I64, P, P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd_dw_noalloc.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P]
+    lib.cdl_huffman_lengths.argtypes = [P, I32, P, P, P, P]
+    lib.cdl_huffman_lengths.restype = C.c_int
     lib.cdl_qconv_fwd.argtypes = [P, P, P, I64, P, P, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qconv_bwd.argtypes = [P, P, P, P, P, I64, P, P, I32, P, P, P, P, P, C.c_size_t, P]
     lib.cdl_qconv_workspace_bytes.argtypes = [P, I32]
@@ -186,6 +188,12 @@ def cdl_workspace_bytes(op, M, N, K) -> int:
 def cdl_workspace_status(ws, stream=None, check=True):
     rc = load_library().cdl_workspace_status(_ptr(ws), _stream(stream))
     return _check(rc, "cdl_workspace_status", check)
+
+
+def cdl_huffman_lengths(hist, nlev, lengths=None, total_bits=None, avg_bits=None, stream=None, check=True):
+    rc = load_library().cdl_huffman_lengths(_ptr(hist), nlev, _ptr(lengths), _ptr(total_bits), _ptr(avg_bits),
+                                            _stream(stream))
+    return _check(rc, "cdl_huffman_lengths", check)
 
 
 def cdl_qlinear_fwd(A_idx, lda, a: IndexDesc, W_idx, ldw, w: IndexDesc, M, N, K, acc_out=None, y_out=None, bias=None,

@@ -228,6 +228,20 @@ int cdl_index_entropy(const uint64_t *hist, int32_t nlev, double *H_bits, float 
                           reinterpret_cast<unsigned long long *>(n_out), static_cast<cudaStream_t>(stream));
 }
 
+int cdl_huffman_lengths(const uint64_t *hist, int32_t nlev, uint8_t *lengths, uint64_t *total_bits, double *avg_bits,
+                        void *stream)
+{
+    if (hist == nullptr || (lengths == nullptr && total_bits == nullptr && avg_bits == nullptr)) return CDL_ERR_ARG;
+    if (nlev < 1 || nlev > CDL_MAX_LEVELS) return CDL_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(hist) & 7u) || (reinterpret_cast<uintptr_t>(total_bits) & 7u) ||
+        (reinterpret_cast<uintptr_t>(avg_bits) & 7u))
+        return CDL_ERR_ALIGN;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    return launch_huffman(reinterpret_cast<const unsigned long long *>(hist), nlev, lengths,
+                          reinterpret_cast<unsigned long long *>(total_bits), avg_bits, static_cast<cudaStream_t>(stream));
+}
+
 size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
 {
     if (M <= 0 || N <= 0 || K <= 0) return 0;

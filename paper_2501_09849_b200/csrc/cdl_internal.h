@@ -53,6 +53,9 @@ struct GemmOperand {
     int absmax;             // bound on |entry| (from the operand's declared index range)
 };
 
+int launch_huffman(const unsigned long long *hist, int nlev, unsigned char *lengths, unsigned long long *total_bits,
+                   double *avg_bits, cudaStream_t stream);
+
 // The X operand as an implicit patch matrix of a convolution (stride 1, zero padding, output the size of the
 // input): X.ptr then is an [N,H,W,C] tensor of index bytes, C a multiple of 128, and the rows / columns of the
 // patch matrix are gathered by TMA im2col loads, never stored.
