@@ -198,6 +198,25 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a,
                     void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Forward products that also emit the hard index of the NEXT layer's activation quantizer (Sec. IV-A Remark /
+ * end of Sec. IV-B: Q_u; Algorithm 1 feeds each layer's output to the next layer's quantizer), taken in the
+ * epilogue from the finished float output, so that a forward-only (inference) pass never writes or re-reads the
+ * fp32 activations:
+ *   idx_next[m,n] = clamp(rint(Y[m,n] / next->q), next->lo, next->hi)        -- the bytes cdl_quantize_hard(Y) writes
+ *   next     index set and step of the next layer's quantizer (with lo = 0 the clamp doubles as the ReLU).
+ *   idx_next [dev] M x N (resp. N x H x W x C_out) index bytes, row pitch N (C_out); nullable = plain forward.
+ *   acc_out, y_out may then both be NULL.  Everything else as cdl_qlinear_fwd / cdl_qconv_fwd.
+ * The reduced dimension is not split across CTAs for these calls; CDL_ERR_OVERFLOW_RISK when it is so long that
+ * its int32 sum could overflow for the declared index ranges.
+ */
+int cdl_qlinear_fwd_next(const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                         const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                         int32_t M, int32_t N, int32_t K,
+                         int32_t *acc_out, float *y_out, const float *bias,
+                         const cdl_index_desc *next, void *idx_next,
+                         void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Backward layer products over the indices (Algorithm 1, backward pass over the quantized weights
  * and activations).  The gradient operand is an index tensor as well: the caller quantizes
  * dL/dY with cdl_quantize_hard (for example lo=-127, hi=127 and a step g->q of its choice) - a
@@ -279,6 +298,11 @@ typedef struct {
 int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,
                   const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out, const float *bias,
                   void *ws, size_t ws_bytes, void *stream);
+
+int cdl_qconv_fwd_next(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw,
+                       const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
+                       int32_t *acc_out, float *y_out, const float *bias,
+                       const cdl_index_desc *next, void *idx_next, void *ws, size_t ws_bytes, void *stream);
 
 int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
                   const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,

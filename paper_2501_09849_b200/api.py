@@ -14,7 +14,7 @@ __all__ = [
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
-    "cdl_huffman_lengths", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
+    "cdl_huffman_lengths", "cdl_qlinear_fwd_next", "cdl_qconv_fwd_next", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
 
@@ -96,6 +96,10 @@ def load_library():
     lib.cdl_qlinear_fwd.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd.argtypes = [P, I64, P, P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, C.c_size_t, P]
     lib.cdl_qlinear_bwd_dw_noalloc.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P]
+    lib.cdl_qlinear_fwd_next.argtypes = [P, I64, P, P, I64, P, I32, I32, I32, P, P, P, P, P, P, C.c_size_t, P]
+    lib.cdl_qconv_fwd_next.argtypes = [P, P, P, I64, P, P, I32, P, P, P, P, P, P, C.c_size_t, P]
+    lib.cdl_qlinear_fwd_next.restype = C.c_int
+    lib.cdl_qconv_fwd_next.restype = C.c_int
     lib.cdl_huffman_lengths.argtypes = [P, I32, P, P, P, P]
     lib.cdl_huffman_lengths.restype = C.c_int
     lib.cdl_qconv_fwd.argtypes = [P, P, P, I64, P, P, I32, P, P, P, P, C.c_size_t, P]
@@ -188,6 +192,24 @@ def cdl_workspace_bytes(op, M, N, K) -> int:
 def cdl_workspace_status(ws, stream=None, check=True):
     rc = load_library().cdl_workspace_status(_ptr(ws), _stream(stream))
     return _check(rc, "cdl_workspace_status", check)
+
+
+def cdl_qlinear_fwd_next(A_idx, lda, a: IndexDesc, W_idx, ldw, w: IndexDesc, M, N, K, next: IndexDesc, idx_next,
+                         acc_out=None, y_out=None, bias=None, ws=None, ws_bytes=0, stream=None, check=True):
+    ac, wc, nc = a._c(), w._c(), next._c()
+    rc = load_library().cdl_qlinear_fwd_next(_ptr(A_idx), lda, C.byref(ac), _ptr(W_idx), ldw, C.byref(wc), M, N, K,
+                                             _ptr(acc_out), _ptr(y_out), _ptr(bias), C.byref(nc), _ptr(idx_next),
+                                             _ptr(ws), ws_bytes, _stream(stream))
+    return _check(rc, "cdl_qlinear_fwd_next", check)
+
+
+def cdl_qconv_fwd_next(X_idx, x: IndexDesc, W_idx, ldw, w: IndexDesc, shape, C_out, next: IndexDesc, idx_next,
+                       acc_out=None, y_out=None, bias=None, ws=None, ws_bytes=0, stream=None, check=True):
+    xc, wc, sc, nc = x._c(), w._c(), shape._c(), next._c()
+    rc = load_library().cdl_qconv_fwd_next(_ptr(X_idx), C.byref(xc), _ptr(W_idx), ldw, C.byref(wc), C.byref(sc), C_out,
+                                           _ptr(acc_out), _ptr(y_out), _ptr(bias), C.byref(nc), _ptr(idx_next),
+                                           _ptr(ws), ws_bytes, _stream(stream))
+    return _check(rc, "cdl_qconv_fwd_next", check)
 
 
 def cdl_huffman_lengths(hist, nlev, lengths=None, total_bits=None, avg_bits=None, stream=None, check=True):

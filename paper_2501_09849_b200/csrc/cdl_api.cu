@@ -270,12 +270,38 @@ int cdl_workspace_status(void *ws, void *stream)
     return CDL_ERR_TIMEOUT;
 }
 
-int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, const void *W_idx, int64_t ldw,
-                    const cdl_index_desc *w, int32_t M, int32_t N, int32_t K, int32_t *acc_out, float *y_out,
-                    const float *bias, void *ws, size_t ws_bytes, void *stream)
+namespace {
+// next layer's quantizer for the fused index output; CDL_OK with out->idx_out == nullptr when none is requested
+int next_quant(const cdl_index_desc *next, void *idx_next, cdl::NextQuant *out)
+{
+    out->idx_out = nullptr;
+    if (idx_next == nullptr) return CDL_OK;
+    if (next == nullptr) return CDL_ERR_ARG;
+    cdl::IndexRange r;
+    int rc = cdl::index_range(next, &r);
+    if (rc != CDL_OK) return rc;
+    out->idx_out = idx_next;
+    out->q = next->q;
+    out->rq = (float)(1.0 / (double)next->q);
+    out->flo = (float)next->lo;
+    out->fhi = (float)next->hi;
+    out->fast_div = (next->q > 1e-30f && next->q < 1e30f) ? 1 : 0;
+    return CDL_OK;
+}
+}  // namespace
+
+int cdl_qlinear_fwd_next(const void *A_idx, int64_t lda, const cdl_index_desc *a, const void *W_idx, int64_t ldw,
+                         const cdl_index_desc *w, int32_t M, int32_t N, int32_t K, int32_t *acc_out, float *y_out,
+                         const float *bias, const cdl_index_desc *next, void *idx_next, void *ws, size_t ws_bytes,
+                         void *stream)
 {
     if (A_idx == nullptr || W_idx == nullptr || M <= 0 || N <= 0 || K <= 0) return CDL_ERR_ARG;
-    if (acc_out == nullptr && y_out == nullptr) return CDL_ERR_ARG;
+    if (acc_out == nullptr && y_out == nullptr && idx_next == nullptr) return CDL_ERR_ARG;
+    NextQuant nq;
+    {
+        const int rcn = next_quant(next, idx_next, &nq);
+        if (rcn != CDL_OK) return rcn;
+    }
     if (lda < K || ldw < N) return CDL_ERR_ARG;
     IndexRange ra, rw;
     int rc;
@@ -294,7 +320,15 @@ int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, con
     GemmOperand X{A_idx, lda, 1, ra.is_unsigned, (int)ra.absmax};
     GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
     return launch_index_gemm_tc(X, Y, M, N, K, acc_out, y_out, scale, bias, static_cast<char *>(ws) + kStatusBytes,
-                                static_cast<int *>(ws), st);
+                                static_cast<int *>(ws), st, nullptr, &nq);
+}
+
+int cdl_qlinear_fwd(const void *A_idx, int64_t lda, const cdl_index_desc *a, const void *W_idx, int64_t ldw,
+                    const cdl_index_desc *w, int32_t M, int32_t N, int32_t K, int32_t *acc_out, float *y_out,
+                    const float *bias, void *ws, size_t ws_bytes, void *stream)
+{
+    return cdl_qlinear_fwd_next(A_idx, lda, a, W_idx, ldw, w, M, N, K, acc_out, y_out, bias, nullptr, nullptr, ws,
+                                ws_bytes, stream);
 }
 
 int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, const void *A_idx, int64_t lda,
@@ -373,14 +407,20 @@ size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
     return kStatusBytes + m;
 }
 
-int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,
-                  const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out, const float *bias,
-                  void *ws, size_t ws_bytes, void *stream)
+int cdl_qconv_fwd_next(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw,
+                       const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out,
+                       const float *bias, const cdl_index_desc *next, void *idx_next, void *ws, size_t ws_bytes,
+                       void *stream)
 {
     int64_t M;
     int taps;
     if (X_idx == nullptr || W_idx == nullptr || !conv_dims(shape, C_out, &M, &taps)) return CDL_ERR_ARG;
-    if (acc_out == nullptr && y_out == nullptr) return CDL_ERR_ARG;
+    if (acc_out == nullptr && y_out == nullptr && idx_next == nullptr) return CDL_ERR_ARG;
+    NextQuant nq;
+    {
+        const int rcn = next_quant(next, idx_next, &nq);
+        if (rcn != CDL_OK) return rcn;
+    }
     if (ldw < C_out) return CDL_ERR_ARG;
     IndexRange rx, rw;
     int rc;
@@ -400,7 +440,15 @@ int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx,
     GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
     return launch_index_gemm_tc(X, Y, (int)M, C_out, K, acc_out, y_out, (x->q * w->q), bias,
                                 static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws),
-                                static_cast<cudaStream_t>(stream), &cg);
+                                static_cast<cudaStream_t>(stream), &cg, &nq);
+}
+
+int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                  const cdl_conv_shape *shape, int32_t C_out, int32_t *acc_out, float *y_out, const float *bias,
+                  void *ws, size_t ws_bytes, void *stream)
+{
+    return cdl_qconv_fwd_next(X_idx, x, W_idx, ldw, w, shape, C_out, acc_out, y_out, bias, nullptr, nullptr, ws, ws_bytes,
+                              stream);
 }
 
 int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,

@@ -73,6 +73,10 @@ struct TcParams {
     int pad_h, pad_w;
     int taps;               // R * S
     int y_tap_rows;         // > 0: the Y block of tap t starts at row (taps - 1 - t) * y_tap_rows of the stored matrix
+    // next layer's hard index from the float output (forward products, single split)
+    unsigned char *nq_out;  // nullptr: not requested
+    float nq_q, nq_rq, nq_flo, nq_fhi;
+    int nq_fast, nq_vec;    // reciprocal product allowed; rows can be written 16 bytes at a time
     int slab_rows;          // 0: splits add into one I x J buffer.  > 0: split s stores its partial tile into rows
                             // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
 };
@@ -289,6 +293,21 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)1 << 46;   // descriptor version for sm_100
     d |= (uint64_t)2 << 61;   // SWIZZLE_128B
     return d;
+}
+
+// clamp(rint(y / q), lo, hi) exactly as the quantizer kernels compute it: reciprocal product, rounding by adding
+// 1.5 * 2^23, and the IEEE quotient itself whenever the product lies within 2^-12 of a half-integer (the product
+// is within 3 ulp of the quotient and indices are at most 255).  A NaN clamps to lo.
+__device__ __forceinline__ int next_hard_index(float y, float q, float rq, float flo, float fhi, int fast)
+{
+    const float magic = 12582912.0f;
+    float c = fminf(fmaxf(fast ? __fmul_rn(y, rq) : __fdiv_rn(y, q), flo), fhi);
+    float t = __fadd_rn(c, magic);
+    if (fast && fabsf(__fsub_rn(c, __fsub_rn(t, magic))) > 0.5f - 0.000244140625f) {
+        c = fminf(fmaxf(__fdiv_rn(y, q), flo), fhi);
+        t = __fadd_rn(c, magic);
+    }
+    return __float_as_int(t) - 0x4B400000;
 }
 
 // PAIR = false: one CTA per 128 x TN tile.  PAIR = true (TN = 256): a cluster of two CTAs per 256 x 256 tile with
@@ -596,7 +615,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, wrow0, P.I);
                     else stage_and_copy(v, P.acc_out, false, 0, wrow0, col0, ncol);
                 }
-                if (P.f_out != nullptr) {
+                if (P.f_out != nullptr || P.nq_out != nullptr) {
                     uint32_t f[32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c) f[c] = __float_as_uint(__fmul_rn((float)(int)v[c], P.scale));
@@ -605,8 +624,34 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
                     }
-                    if (P.tma_f) stage_and_send(f, &map_f, false, col0, wrow0, P.I);
-                    else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, wrow0, col0, ncol);
+                    if (P.nq_out != nullptr && wrow0 + lane < P.I) {
+                        // the next layer's index of this thread's 32 outputs: 32 consecutive bytes of its row
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int c4 = 0; c4 < 8; ++c4) {
+                            uint32_t word = 0u;
+#pragma unroll
+                            for (int b = 0; b < 4; ++b) {
+                                const int k = next_hard_index(__uint_as_float(f[4 * c4 + b]), P.nq_q, P.nq_rq, P.nq_flo,
+                                                              P.nq_fhi, P.nq_fast);
+                                word |= ((uint32_t)k & 0xffu) << (8 * b);
+                            }
+                            pk[c4] = word;
+                        }
+                        unsigned char *dst = P.nq_out + (long long)(wrow0 + lane) * P.J + col0;
+                        if (P.nq_vec) {         // J is a multiple of 16: each half of the chunk is wholly inside or outside
+                            if (ncol > 0) *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            if (ncol > 16) *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c < ncol) dst[c] = (unsigned char)(pk[c >> 2] >> (8 * (c & 3)));
+                        }
+                    }
+                    if (P.f_out != nullptr) {
+                        if (P.tma_f) stage_and_send(f, &map_f, false, col0, wrow0, P.I);
+                        else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, wrow0, col0, ncol);
+                    }
                 }
             };
 
@@ -822,7 +867,7 @@ size_t tc_gemm_scratch_bytes(int I, int J, int R)
 // bytes, used only when the reduced dimension is split and no int32 output was requested.
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream, const ConvGather *conv)
+                         cudaStream_t stream, const ConvGather *conv, const NextQuant *next)
 {
     const bool a_mn = conv != nullptr ? conv->transposed != 0 : (X.stride_outer == 1 && X.stride_red != 1);
     const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
@@ -836,7 +881,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const bool wide = (long long)R * X.absmax * Y.absmax >= ((long long)1 << 31);
     if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
     const Plan pl = plan(I, J, R, wide ? min_exact_splits(R, X.absmax, Y.absmax) : 1);
-    const int TN = pl.TN, splits = pl.splits;
+    const bool want_next = next != nullptr && next->idx_out != nullptr;
+    if (want_next && wide) return CDL_ERR_OVERFLOW_RISK;     // the index is taken from one finished accumulator
+    const int TN = pl.TN, splits = want_next ? 1 : pl.splits;
     const bool pair = pl.pair != 0;
     P.TN = TN;
     P.tiles_i = (I + pl.tile_rows - 1) / pl.tile_rows;
@@ -852,6 +899,18 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.b_mn_major = b_mn ? 1 : 0;
     P.idesc = (2u << 4) | ((X.is_unsigned ? 0u : 1u) << 7) | ((Y.is_unsigned ? 0u : 1u) << 10) |
               ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(pl.tile_rows >> 4) << 24);
+    P.nq_out = nullptr;
+    P.nq_q = P.nq_rq = P.nq_flo = P.nq_fhi = 0.0f;
+    P.nq_fast = P.nq_vec = 0;
+    if (next != nullptr && next->idx_out != nullptr) {
+        P.nq_out = static_cast<unsigned char *>(next->idx_out);
+        P.nq_q = next->q;
+        P.nq_rq = next->rq;
+        P.nq_flo = next->flo;
+        P.nq_fhi = next->fhi;
+        P.nq_fast = next->fast_div;
+        P.nq_vec = ((J & 15) == 0 && (reinterpret_cast<uintptr_t>(next->idx_out) & 15u) == 0) ? 1 : 0;
+    }
     P.conv = 0;
     P.cH = P.cW = P.cC = P.cS = P.cblocks = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
     if (conv != nullptr) {

@@ -67,10 +67,19 @@ struct ConvGather {
                             //      one of the mirrored tap, rows (taps - 1 - t) * y_tap_rows ..  (backward-data product)
 };
 
+// Hard index of the next layer's quantizer, computed in the forward product's epilogue from the float output:
+// idx = clamp(rint(y / q), lo, hi) with the arithmetic of the quantizer kernels (bit-identical to quantizing Y).
+struct NextQuant {
+    void *idx_out;      // I x J index bytes, row pitch J
+    float q, rq;        // step and RN(1/q)
+    float flo, fhi;     // index range as floats
+    int fast_div;       // as QuantDev::fast_div
+};
+
 // Tensor-core index GEMM (TMA + tcgen05 + TMEM); operands need 16-byte aligned bases and pitches.
 size_t tc_gemm_scratch_bytes(int I, int J, int R);
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream, const ConvGather *conv = nullptr);
+                         cudaStream_t stream, const ConvGather *conv = nullptr, const NextQuant *next = nullptr);
 
 }  // namespace cdl
