@@ -43,6 +43,9 @@ namespace {
 #ifndef CDL_Q_MINBLOCKS
 #define CDL_Q_MINBLOCKS 1
 #endif
+#ifndef CDL_Q_PREFETCH
+#define CDL_Q_PREFETCH 0     // 1: the loads of the next iteration are issued before the arithmetic of this one
+#endif
 #ifdef CDL_Q_PLAIN_LDST
 #define CDL_LD(p) (*(p))
 #define CDL_ST(p, v) (*(p) = (v))
@@ -366,7 +369,7 @@ __device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }   // a - b, one rounding
 
 template <int MODE, bool RATE>
-__device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const float *__restrict__ Ltab, float2 x, float2 g)
+__device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const float2 *__restrict__ Dtab, float2 x, float2 g)
 {
     constexpr bool kRate = RATE && MODE == MODE_BWD;
     PairOut o;
@@ -417,9 +420,10 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
         const float2 covj = sub2(m1, __fmul2_rn(m1, m2));
         float2 gx = __fmul2_rn(g, __fmul2_rn(f2(P.a2), varj));
         if (kRate) {
-            const float Lc0 = Ltab[k0 - P.lo], Lc1 = Ltab[k1 - P.lo];
-            const float2 l1 = __fmul2_rn(make_float2(Ltab[min(k0 + 1, P.hi) - P.lo] - Lc0, Ltab[min(k1 + 1, P.hi) - P.lo] - Lc1), e1);
-            const float2 lm = __fmul2_rn(make_float2(Ltab[max(k0 - 1, P.lo) - P.lo] - Lc0, Ltab[max(k1 - 1, P.lo) - P.lo] - Lc1), em);
+            // log2 p of the upper / lower neighbour relative to the level's own: one 8-byte table entry per element
+            const float2 d0 = Dtab[k0 - P.lo], d1 = Dtab[k1 - P.lo];
+            const float2 l1 = __fmul2_rn(make_float2(d0.x, d1.x), e1);
+            const float2 lm = __fmul2_rn(make_float2(d0.y, d1.y), em);
             const float2 rate = __fmul2_rn(sub2(sub2(l1, lm), __fmul2_rn(m1, __fadd2_rn(l1, lm))), rS);
             gx = __ffma2_rn(f2(P.rate_c), rate, gx);
         }
@@ -428,8 +432,8 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
         const float2 dmk = __ffma2_rn(kn, f2(-q), dh);                 // d - kn q
         const float2 dq = __ffma2_rn(f2(P.two_aq), sub2(__fmul2_rn(dmk, varj), qc), __fadd2_rn(kn, m1));
         const float2 da = __fmul2_rn(f2(P.q2), sub2(__fmul2_rn(__fmul2_rn(f2(2.0f), dh), varj), qc));
-        o.tq = __fmul2_rn(g, dq);
-        o.ta = __fmul2_rn(g, da);
+        o.tq = dq;          // the caller accumulates g * dq and g * da
+        o.ta = da;
     }
     return o;
 }
@@ -461,10 +465,17 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) mp_s[k] = 0ull;
     }
 
+    constexpr bool kPairRate = MODE == MODE_BWD && RATE && PATH == PATH_NEAR3;
+    __shared__ float2 Dtab[kPairRate ? CDL_MAX_LEVELS : 1];     // (L[k+1] - L[k], L[k-1] - L[k]), clamped at the ends
     if (MODE == MODE_BWD && RATE) {
-        for (int k = threadIdx.x; k < P.nlev; k += kThreads) {
+        auto log2p = [&](int k) {
             const float p = P.level_prob[k];
-            Ltab[k] = (p < 9.31322574615478515625e-10f) ? -30.0f : log2f(p);   // 2^-30
+            return (p < 9.31322574615478515625e-10f) ? -30.0f : log2f(p);   // 2^-30
+        };
+        for (int k = threadIdx.x; k < P.nlev; k += kThreads) {
+            const float Lk = log2p(k);
+            Ltab[k] = Lk;
+            if (kPairRate) Dtab[k] = make_float2(log2p(min(k + 1, P.nlev - 1)) - Lk, log2p(max(k - 1, 0)) - Lk);
         }
     }
     if (do_hist)
@@ -481,8 +492,31 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     float4 *gx4 = reinterpret_cast<float4 *>(gx + head);
     unsigned int *idx4 = reinterpret_cast<unsigned int *>(idx + head);
 
+#if CDL_Q_PREFETCH
+    float4 xn[kBatch], gn[kBatch];
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+        const int64_t i = tid + b * stride;
+        if (i < n4) {
+            xn[b] = CDL_LD(x4 + i);
+            if (MODE == MODE_BWD) gn[b] = CDL_LD(g4 + i);
+        }
+    }
+#endif
     for (int64_t base = tid; base < n4; base += stride * kBatch) {
         float4 xv[kBatch], gv[kBatch];
+#if CDL_Q_PREFETCH
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            xv[b] = xn[b];
+            if (MODE == MODE_BWD) gv[b] = gn[b];
+            const int64_t i = base + stride * kBatch + b * stride;
+            if (i < n4) {
+                xn[b] = CDL_LD(x4 + i);
+                if (MODE == MODE_BWD) gn[b] = CDL_LD(g4 + i);
+            }
+        }
+#else
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             const int64_t i = base + b * stride;
@@ -491,7 +525,9 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 if (MODE == MODE_BWD) gv[b] = CDL_LD(g4 + i);
             }
         }
+#endif
         float part_q = 0.0f, part_a = 0.0f;
+        float2 part_q2 = make_float2(0.0f, 0.0f), part_a2 = make_float2(0.0f, 0.0f);    // pair path: two running sums each
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             const int64_t i = base + b * stride;
@@ -524,14 +560,17 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 if (kPairs) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const PairOut o = quant_pair_near3<MODE, RATE>(P, Ltab, make_float2(xs[2 * h], xs[2 * h + 1]),
+                        const PairOut o = quant_pair_near3<MODE, RATE>(P, Dtab, make_float2(xs[2 * h], xs[2 * h + 1]),
                                                                        make_float2(gs[2 * h], gs[2 * h + 1]));
                         ys[2 * h] = o.y.x;
                         ys[2 * h + 1] = o.y.y;
                         gxs[2 * h] = o.gx.x;
                         gxs[2 * h + 1] = o.gx.y;
-                        part_q += o.tq.x + o.tq.y;
-                        part_a += o.ta.x + o.ta.y;
+                        if (MODE == MODE_BWD) {
+                            const float2 gg = make_float2(gs[2 * h], gs[2 * h + 1]);
+                            part_q2 = __ffma2_rn(gg, o.tq, part_q2);
+                            part_a2 = __ffma2_rn(gg, o.ta, part_a2);
+                        }
                         packed |= (((unsigned int)o.k0[0] & 0xffu) | (((unsigned int)o.k0[1] & 0xffu) << 8)) << (16 * h);
                         if (MODE != MODE_BWD && do_hist) {
                             hist_add(hist_s, o.k0[0] - P.lo, lane);
@@ -555,8 +594,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
             }
         }
         if (MODE == MODE_BWD) {
-            acc_q += (double)part_q;
-            acc_a += (double)part_a;
+            acc_q += (double)(part_q + (part_q2.x + part_q2.y));
+            acc_a += (double)(part_a + (part_a2.x + part_a2.y));
         }
     }
 
