@@ -12,7 +12,7 @@
 // pipeline stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is
 // [rows][128 bytes] with the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or
 // columns outside the matrix are zero-filled by TMA, which makes ragged edges and R tails exact.
-// Warp roles (320 threads): warp 0 issues TMA, warp 1 owns TMEM and issues the MMAs, warps 2-9 run the
+// Warp roles (352 threads): warps 0 and 10 issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs, warps 2-9 run the
 // epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
 // Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to the warp's
 // swizzled 32 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that
@@ -30,7 +30,11 @@ namespace cdl {
 namespace {
 
 constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each taking every other 32-column chunk
-constexpr int kThreadsTC = 64 + 32 * kEpiWarps;
+#ifndef CDL_G_SPLIT_PRODUCER
+#define CDL_G_SPLIT_PRODUCER 1
+#endif
+constexpr bool kSplitProducer = CDL_G_SPLIT_PRODUCER != 0;   // a second TMA warp issues the Y-operand loads
+constexpr int kThreadsTC = 64 + 32 * kEpiWarps + (kSplitProducer ? 32 : 0);
 // Shared memory is divided between operand stages and epilogue staging blocks (4 KB each, per epilogue warp).
 // Which of the two needs the bytes in flight depends on the shape: a long reduced dimension loads much more than
 // it stores, a short one (two stages per 128 KB of output) the opposite.
@@ -384,8 +388,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const uint32_t stage_tx = (uint32_t)kABytes + b_bytes;
     bool failed = false;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer (one lane)
+    if (warp == 0 || warp == 2 + kEpiWarps) {
+        // ------------------------------------------------------------ TMA producer (one lane; with a second TMA
+        // warp the first issues the X-operand loads and arms the barrier, the second issues the Y-operand loads)
+        const bool do_a = warp == 0, do_b = !kSplitProducer || warp != 0;
         if (lane == 0) {
             uint32_t it = 0;
             for (int u = cta_first; u < units && !failed; u += cta_step) {
@@ -450,18 +456,25 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     }
                     if (PAIR) {
                         // both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
-                        if (rank == 0) mbar_expect_tx(full_bar(s), 2u * stage_tx);
-                        if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
-                        else if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
-                        else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
-                        if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, b_row, b_red, full_bar(s));
-                        else tma_load_2d_pair(sb, &map_b, b_red, b_row, full_bar(s));
+                        if (rank == 0 && do_a) mbar_expect_tx(full_bar(s), 2u * stage_tx);
+                        if (do_a) {
+                            if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
+                            else if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
+                            else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
+                        }
+                        if (do_b) {
+                            if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, b_row, b_red, full_bar(s));
+                            else tma_load_2d_pair(sb, &map_b, b_red, b_row, full_bar(s));
+                        }
                         continue;
                     }
-                    mbar_expect_tx(full_bar(s), stage_tx);
-                    if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
-                    else if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
-                    else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
+                    if (do_a) {
+                        mbar_expect_tx(full_bar(s), stage_tx);
+                        if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
+                        else if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
+                        else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
+                    }
+                    if (!do_b) continue;
                     if (P.b_mn_major) {
                         for (int bb = 0; bb < b_blocks; ++bb)
                             tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, b_row + bb * 128, b_red, full_bar(s));
