@@ -240,6 +240,27 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
                     void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Backward layer products for a real-valued incoming gradient (Algorithm 1's backward pass as printed: dL/dY is
+ * not quantized there; cdl_qlinear_bwd is the int8-gradient reading).  The gradient is expanded in two int8 digits,
+ *   g ~ q1 i1 + q2 i2,  q1 = g_absmax / 127,  q2 = q1 / 254,
+ *   i1 = clamp(rint(g / q1), -127, 127),  i2 = clamp(rint(RN(g - i1 q1) / q2), -127, 127)      (binary32),
+ * so |g - (q1 i1 + q2 i2)| <= q1 / 508 = g_absmax / 64516 for |g| <= g_absmax (larger entries saturate), and each
+ * digit plane goes through the exact integer product of cdl_qlinear_bwd:
+ *   dX[m,k] = RN(RN((float)(I1 W^T)[m,k] * (q1 w->q)) + RN((float)(I2 W^T)[m,k] * (q2 w->q)))      and dW likewise with a->q.
+ * Against the products with the real gradient the error is at most (g_absmax / 64516) * sum_n |w->q W_idx[k,n]| per
+ * entry of dX (sum_m |a->q A_idx[m,k]| for dW) plus binary32 rounding of the result.
+ *   G [dev] M x N floats (row pitch N); g_absmax > 0: the caller's bound on |G|.
+ *   dX [dev] M x K floats, dW [dev] K x N floats, each nullable; A_idx / W_idx as in cdl_qlinear_bwd.
+ *   ws [dev]: cdl_qlinear_bwd_fp_workspace_bytes(M, N, K) bytes (holds the two digit planes), 256-byte aligned.
+ */
+int cdl_qlinear_bwd_fp(const float *G, float g_absmax,
+                       const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                       const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                       int32_t M, int32_t N, int32_t K, float *dX, float *dW,
+                       void *ws, size_t ws_bytes, void *stream);
+size_t cdl_qlinear_bwd_fp_workspace_bytes(int32_t M, int32_t N, int32_t K);
+
+/*
  * Weight-gradient product for callers that cannot allocate device memory.  (The paper has no counterpart
  * of this entry point; it is a packaging variant of the dW half of cdl_qlinear_bwd.)
  *

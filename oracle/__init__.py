@@ -250,6 +250,22 @@ def conv_dw(X, G, R, S, pad_h, pad_w):
     return acc
 
 
+def gradient_digits(G, g_absmax):
+    """Two-digit integer expansion of a real gradient tensor (backward products with an unquantized dL/dY):
+    q1 = g_absmax / 127, q2 = q1 / 254 (binary32), i1 = hard index of g on step q1 in [-127, 127], r = the binary32
+    value nearest g - i1 q1, i2 = hard index of r on step q2.  Returns (i1, i2, q1, q2)."""
+    f32 = np.float32
+    G = _f32(G)
+    q1 = f32(f32(g_absmax) / f32(127.0))
+    q2 = f32(q1 / f32(254.0))
+    i1, _ = hard(G.reshape(-1), q1, -127, 127)
+    # g - i1 q1 with one rounding: the product has at most 31 significant bits and the difference of two nearby
+    # numbers is exact in binary64, so rounding the binary64 result to binary32 is the fused operation
+    r = (G.reshape(-1).astype(np.float64) - i1.astype(np.float64) * np.float64(q1)).astype(f32)
+    i2, _ = hard(r, q2, -127, 127)
+    return i1.reshape(G.shape), i2.reshape(G.shape), q1, q2
+
+
 def huffman_lengths(hist):
     """Code lengths of a Huffman code for the symbols with a non-zero count (Sec. VI-B: the average number of bits per
     weight / activation is measured with Huffman coding), by the textbook construction: repeatedly merge the two

@@ -504,4 +504,74 @@ int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx,
     return CDL_OK;
 }
 
+namespace {
+size_t align256(size_t v) { return (v + 255u) & ~(size_t)255u; }
+int64_t ld16(int64_t n) { return (n + 15) / 16 * 16; }
+}  // namespace
+
+size_t cdl_qlinear_bwd_fp_workspace_bytes(int32_t M, int32_t N, int32_t K)
+{
+    const size_t base = cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K);
+    if (base == 0) return 0;
+    return align256(base) + 2 * align256((size_t)M * (size_t)ld16(N));
+}
+
+int cdl_qlinear_bwd_fp(const float *G, float g_absmax, const void *A_idx, int64_t lda, const cdl_index_desc *a,
+                       const void *W_idx, int64_t ldw, const cdl_index_desc *w, int32_t M, int32_t N, int32_t K,
+                       float *dX, float *dW, void *ws, size_t ws_bytes, void *stream)
+{
+    if (G == nullptr || M <= 0 || N <= 0 || K <= 0 || (dX == nullptr && dW == nullptr)) return CDL_ERR_ARG;
+    if (!(g_absmax > 0.0f) || !(g_absmax < 1e30f)) return CDL_ERR_RANGE;
+    if ((dX != nullptr && W_idx == nullptr) || (dW != nullptr && A_idx == nullptr)) return CDL_ERR_ARG;
+    if (bad_f32_ptr(G)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qlinear_bwd_fp_workspace_bytes(M, N, K))
+        return CDL_ERR_WORKSPACE;
+    const float q1 = g_absmax / 127.0f, q2 = q1 / 254.0f;
+    const int64_t ldg = ld16(N);
+    const size_t base = align256(cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K));
+    const size_t plane = align256((size_t)M * (size_t)ldg);
+    char *d1 = static_cast<char *>(ws) + base, *d2 = d1 + plane;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ldg != N) {      // the pad columns are operands of the TMA loads: keep them defined
+        if (cudaMemsetAsync(d1, 0, 2 * plane, st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CDL_ERR_LAUNCH;
+        }
+    }
+    if ((rc = launch_gradient_digits(G, M, N, (int)ldg, q1, q2, d1, d2, st)) != CDL_OK) return rc;
+    const cdl_index_desc g1{q1, -127, 127}, g2{q2, -127, 127};
+    // first digit stores, second digit adds: dX = RN(RN(acc1 s1) + RN(acc2 s2))
+    IndexRange rg{false, 127}, ra{false, 0}, rw{false, 0};
+    if (dW != nullptr && (rc = index_range(a, &ra)) != CDL_OK) return rc;
+    if (dX != nullptr) {
+        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+        if ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u) || ldw < N) return CDL_ERR_ALIGN;
+    }
+    if (dW != nullptr && ((lda & 15) || (reinterpret_cast<uintptr_t>(A_idx) & 15u) || lda < K)) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(dX) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    char *scratch = static_cast<char *>(ws) + kStatusBytes;
+    for (int pass = 0; pass < 2; ++pass) {
+        const char *dig = pass == 0 ? d1 : d2;
+        const float qg = pass == 0 ? g1.q : g2.q;
+        if (dX != nullptr) {
+            GemmOperand X{dig, ldg, 1, false, (int)rg.absmax};
+            GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
+            rc = launch_index_gemm_tc(X, Y, M, K, N, nullptr, dX, (qg * w->q), nullptr, scratch, static_cast<int *>(ws), st,
+                                      nullptr, nullptr, pass == 1);
+            if (rc != CDL_OK) return rc;
+        }
+        if (dW != nullptr) {
+            GemmOperand X{A_idx, 1, lda, ra.is_unsigned, (int)ra.absmax};
+            GemmOperand Y{dig, 1, ldg, false, (int)rg.absmax};
+            rc = launch_index_gemm_tc(X, Y, K, N, M, nullptr, dW, (qg * a->q), nullptr, scratch, static_cast<int *>(ws), st,
+                                      nullptr, nullptr, pass == 1);
+            if (rc != CDL_OK) return rc;
+        }
+    }
+    return CDL_OK;
+}
+
 }  // extern "C"

@@ -66,6 +66,7 @@ struct TcParams {
     int32_t *acc_out;       // int32 output or accumulation buffer (required when splits > 1)
     float *f_out;           // float output (written by the epilogue only when splits == 1)
     float scale;
+    int f_acc;              // 1: the float output is added to what f_out holds (one binary32 addition per element)
     const float *bias;
     int *status;
     int tma_f, tma_acc;     // the float / int32 output goes through shared memory and TMA
@@ -579,7 +580,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // Same staging, then the warp copies its 32 rows out itself, one row (up to 128 contiguous bytes) per
         // instruction: for outputs TMA cannot take (row pitch or base not a multiple of 16 bytes, 16-column tiles).
         auto stage_and_copy = [&](const uint32_t (&w)[32], int32_t *out, bool reduce, long long row_off, int row0,
-                                  int col0, int ncol) {
+                                  int col0, int ncol, bool as_float = false) {
             const uint32_t blk = stage(w);
             __syncwarp();
             for (int rr = 0; rr < 32; ++rr) {
@@ -590,7 +591,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                              : "r"(blk + (uint32_t)rr * 128u + (uint32_t)(((lane >> 2) ^ (rr & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
                 if (lane < ncol) {
                     int32_t *q = out + (row_off + grow) * P.J + col0 + lane;
-                    if (reduce) asm volatile("red.global.add.s32 [%0], %1;" ::"l"(q), "r"(val) : "memory");
+                    if (reduce && as_float) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(q), "f"(__uint_as_float(val)) : "memory");
+                    else if (reduce) asm volatile("red.global.add.s32 [%0], %1;" ::"l"(q), "r"(val) : "memory");
                     else *q = (int32_t)val;
                 }
             }
@@ -662,8 +664,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         }
                     }
                     if (P.f_out != nullptr) {
-                        if (P.tma_f) stage_and_send(f, &map_f, false, col0, wrow0, P.I);
-                        else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), false, 0, wrow0, col0, ncol);
+                        if (P.tma_f) stage_and_send(f, &map_f, P.f_acc != 0, col0, wrow0, P.I);
+                        else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), P.f_acc != 0, 0, wrow0, col0, ncol, true);
                     }
                 }
             };
@@ -710,20 +712,20 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
 // float output of a split run: f = (float)acc * scale (+ bias[j])
 __global__ void scale_acc_kernel(const int32_t *__restrict__ acc, float *__restrict__ f, long long n, int J, float scale,
-                                 const float *__restrict__ bias)
+                                 const float *__restrict__ bias, int accumulate)
 {
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
         float v = __fmul_rn((float)acc[i], scale);
         if (bias != nullptr) v = __fadd_rn(v, bias[i % J]);
-        f[i] = v;
+        f[i] = accumulate ? __fadd_rn(f[i], v) : v;
     }
 }
 
 // float output of a split run whose partial sums sit in per-split slabs: the slabs are summed in int64 (each
 // slab is exact in int32, the total need not be), converted once and scaled.
 __global__ void sum_slabs_kernel(const int32_t *__restrict__ slabs, int splits, long long slab_elems, float *__restrict__ f,
-                                 long long n, int J, float scale, const float *__restrict__ bias)
+                                 long long n, int J, float scale, const float *__restrict__ bias, int accumulate)
 {
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
@@ -731,7 +733,7 @@ __global__ void sum_slabs_kernel(const int32_t *__restrict__ slabs, int splits, 
         for (int sp = 0; sp < splits; ++sp) acc += (long long)slabs[sp * slab_elems + i];
         float v = __fmul_rn(__ll2float_rn(acc), scale);
         if (bias != nullptr) v = __fadd_rn(v, bias[i % J]);
-        f[i] = v;
+        f[i] = accumulate ? __fadd_rn(f[i], v) : v;
     }
 }
 
@@ -880,7 +882,7 @@ size_t tc_gemm_scratch_bytes(int I, int J, int R)
 // bytes, used only when the reduced dimension is split and no int32 output was requested.
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream, const ConvGather *conv, const NextQuant *next)
+                         cudaStream_t stream, const ConvGather *conv, const NextQuant *next, bool accumulate_f)
 {
     const bool a_mn = conv != nullptr ? conv->transposed != 0 : (X.stride_outer == 1 && X.stride_red != 1);
     const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
@@ -940,6 +942,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         P.y_tap_rows = conv->y_tap_rows;
     }
     P.scale = scale;
+    P.f_acc = accumulate_f ? 1 : 0;
     P.bias = bias;
     P.status = status;
     P.f_out = f_out;
@@ -1049,9 +1052,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     if (f_out != nullptr && (splits > 1 || wide)) {
         const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
         if (wide)
-            sum_slabs_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, splits, (long long)P.slab_rows * J, f_out, n_out, J, scale, bias);
+            sum_slabs_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, splits, (long long)P.slab_rows * J, f_out, n_out, J, scale, bias, P.f_acc);
         else
-            scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias);
+            scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias, P.f_acc);
         if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     }
     return CDL_OK;

@@ -53,6 +53,8 @@ struct GemmOperand {
     int absmax;             // bound on |entry| (from the operand's declared index range)
 };
 
+int launch_gradient_digits(const float *g, long long rows, int cols, int ld, float q1, float q2, void *d1, void *d2,
+                           cudaStream_t stream);
 int launch_huffman(const unsigned long long *hist, int nlev, unsigned char *lengths, unsigned long long *total_bits,
                    double *avg_bits, cudaStream_t stream);
 
@@ -80,6 +82,7 @@ struct NextQuant {
 size_t tc_gemm_scratch_bytes(int I, int J, int R);
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream, const ConvGather *conv = nullptr, const NextQuant *next = nullptr);
+                         cudaStream_t stream, const ConvGather *conv = nullptr, const NextQuant *next = nullptr,
+                         bool accumulate_f = false);   // accumulate_f: f_out += result instead of f_out = result
 
 }  // namespace cdl

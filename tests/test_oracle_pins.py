@@ -397,3 +397,22 @@ def test_soft_histogram_two_levels_closed_form():
     s = oracle.mpmf(x, q, 0, 1, alpha)
     sig = 1.0 / (1.0 + np.exp(-float(alpha) * float(q) * (2.0 * x.astype(np.float64) - float(q))))
     assert s[1] == pytest.approx(sig.sum(), rel=1e-12) and s[0] == pytest.approx((1 - sig).sum(), rel=1e-12)
+
+
+def test_gradient_digits_reconstruct_the_gradient_within_half_a_fine_step():
+    # pins the two-digit expansion to its defining property: |g - (q1 i1 + q2 i2)| <= q2 / 2 inside the range,
+    # digits within [-127, 127], and saturation outside
+    rng = np.random.default_rng(3)
+    g = rng.normal(0, 1e-2, 20000).astype(np.float32)
+    absmax = float(np.abs(g).max())
+    i1, i2, q1, q2 = oracle.gradient_digits(g, absmax)
+    assert np.abs(i1).max() <= 127 and np.abs(i2).max() <= 127
+    rec = np.float64(q1) * i1 + np.float64(q2) * i2
+    assert np.abs(g.astype(np.float64) - rec).max() <= float(q2) / 2 * (1 + 1e-6)
+    assert np.isclose(float(q2) * 254, float(q1), rtol=1e-6) and np.isclose(float(q1) * 127, absmax, rtol=1e-6)
+    # a bound smaller than the data: both digits saturate with the sign of g
+    i1s, i2s, _, _ = oracle.gradient_digits(np.array([1.0, -1.0], dtype=np.float32), 0.5)
+    assert list(i1s) == [127, -127] and list(i2s) == [127, -127]
+    # exact multiples of the coarse step have a zero fine digit
+    i1m, i2m, q1m, _ = oracle.gradient_digits((np.arange(-5, 6) * np.float32(2.0 / 127)).astype(np.float32), 2.0)
+    assert list(i1m) == list(range(-5, 6)) and not i2m.any()
