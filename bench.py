@@ -51,6 +51,8 @@ def parse_args():
                     choices=["resnet18_layer3_conv", "cifar_resnet20_conv", "tiny", "resnet18_b256"])
     ap.add_argument("--batch", type=int, default=256, help="batch size of the resnet18_b256 workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--conv-form", action="store_true",
+                    help="resnet18_b256: run the layers that cdl_qconv_* supports in convolution form")
     ap.add_argument("--no-implicit", action="store_true", help="skip the extra measurement of the layer in convolution form")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step one by one instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
@@ -488,21 +490,24 @@ def run_network(args):
         x = torch.randn(n_x, device="cuda", generator=gen).abs_()
         wq = inputs.Quantizer(float(w.std()) / 3.0, -3, 3, 100.0, 0.01, 0)
         xq = inputs.Quantizer(float(2.0 * x.mean() / 8.0 ** 0.5), 0, 15, 100.0, 0.01, 5)
-        st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g, need_dx=(name != "conv1"))   # the image needs no gradient
+        geo = inputs.resnet18_conv_geometry(name) if args.conv_form else None
+        shape = cdl.ConvShape(args.batch, geo[0], geo[1], geo[2], geo[3], geo[4]) if geo else None
+        st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g, need_dx=(name != "conv1"), conv=shape)   # the image needs no gradient
         st.w.copy_(w)
         st.x.copy_(x)
         del w, x
-        # im2col index matrix drawn from the quantized activations' own level histogram
-        hist = torch.zeros(16, dtype=torch.int64, device="cuda")
-        cdl.cdl_quantize_hard(st.x, n_x, cdl.QuantParams(xq.q, 0, 15), None, hist)
-        cdf = torch.cumsum(hist.double() / float(n_x), 0).float()
-        rows = max(1, (1 << 26) // K)
-        for r0 in range(0, M, rows):
-            r1 = min(M, r0 + rows)
-            u = torch.rand((r1 - r0, K), device="cuda", generator=gen)
-            st.A_idx[r0:r1, :K] = torch.searchsorted(cdf, u).clamp_(max=15).to(torch.uint8)
+        if shape is None:
+            # im2col index matrix drawn from the quantized activations' own level histogram
+            hist = torch.zeros(16, dtype=torch.int64, device="cuda")
+            cdl.cdl_quantize_hard(st.x, n_x, cdl.QuantParams(xq.q, 0, 15), None, hist)
+            cdf = torch.cumsum(hist.double() / float(n_x), 0).float()
+            rows = max(1, (1 << 26) // K)
+            for r0 in range(0, M, rows):
+                r1 = min(M, r0 + rows)
+                u = torch.rand((r1 - r0, K), device="cuda", generator=gen)
+                st.A_idx[r0:r1, :K] = torch.searchsorted(cdf, u).clamp_(max=15).to(torch.uint8)
+            st.gx_in.copy_(torch.randn(n_x, device="cuda", generator=gen))
         st.dY.copy_(torch.randn((M, Np), device="cuda", generator=gen) * G_STD)
-        st.gx_in.copy_(torch.randn(n_x, device="cuda", generator=gen))
         layers.append((name, M, K, N, n_x, st))
     torch.cuda.synchronize()
 
@@ -515,6 +520,26 @@ def run_network(args):
     for _ in range(warm):
         run_all()
     torch.cuda.synchronize()
+    # the whole network step as one CUDA graph (each layer recorded on three streams), replayed `steps` times
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for *_, st in layers:
+                    st.run_forked()
+        stream.wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for _ in range(steps):
+            graph.replay()
+        g1.record(stream)
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / steps
     ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in layers] for _ in range(steps)]
     cnt = {}
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -535,6 +560,9 @@ def run_network(args):
     torch.cuda.synchronize()
     clocks = sampler.stop(wall0, time.time())
     ms_step = t0.elapsed_time(t1) / steps
+    call_by_call_ms = ms_step
+    if graph is not None:
+        ms_step = graph_ms
     pk, pk_kind = peaks()
     hbm = float(pk["hbm_gbs"])
     table, tot_ops, tot_q, gemm_ms, quant_ms = [], 0.0, 0, 0.0, 0.0
@@ -557,7 +585,12 @@ def run_network(args):
         "metric": METRIC, "value": tot_q / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32+s8",
         "data": "synthetic",
-        "config": {"workload": "resnet18_b256", "batch": args.batch, "layers": len(layers), "weight_levels": 7,
+        "config": {"workload": "resnet18_b256", "batch": args.batch, "layers": len(layers),
+                   "form": ("convolution form for the %d stride-1 3x3 layers with >= 128 channels, stored patch matrices "
+                            "for the rest" % sum(1 for *_, st in layers if st.conv is not None)) if args.conv_form
+                   else "stored patch matrices (im2col GEMMs)",
+                   "launch": "stream launches" if graph is None else "CUDA graph replay of the network step",
+                   "call_by_call_ms": call_by_call_ms, "weight_levels": 7,
                    "activation_levels": 16, "window_x": 5, "l2": "every layer's tensors exceed the 126 MB L2"},
         "network_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": tot_ops / (gemm_ms * 1e-3) / 1e12,
         "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": tot_q / (quant_ms * 1e-3) / 1e9,

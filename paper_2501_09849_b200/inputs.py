@@ -156,3 +156,14 @@ def resnet18_layers(batch: int = 256):
     L += [("layer4.ds", b * 7 * 7, 256, 512, b * 14 * 14 * 256)]
     L += [("fc", b, 512, 1000, b * 512)]
     return L
+
+
+def resnet18_conv_geometry(name: str):
+    """(H, W, C, R, S) of the ResNet-18 layers that are stride-1 3x3 convolutions over at least 128 channels (the
+    layers the convolution form of the products covers), else None."""
+    side = {"layer2": (28, 128), "layer3": (14, 256), "layer4": (7, 512)}
+    stage, _, idx = name.partition(".")
+    if stage in side and idx in ("1", "2", "3"):
+        hw, c = side[stage]
+        return hw, hw, c, 3, 3
+    return None
