@@ -586,7 +586,7 @@ def run_network(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32+s8",
         "data": "synthetic",
         "config": {"workload": "resnet18_b256", "batch": args.batch, "layers": len(layers),
-                   "form": ("convolution form for the %d stride-1 3x3 layers with >= 128 channels, stored patch matrices "
+                   "form": ("convolution form for the %d stride-1 3x3 layers, stored patch matrices "
                             "for the rest" % sum(1 for *_, st in layers if st.conv is not None)) if args.conv_form
                    else "stored patch matrices (im2col GEMMs)",
                    "launch": "stream launches" if graph is None else "CUDA graph replay of the network step",

@@ -296,7 +296,7 @@ int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_d
  * tensors: the patch matrix whose rows cdl_qlinear_* takes as A_idx is never written to memory, its tiles are
  * gathered by the loads of the kernel, with zero (= index 0 = level 0) outside the image.
  * Stride 1, filter R x S with R and S odd, padding (R-1)/2 and (S-1)/2: the output has the spatial size of the
- * input (3 x 3 and 1 x 1 layers of a ResNet).  C and C_out multiples of 128 (else CDL_ERR_ARG: form the patch
+ * input (3 x 3 and 1 x 1 layers of a ResNet).  C and C_out multiples of 64 (else CDL_ERR_ARG: form the patch
  * matrix and call cdl_qlinear_*).
  *   X_idx [dev] N x H x W x C index bytes (signedness from x);  G_idx [dev] N x H x W x C_out int8;
  *   W_idx [dev] (R*S*C) x C_out int8, row (r*S + s)*C + c, leading dimension ldw (multiple of 16);

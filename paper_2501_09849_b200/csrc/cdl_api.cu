@@ -386,10 +386,10 @@ bool conv_dims(const cdl_conv_shape *s, int32_t C_out, int64_t *M, int *taps)
 {
     if (s == nullptr || s->N <= 0 || s->H <= 0 || s->W <= 0 || s->C <= 0 || C_out <= 0) return false;
     if (s->R <= 0 || s->S <= 0 || (s->R & 1) == 0 || (s->S & 1) == 0 || s->R > 127 || s->S > 127) return false;
-    if ((s->C % 128) != 0 || (C_out % 128) != 0) return false;
+    if ((s->C % 64) != 0 || (C_out % 64) != 0) return false;
     *M = (int64_t)s->N * s->H * s->W;
     *taps = s->R * s->S;
-    if (*M > 0x7fffff00ll || (int64_t)*taps * s->C > 0x7fffff00ll || (int64_t)*taps * C_out > 0x7fffff00ll) return false;
+    if (*M > 0x7fffff00ll || (int64_t)*taps * (s->C + 64) > 0x7fffff00ll || (int64_t)*taps * (C_out + 64) > 0x7fffff00ll) return false;
     return true;
 }
 }  // namespace
@@ -399,9 +399,11 @@ size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
     int64_t M;
     int taps;
     if (!conv_dims(shape, C_out, &M, &taps)) return 0;
-    const size_t f = tc_gemm_scratch_bytes((int)M, C_out, taps * shape->C);
-    const size_t dx = tc_gemm_scratch_bytes((int)M, shape->C, taps * C_out);
-    const size_t dw = tc_gemm_scratch_bytes(taps * shape->C, C_out, (int)M);
+    // the tiling pads every tap to whole 128-channel blocks
+    const int cp = (shape->C + 127) / 128 * 128, cop = (C_out + 127) / 128 * 128;
+    const size_t f = tc_gemm_scratch_bytes((int)M, C_out, taps * cp);
+    const size_t dx = tc_gemm_scratch_bytes((int)M, shape->C, taps * cop);
+    const size_t dw = tc_gemm_scratch_bytes(taps * cp, C_out, (int)M);
     size_t m = f > dx ? f : dx;
     if (dw > m) m = dw;
     return kStatusBytes + m;

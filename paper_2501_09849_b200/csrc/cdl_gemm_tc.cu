@@ -56,7 +56,8 @@ constexpr int kPlanSMs = 148;           // B200: splits are planned for this cou
 constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s
 
 struct TcParams {
-    int I, J, R;            // output rows, output columns, reduced extent
+    int I, J, R;            // rows the tiling runs over, output columns, reduced extent of the tiling
+    int I_out;              // rows of the output matrix (differs from I only for a padded transposed patch matrix)
     int TN;                 // output columns per tile (multiple of 16, <= 256)
     int tiles_i, tiles_j;   // tile grid
     int splits;             // splits of the reduced dimension
@@ -74,7 +75,8 @@ struct TcParams {
     // tensor instead of being read from a stored matrix.
     int conv;               // 0: stored matrix; 1: X(i = pixel, r = tap * C + c); 2: X(i = tap * C + c, r = pixel)
     int cH, cW, cC, cS;     // image height and width, channels, filter width
-    int cblocks;            // 128-channel blocks per tap (C / 128)
+    int cblocks;            // 128-channel blocks per tap (C rounded up to 128: channels past C read as zero)
+    int cpad;               // 128 * cblocks
     int pad_h, pad_w;
     int taps;               // R * S
     int y_tap_rows;         // > 0: the Y block of tap t starts at row (taps - 1 - t) * y_tap_rows of the stored matrix
@@ -408,9 +410,9 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 if (P.conv != 0) {
                     // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
                     const int i0 = arow < P.I ? arow : 0;
-                    g_tap = P.conv == 1 ? rb0 / P.cblocks : i0 / P.cC;
+                    g_tap = P.conv == 1 ? rb0 / P.cblocks : i0 / P.cpad;
                     g_cb = P.conv == 1 ? rb0 % P.cblocks : 0;
-                    g_c0 = P.conv == 1 ? 0 : i0 % P.cC;
+                    g_c0 = P.conv == 1 ? 0 : i0 % P.cpad;
                     const int pix = P.conv == 1 ? i0 : rb0 * BR;
                     g_n = pix / (P.cH * P.cW);
                     const int rem = pix - g_n * (P.cH * P.cW);
@@ -431,7 +433,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const uint32_t sb = sa + kABytes;
                     int b_row = tj * P.TN + brow;
                     if (P.y_tap_rows > 0) b_row += (P.taps - 1 - g_tap) * P.y_tap_rows;
-                    const int b_red = P.y_tap_rows > 0 ? g_cb * BR : rb * BR;   // Y coordinate along r
+                    // Y coordinate along r: the stored matrix has C (not the padded count) rows per tap
+                    const int b_red = P.y_tap_rows > 0 ? g_cb * BR : (P.conv == 1 ? g_tap * P.cC + g_cb * BR : rb * BR);
                     const int g_c = P.conv == 1 ? g_cb * BR : g_c0;
                     const int c_w = g_w - P.pad_w, c_h = g_h - P.pad_h, c_n = g_n, c_ow = g_ow, c_oh = g_oh;
                     if (P.conv == 1) {            // next stage: next channel block, then next tap
@@ -585,7 +588,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             __syncwarp();
             for (int rr = 0; rr < 32; ++rr) {
                 const int grow = row0 + rr;
-                if (grow >= P.I) break;                                    // uniform over the warp
+                if (grow >= P.I_out) break;                                // uniform over the warp
                 uint32_t val;
                 asm volatile("ld.shared.b32 %0, [%1];" : "=r"(val)
                              : "r"(blk + (uint32_t)rr * 128u + (uint32_t)(((lane >> 2) ^ (rr & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
@@ -611,10 +614,16 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 break;
             }
             tc_fence_after();
-            const int wrow0 = ti * TMU + (int)rank * TM + quarter * 32;     // first output row of this warp
+            // first output row of this warp; a transposed patch matrix whose taps are padded to 128 channels has
+            // rows that exist only in the tiling (never stored) and the others move up
+            int wrow0 = ti * TMU + (int)rank * TM + quarter * 32;
+            if (P.conv == 2 && P.cpad != P.cC) {
+                const int tap = wrow0 / P.cpad, c = wrow0 - tap * P.cpad;
+                wrow0 = c < P.cC ? tap * P.cC + c : 0x7fffff00;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
             const int tile_cols = min(P.TN, P.J - tj * P.TN);
-            const int nchunks = wrow0 < P.I ? (tile_cols + 31) / 32 : 0;   // uniform over the warp
+            const int nchunks = wrow0 < P.I_out ? (tile_cols + 31) / 32 : 0;   // uniform over the warp
 
             // one chunk = 32 columns of the warp's 32 rows
             auto emit = [&](const uint32_t (&v)[32], int ch) {
@@ -627,7 +636,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     return;
                 }
                 if (P.acc_out != nullptr) {
-                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, wrow0, P.I);
+                    if (P.tma_acc) stage_and_send(v, &map_acc, false, col0, wrow0, P.I_out);
                     else stage_and_copy(v, P.acc_out, false, 0, wrow0, col0, ncol);
                 }
                 if (P.f_out != nullptr || P.nq_out != nullptr) {
@@ -639,7 +648,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         for (int c = 0; c < 32; ++c)
                             if (c < ncol) f[c] = __float_as_uint(__fadd_rn(__uint_as_float(f[c]), P.bias[col0 + c]));
                     }
-                    if (P.nq_out != nullptr && wrow0 + lane < P.I) {
+                    if (P.nq_out != nullptr && wrow0 + lane < P.I_out) {
                         // the next layer's index of this thread's 32 outputs: 32 consecutive bytes of its row
                         uint32_t pk[8];
 #pragma unroll
@@ -664,7 +673,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         }
                     }
                     if (P.f_out != nullptr) {
-                        if (P.tma_f) stage_and_send(f, &map_f, P.f_acc != 0, col0, wrow0, P.I);
+                        if (P.tma_f) stage_and_send(f, &map_f, P.f_acc != 0, col0, wrow0, P.I_out);
                         else stage_and_copy(f, reinterpret_cast<int32_t *>(P.f_out), P.f_acc != 0, 0, wrow0, col0, ncol, true);
                     }
                 }
@@ -886,25 +895,33 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
 {
     const bool a_mn = conv != nullptr ? conv->transposed != 0 : (X.stride_outer == 1 && X.stride_red != 1);
     const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
+    // extents the tiling runs over: a patch matrix has its taps padded to whole 128-channel blocks
+    int It = I, Rt = R;
+    if (conv != nullptr) {
+        const int cpad = (conv->C + BR - 1) / BR * BR;
+        if (conv->transposed) It = conv->R * conv->S * cpad;
+        else Rt = conv->R * conv->S * cpad;
+    }
     TcParams P;
-    P.I = I;
+    P.I = It;
+    P.I_out = I;
     P.J = J;
-    P.R = R;
+    P.R = Rt;
     // Exactness: a part of the reduced dimension is summed in int32, so |sum| <= rows * xmax * ymax must stay
     // below 2^31 per part.  When the whole dimension does not satisfy that, it is cut into enough parts, each part
     // keeps its own slab, and the slabs are summed in int64 (float output only).
-    const bool wide = (long long)R * X.absmax * Y.absmax >= ((long long)1 << 31);
+    const bool wide = (long long)Rt * X.absmax * Y.absmax >= ((long long)1 << 31);
     if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
-    const Plan pl = plan(I, J, R, wide ? min_exact_splits(R, X.absmax, Y.absmax) : 1);
+    const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1);
     const bool want_next = next != nullptr && next->idx_out != nullptr;
     if (want_next && wide) return CDL_ERR_OVERFLOW_RISK;     // the index is taken from one finished accumulator
     const int TN = pl.TN, splits = want_next ? 1 : pl.splits;
     const bool pair = pl.pair != 0;
     P.TN = TN;
-    P.tiles_i = (I + pl.tile_rows - 1) / pl.tile_rows;
+    P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
     P.slab_rows = wide ? P.tiles_i * pl.tile_rows : 0;
     P.tiles_j = (J + TN - 1) / TN;
-    P.rblocks = (R + BR - 1) / BR;
+    P.rblocks = (Rt + BR - 1) / BR;
     const int sms = sm_count();
     if (sms <= 0) return CDL_ERR_LAUNCH;
     const long long tiles = (long long)P.tiles_i * P.tiles_j;
@@ -927,15 +944,16 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         P.nq_vec = ((J & 15) == 0 && (reinterpret_cast<uintptr_t>(next->idx_out) & 15u) == 0) ? 1 : 0;
     }
     P.conv = 0;
-    P.cH = P.cW = P.cC = P.cS = P.cblocks = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
+    P.cH = P.cW = P.cC = P.cS = P.cblocks = P.cpad = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
     if (conv != nullptr) {
-        if (conv->C % BR != 0 || (conv->R & 1) == 0 || (conv->S & 1) == 0) return CDL_ERR_ARG;
+        if (conv->C % 64 != 0 || (conv->R & 1) == 0 || (conv->S & 1) == 0) return CDL_ERR_ARG;
         P.conv = conv->transposed ? 2 : 1;
         P.cH = conv->H;
         P.cW = conv->W;
         P.cC = conv->C;
         P.cS = conv->S;
-        P.cblocks = conv->C / BR;
+        P.cblocks = (conv->C + BR - 1) / BR;
+        P.cpad = P.cblocks * BR;
         P.pad_h = (conv->R - 1) / 2;
         P.pad_w = (conv->S - 1) / 2;
         P.taps = conv->R * conv->S;

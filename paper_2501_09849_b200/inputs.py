@@ -159,11 +159,11 @@ def resnet18_layers(batch: int = 256):
 
 
 def resnet18_conv_geometry(name: str):
-    """(H, W, C, R, S) of the ResNet-18 layers that are stride-1 3x3 convolutions over at least 128 channels (the
-    layers the convolution form of the products covers), else None."""
-    side = {"layer2": (28, 128), "layer3": (14, 256), "layer4": (7, 512)}
+    """(H, W, C, R, S) of the ResNet-18 layers that are stride-1 3x3 convolutions with as many output as input
+    channels (the layers the convolution form of the products covers), else None."""
+    side = {"layer1": (56, 64), "layer2": (28, 128), "layer3": (14, 256), "layer4": (7, 512)}
     stage, _, idx = name.partition(".")
-    if stage in side and idx in ("1", "2", "3"):
+    if stage in side and (idx in ("1", "2", "3") or (stage == "layer1" and idx == "0")):
         hw, c = side[stage]
         return hw, hw, c, 3, 3
     return None

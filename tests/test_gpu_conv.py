@@ -101,13 +101,26 @@ def test_resnet_layer_geometry_14x14(torch):
     run_all(torch, X, Wt, G, 3, 3)
 
 
+@pytest.mark.parametrize("C,CO", [(64, 64), (64, 128), (192, 64), (128, 192), (320, 256)])
+def test_channel_counts_that_are_not_multiples_of_128(torch, C, CO):
+    # a tap then fills its last 128-channel block only partly: the missing channels read as zero
+    X, Wt, G = make(20 + C + CO, 3, 9, 10, C, CO, 3, 3)
+    run_all(torch, X, Wt, G, 3, 3)
+
+
+def test_resnet_layer1_geometry_sampled(torch):
+    # 64 -> 64 channels on 56 x 56 images (ResNet-18 layer1), fewer images; whole images checked
+    X, Wt, G = make(31, 8, 56, 56, 64, 64, 3, 3)
+    run_all(torch, X, Wt, G, 3, 3)
+
+
 def test_unsupported_shapes_are_refused(torch):
     ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
     t = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     y = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
     x, w = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7)
-    for shape, co in ((cdl.ConvShape(1, 4, 4, 64, 3, 3), 128), (cdl.ConvShape(1, 4, 4, 128, 2, 2), 128),
-                      (cdl.ConvShape(1, 4, 4, 128, 3, 3), 64)):
+    for shape, co in ((cdl.ConvShape(1, 4, 4, 32, 3, 3), 128), (cdl.ConvShape(1, 4, 4, 128, 2, 2), 128),
+                      (cdl.ConvShape(1, 4, 4, 128, 3, 3), 96)):
         assert cdl.cdl_qconv_workspace_bytes(shape, co) == 0
         assert cdl.cdl_qconv_fwd(t, x, t, co, w, shape, co, None, y, None, ws, 1 << 20, check=False) == -1
 
