@@ -54,6 +54,12 @@ constexpr int kOutWarpBytes = 32 * 128;  // epilogue staging block of one warp: 
 constexpr int kSmemBytes = 232448 - 1024;
 constexpr int kPlanSMs = 148;           // B200: splits are planned for this count so that workspace sizes are fixed
 constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s
+#ifndef CDL_G_TRYWAIT_HINT_NS
+#define CDL_G_TRYWAIT_HINT_NS 20000
+#endif
+// Upper bound, in nanoseconds, on how long one try_wait may keep its thread suspended while the phase is pending:
+// a suspended poller leaves the issue slots of its scheduler to the epilogue warps that share it.
+constexpr unsigned int kTryWaitHintNs = CDL_G_TRYWAIT_HINT_NS;
 
 struct TcParams {
     int I, J, R;            // rows the tiling runs over, output columns, reduced extent of the tiling
@@ -108,10 +114,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kTryWaitHintNs)
         : "memory");
     return ok != 0;
 }
