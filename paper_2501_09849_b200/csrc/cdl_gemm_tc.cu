@@ -877,13 +877,13 @@ int min_exact_splits(int R, long long xmax, long long ymax)
 }
 }  // namespace
 
-// Scratch bytes a product may need: the int32 accumulation buffer of a split run and, when the reduced dimension
-// is long enough that its int32 total could overflow for byte operands of the widest range, the per-split slabs.
+// Scratch bytes a product may need: one int32 slab per split of the reduced dimension (also when the dimension is
+// so long that its int32 total could overflow for byte operands of the widest range and it has to be cut).
 size_t tc_gemm_scratch_bytes(int I, int J, int R)
 {
     Plan p = plan(I, J, R, 1);
     size_t need = 0;
-    if (p.splits > 1) need = (size_t)I * (size_t)J * sizeof(int32_t);
+    if (p.splits > 1) need = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t) * p.splits;
     if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
         p = plan(I, J, R, min_exact_splits(R, 255, 128));
         const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
@@ -897,7 +897,8 @@ size_t tc_gemm_scratch_bytes(int I, int J, int R)
 // bytes, used only when the reduced dimension is split and no int32 output was requested.
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
-                         cudaStream_t stream, const ConvGather *conv, const NextQuant *next, bool accumulate_f)
+                         cudaStream_t stream, const ConvGather *conv, const NextQuant *next, bool accumulate_f,
+                         bool compact_scratch)
 {
     const bool a_mn = conv != nullptr ? conv->transposed != 0 : (X.stride_outer == 1 && X.stride_red != 1);
     const bool b_mn = Y.stride_outer == 1 && Y.stride_red != 1;
@@ -925,7 +926,11 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const bool pair = pl.pair != 0;
     P.TN = TN;
     P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
-    P.slab_rows = wide ? P.tiles_i * pl.tile_rows : 0;
+    // A split reduction with only a float output keeps one slab per split (plain stores, no clear, no atomics in L2)
+    // and sums the slabs in the conversion kernel; with compact_scratch (or an int32 output) the splits add into
+    // one I x J buffer instead.
+    const bool slabs = wide || (splits > 1 && acc_out == nullptr && !compact_scratch);
+    P.slab_rows = slabs ? P.tiles_i * pl.tile_rows : 0;
     P.tiles_j = (J + TN - 1) / TN;
     P.rblocks = (Rt + BR - 1) / BR;
     const int sms = sm_count();
@@ -972,7 +977,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.f_out = f_out;
     P.acc_out = acc_out;
     const long long n_out = (long long)I * J;
-    if (wide) {
+    if (slabs) {
         P.acc_out = static_cast<int32_t *>(scratch);       // slabs: every element is written, nothing to clear
         if (P.acc_out == nullptr) return CDL_ERR_WORKSPACE;
     } else if (splits > 1) {
@@ -1000,12 +1005,12 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const bool out_ok = TN >= 32 && (J & 3) == 0;
     P.tma_f = 0;
     P.tma_acc = 0;
-    if (out_ok && splits == 1 && !wide && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
+    if (out_ok && splits == 1 && !slabs && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
         ok = ok && encode_out_map(&map_f, f_out, (uint64_t)J, (uint64_t)I, true);
         P.tma_f = 1;
     }
     if (out_ok && P.acc_out != nullptr && (reinterpret_cast<uintptr_t>(P.acc_out) & 15u) == 0) {
-        const uint64_t acc_rows = wide ? (uint64_t)splits * (uint64_t)P.slab_rows : (uint64_t)I;
+        const uint64_t acc_rows = slabs ? (uint64_t)splits * (uint64_t)P.slab_rows : (uint64_t)I;
         ok = ok && encode_out_map(&map_acc, P.acc_out, (uint64_t)J, acc_rows, false);
         P.tma_acc = 1;
     }
@@ -1073,9 +1078,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         else index_gemm_tc_kernel<false, false><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
-    if (f_out != nullptr && (splits > 1 || wide)) {
+    if (f_out != nullptr && (splits > 1 || slabs)) {
         const int blocks = (int)((n_out + 255) / 256 < 4096 ? (n_out + 255) / 256 : 4096);
-        if (wide)
+        if (slabs)
             sum_slabs_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, splits, (long long)P.slab_rows * J, f_out, n_out, J, scale, bias, P.f_acc);
         else
             scale_acc_kernel<<<blocks, 256, 0, stream>>>(P.acc_out, f_out, n_out, J, scale, bias, P.f_acc);
@@ -1141,5 +1146,5 @@ extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const 
     GemmOperand X{A_idx, 1, lda, a->lo >= 0, (int)amax};
     GemmOperand Y{G_idx, 1, ldg, false, (int)gmax};
     return launch_index_gemm_tc(X, Y, K, N, M, nullptr, dW, g->q * a->q, nullptr, base + kStaticStatusBytes,
-                                reinterpret_cast<int *>(base), st);
+                                reinterpret_cast<int *>(base), st, nullptr, nullptr, false, true);
 }

@@ -83,6 +83,7 @@ size_t tc_gemm_scratch_bytes(int I, int J, int R);
 int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int J, int R, int32_t *acc_out,
                          float *f_out, float scale, const float *bias, void *scratch, int *status,
                          cudaStream_t stream, const ConvGather *conv = nullptr, const NextQuant *next = nullptr,
-                         bool accumulate_f = false);   // accumulate_f: f_out += result instead of f_out = result
+                         bool accumulate_f = false,    // f_out += result instead of f_out = result
+                         bool compact_scratch = false); // split runs add into one I x J buffer (scratch of I * J * 4 bytes)
 
 }  // namespace cdl
