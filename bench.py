@@ -169,9 +169,28 @@ def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, p
             k["roofline_frac"] = round(max(t_tensor, t_hbm) / (t * 1e-3), 4)
         kern[name] = k
     quant_elems = sum(m["elems"] for m in model.values())
+    # end to end: this form's inputs (w, x, dL/dY) from pinned host memory every step, scalars and dL/dw back
+    pinned = {k: t.cpu().pin_memory() for k, t in cs.input_tensors().items()}
+    out_host = {"scalars": torch.empty(6, dtype=torch.float64).pin_memory(),
+                "dw": torch.empty(cs.n_w, dtype=torch.float32).pin_memory()}
+    e_steps = max(3, min(steps, 10))
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(e_steps):
+        for k, t in cs.input_tensors().items():
+            t.copy_(pinned[k], non_blocking=True)
+        graph.replay()
+        out_host["scalars"].copy_(cs.scalars, non_blocking=True)
+        out_host["dw"].copy_(cs.dw, non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e_steps
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
     status = cdl.cdl_workspace_status(cs.ws, check=False)
     return {"ms_per_step": ms, "value": quant_elems / (ms * 1e-3) / 1e9, "unit": UNIT, "steps": steps,
-            "h2d_bytes_per_step_if_e2e": sum(t.numel() * t.element_size() for t in cs.input_tensors().values()),
+            "e2e": {"value": quant_elems / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e_steps},
             "gpu_launches": steps * cs.kernels_per_step(), "device_status": status, "kernels": kern,
             "note": "same layer through cdl_qconv_fwd/bwd: no stored patch matrix, dX in the layout of x"}
 
