@@ -368,6 +368,26 @@ struct PairOut {
 __device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, f2(-1.0f), a); }   // a - b, one rounding
 
+// hard indices of two elements (see quant_elem for the arithmetic)
+__device__ __forceinline__ void hard_pair(const QuantDev &P, float2 x, int &k0, int &k1)
+{
+    const float q = P.q;
+    float2 c = P.fast_div ? __fmul2_rn(x, f2(P.rq)) : make_float2(__fdiv_rn(x.x, q), __fdiv_rn(x.y, q));
+    c.x = fminf(fmaxf(c.x, P.flo), P.fhi);
+    c.y = fminf(fmaxf(c.y, P.flo), P.fhi);
+    float2 t = __fadd2_rn(c, f2(kMagic));
+    if (P.fast_div) {
+        const float2 df = sub2(c, __fadd2_rn(t, f2(-kMagic)));
+        if (fabsf(df.x) > kTieGuard || fabsf(df.y) > kTieGuard) {
+            c.x = fminf(fmaxf(__fdiv_rn(x.x, q), P.flo), P.fhi);
+            c.y = fminf(fmaxf(__fdiv_rn(x.y, q), P.flo), P.fhi);
+            t = __fadd2_rn(c, f2(kMagic));
+        }
+    }
+    k0 = __float_as_int(t.x) - kMagicBits;
+    k1 = __float_as_int(t.y) - kMagicBits;
+}
+
 template <int MODE, bool RATE>
 __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const float2 *__restrict__ Dtab, float2 x, float2 g)
 {
@@ -578,8 +598,20 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                         }
                     }
                 }
+                if (MODE == MODE_HARD) {
 #pragma unroll
-                for (int c = 0; c < (kPairs ? 0 : 4); ++c) {
+                    for (int h = 0; h < 2; ++h) {
+                        int k0, k1;
+                        hard_pair(P, make_float2(xs[2 * h], xs[2 * h + 1]), k0, k1);
+                        packed |= (((unsigned int)k0 & 0xffu) | (((unsigned int)k1 & 0xffu) << 8)) << (16 * h);
+                        if (do_hist) {
+                            hist_add(hist_s, k0 - P.lo, lane);
+                            hist_add(hist_s, k1 - P.lo, lane);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < ((kPairs || MODE == MODE_HARD) ? 0 : 4); ++c) {
                     const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
                     ys[c] = o.y;
                     gxs[c] = o.gx;
