@@ -260,6 +260,7 @@ int cdl_qlinear_bwd_fp(const float *G, float g_absmax,
                        void *ws, size_t ws_bytes, void *stream);
 size_t cdl_qlinear_bwd_fp_workspace_bytes(int32_t M, int32_t N, int32_t K);
 
+
 /*
  * Weight-gradient product for callers that cannot allocate device memory.  (The paper has no counterpart
  * of this entry point; it is a packaging variant of the dW half of cdl_qlinear_bwd.)
@@ -331,6 +332,15 @@ int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx,
 
 /* Bytes of device workspace cdl_qconv_fwd / cdl_qconv_bwd need; 0 for an unsupported shape. */
 size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out);
+
+/* cdl_qlinear_bwd_fp for a convolutional layer (shapes, layouts and limits of cdl_qconv_bwd): G [dev] N x H x W x C_out floats;
+ * dX [dev] N x H x W x C floats, dW [dev] (R*S*C) x C_out floats, each nullable;
+ * ws [dev]: cdl_qconv_bwd_fp_workspace_bytes(shape, C_out) bytes, 256-byte aligned. */
+int cdl_qconv_bwd_fp(const float *G, float g_absmax, const void *X_idx, const cdl_index_desc *x,
+                     const void *W_idx, int64_t ldw, const cdl_index_desc *w,
+                     const cdl_conv_shape *shape, int32_t C_out, float *dX, float *dW,
+                     void *ws, size_t ws_bytes, void *stream);
+size_t cdl_qconv_bwd_fp_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out);
 
 #define CDL_OP_QLINEAR_FWD 1
 #define CDL_OP_QLINEAR_BWD 2

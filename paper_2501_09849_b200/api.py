@@ -14,7 +14,7 @@ __all__ = [
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
-    "cdl_huffman_lengths", "cdl_qlinear_bwd_fp", "cdl_qlinear_bwd_fp_workspace_bytes", "cdl_qlinear_fwd_next", "cdl_qconv_fwd_next", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
+    "cdl_huffman_lengths", "cdl_qconv_bwd_fp", "cdl_qconv_bwd_fp_workspace_bytes", "cdl_qlinear_bwd_fp", "cdl_qlinear_bwd_fp_workspace_bytes", "cdl_qlinear_fwd_next", "cdl_qconv_fwd_next", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
 
@@ -104,6 +104,10 @@ def load_library():
     lib.cdl_qlinear_bwd_fp.restype = C.c_int
     lib.cdl_qlinear_bwd_fp_workspace_bytes.argtypes = [I32, I32, I32]
     lib.cdl_qlinear_bwd_fp_workspace_bytes.restype = C.c_size_t
+    lib.cdl_qconv_bwd_fp.argtypes = [P, C.c_float, P, P, P, I64, P, P, I32, P, P, P, C.c_size_t, P]
+    lib.cdl_qconv_bwd_fp.restype = C.c_int
+    lib.cdl_qconv_bwd_fp_workspace_bytes.argtypes = [P, I32]
+    lib.cdl_qconv_bwd_fp_workspace_bytes.restype = C.c_size_t
     lib.cdl_huffman_lengths.argtypes = [P, I32, P, P, P, P]
     lib.cdl_huffman_lengths.restype = C.c_int
     lib.cdl_qconv_fwd.argtypes = [P, P, P, I64, P, P, I32, P, P, P, P, C.c_size_t, P]
@@ -229,6 +233,22 @@ def cdl_qlinear_bwd_fp(G, g_absmax, A_idx, lda, a, W_idx, ldw, w, M, N, K, dX=No
                                            C.byref(wc) if wc is not None else None, M, N, K, _ptr(dX), _ptr(dW),
                                            _ptr(ws), ws_bytes, _stream(stream))
     return _check(rc, "cdl_qlinear_bwd_fp", check)
+
+
+def cdl_qconv_bwd_fp_workspace_bytes(shape, C_out):
+    sc = shape._c()
+    return int(load_library().cdl_qconv_bwd_fp_workspace_bytes(C.byref(sc), C_out))
+
+
+def cdl_qconv_bwd_fp(G, g_absmax, X_idx, x, W_idx, ldw, w, shape, C_out, dX=None, dW=None, ws=None, ws_bytes=0,
+                     stream=None, check=True):
+    sc = shape._c()
+    xc = x._c() if x is not None else None
+    wc = w._c() if w is not None else None
+    rc = load_library().cdl_qconv_bwd_fp(_ptr(G), float(g_absmax), _ptr(X_idx), C.byref(xc) if xc is not None else None,
+                                         _ptr(W_idx), ldw, C.byref(wc) if wc is not None else None, C.byref(sc), C_out,
+                                         _ptr(dX), _ptr(dW), _ptr(ws), ws_bytes, _stream(stream))
+    return _check(rc, "cdl_qconv_bwd_fp", check)
 
 
 def cdl_huffman_lengths(hist, nlev, lengths=None, total_bits=None, avg_bits=None, stream=None, check=True):

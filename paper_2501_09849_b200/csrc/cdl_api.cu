@@ -576,4 +576,65 @@ int cdl_qlinear_bwd_fp(const float *G, float g_absmax, const void *A_idx, int64_
     return CDL_OK;
 }
 
+size_t cdl_qconv_bwd_fp_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
+{
+    const size_t base = cdl_qconv_workspace_bytes(shape, C_out);
+    if (base == 0) return 0;
+    const size_t pixels = (size_t)shape->N * shape->H * shape->W;
+    return align256(base) + 2 * align256(pixels * (size_t)C_out);
+}
+
+int cdl_qconv_bwd_fp(const float *G, float g_absmax, const void *X_idx, const cdl_index_desc *x, const void *W_idx,
+                     int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out, float *dX, float *dW,
+                     void *ws, size_t ws_bytes, void *stream)
+{
+    int64_t M;
+    int taps;
+    if (G == nullptr || !conv_dims(shape, C_out, &M, &taps) || (dX == nullptr && dW == nullptr)) return CDL_ERR_ARG;
+    if (!(g_absmax > 0.0f) || !(g_absmax < 1e30f)) return CDL_ERR_RANGE;
+    if (bad_f32_ptr(G)) return CDL_ERR_ALIGN;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_bwd_fp_workspace_bytes(shape, C_out))
+        return CDL_ERR_WORKSPACE;
+    const float q1 = g_absmax / 127.0f, q2 = q1 / 254.0f;
+    const size_t base = align256(cdl_qconv_workspace_bytes(shape, C_out));
+    const size_t plane = align256((size_t)M * (size_t)C_out);
+    char *d1 = static_cast<char *>(ws) + base, *d2 = d1 + plane;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = launch_gradient_digits(G, M, C_out, C_out, q1, q2, d1, d2, st)) != CDL_OK) return rc;
+    // each digit plane is a gradient index tensor of its own step: the first pass stores, the second adds.  The
+    // products share the front of the workspace (status word, split slabs); calls on one stream run in order.
+    for (int pass = 0; pass < 2; ++pass) {
+        const cdl_index_desc gd{pass == 0 ? q1 : q2, -127, 127};
+        const char *dig = pass == 0 ? d1 : d2;
+        if (pass == 0) {
+            rc = cdl_qconv_bwd(dig, &gd, X_idx, x, W_idx, ldw, w, shape, C_out, nullptr, dX, nullptr, dW, ws, base, stream);
+            if (rc != CDL_OK) return rc;
+            continue;
+        }
+        // second digit: same validation already passed; accumulate into the outputs of the first
+        IndexRange rg{false, 127}, rx{false, 0}, rw{false, 0};
+        if (dW != nullptr && (rc = index_range(x, &rx)) != CDL_OK) return rc;
+        if (dX != nullptr && (rc = index_range(w, &rw)) != CDL_OK) return rc;
+        if (dX != nullptr) {
+            ConvGather cg{shape->N, shape->H, shape->W, C_out, shape->R, shape->S, 0, shape->C};
+            GemmOperand X{dig, 0, 0, false, (int)rg.absmax};
+            GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
+            rc = launch_index_gemm_tc(X, Y, (int)M, shape->C, taps * C_out, nullptr, dX, (gd.q * w->q), nullptr,
+                                      static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg, nullptr, true);
+            if (rc != CDL_OK) return rc;
+        }
+        if (dW != nullptr) {
+            ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 1, 0};
+            GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
+            GemmOperand Y{dig, 1, C_out, false, (int)rg.absmax};
+            rc = launch_index_gemm_tc(X, Y, taps * shape->C, C_out, (int)M, nullptr, dW, (gd.q * x->q), nullptr,
+                                      static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg, nullptr, true);
+            if (rc != CDL_OK) return rc;
+        }
+    }
+    return CDL_OK;
+}
+
 }  // extern "C"

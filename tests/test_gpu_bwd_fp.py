@@ -92,3 +92,28 @@ def test_single_outputs_and_saturation(torch):
     t = (oracle.gemm_dw(A, i1.astype(np.int8)).astype(f32) * f32(q1 * f32(a.q)) +
          oracle.gemm_dw(A, i2.astype(np.int8)).astype(f32) * f32(q2 * f32(a.q))).astype(f32)
     assert np.array_equal(dW.cpu().numpy(), t)
+
+
+def test_convolution_form(torch):
+    rng = np.random.default_rng(17)
+    N, H, W, C, CO, R, S = 3, 10, 9, 128, 192, 3, 3
+    X = (rng.integers(0, 16, (N, H, W, C)) * (rng.random((N, H, W, C)) < 0.6)).astype(np.uint8)
+    Wt = rng.integers(-7, 8, (R * S * C, CO)).astype(np.int8)
+    G = (rng.normal(0, 1e-2, (N, H, W, CO)) * rng.lognormal(0, 1, (N, H, W, CO))).astype(f32)
+    absmax = float(np.abs(G).max())
+    x, w = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7)
+    shape = cdl.ConvShape(N, H, W, C, R, S)
+    nb = cdl.cdl_qconv_bwd_fp_workspace_bytes(shape, CO)
+    ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    dX = torch.full((N, H, W, C), 7.0, dtype=torch.float32, device="cuda")
+    dW = torch.full((R * S * C, CO), 7.0, dtype=torch.float32, device="cuda")
+    cdl.cdl_qconv_bwd_fp(dev(torch, G), absmax, dev(torch, X), x, dev(torch, Wt), CO, w, shape, CO, dX, dW, ws, nb)
+    torch.cuda.synchronize()
+    assert cdl.cdl_workspace_status(ws, check=False) == 0
+    i1, i2, q1, q2 = oracle.gradient_digits(G, absmax)
+    I1, I2 = i1.astype(np.int8), i2.astype(np.int8)
+
+    def combine(acc1, acc2, qb):
+        return (acc1.astype(f32) * f32(q1 * f32(qb)) + acc2.astype(f32) * f32(q2 * f32(qb))).astype(f32)
+    assert np.array_equal(dX.cpu().numpy(), combine(oracle.conv_dx(I1, Wt, X.shape, R, S, 1, 1), oracle.conv_dx(I2, Wt, X.shape, R, S, 1, 1), w.q))
+    assert np.array_equal(dW.cpu().numpy(), combine(oracle.conv_dw(X, I1, R, S, 1, 1), oracle.conv_dw(X, I2, R, S, 1, 1), x.q))
