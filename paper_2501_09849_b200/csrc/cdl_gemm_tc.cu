@@ -8,19 +8,26 @@
 //   dX       dA = G W^T    X = G [M,N] (r = n contiguous: K-major)   Y-op = W [K,N] (r = n contiguous: K-major)
 //   dW       dW = A^T G    X = A [M,K] (i = k contiguous: MN-major)  Y-op = G [M,N] (j contiguous: MN-major)
 //
-// Tiling: 128 x TN output tile per work unit (TN in {16..256}), 128 bytes of the reduced dimension per
-// pipeline stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is
-// [rows][128 bytes] with the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or
-// columns outside the matrix are zero-filled by TMA, which makes ragged edges and R tails exact.
-// Warp roles (352 threads): warps 0 and 10 issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs, warps 2-9 run the
-// epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
+// In convolution form the X operand is not a stored matrix: its tiles are gathered from an NHWC index tensor by
+// TMA im2col loads (patch matrix of a stride-1 convolution, or its transpose for dW), see ConvGather.
+//
+// Tiling: 128 x TN output tile per work unit (TN in {16..256}), or a 256 x 256 tile shared by a pair of CTAs
+// (tcgen05 cta_group::2) when the output is wide and tall enough; 128 bytes of the reduced dimension per pipeline
+// stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is [rows][128 bytes] with
+// the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or columns outside the matrix
+// are zero-filled by TMA, which makes ragged edges and R tails exact.
+// Warp roles (352 threads): warps 0 and 10 issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs,
+// warps 2-9 run the epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
 // Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to the warp's
-// swizzled 32 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that
-// global memory sees whole 128-byte lines.  The per-chunk chain (TMEM load, convert, stage, proxy fence, store)
-// is a string of latencies, so two warps share each TMEM lane quarter and take alternate chunks.  Work units are (tile, split of the reduced dimension); with more
-// than one split the staging block is added into an int32 buffer with a TMA bulk reduce-add (integer, so the
+// swizzled 32 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that global
+// memory sees whole 128-byte lines.  The per-chunk chain (TMEM load, convert, stage, proxy fence, store) is a
+// string of latencies, so two warps share each TMEM lane quarter and take alternate chunks.  Work units are
+// (tile, split of the reduced dimension); with more than one split every split stores its partial tile into a
+// slab of its own and a small kernel sums the slabs in int64 (or, when the caller wants the int32 accumulators
+// or scratch is tight, the staging blocks are added into one buffer with TMA bulk reduce-adds: integers, so the
 // result does not depend on order).  Outputs whose pitch or base is not 16-byte aligned, and tiles 16 columns
-// wide, go through the same staging block and are copied out by the warps one row at a time.
+// wide, go through the same staging block and are copied out by the warps one row at a time.  Optional extras
+// of the epilogue: bias, the next layer's hard index, adding to the float output instead of storing it.
 // Every wait is bounded: on expiry the kernel records CDL_ERR_TIMEOUT in the status word and winds down.
 #include <cuda.h>
 
