@@ -16,8 +16,9 @@
 // stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is [rows][128 bytes] with
 // the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or columns outside the matrix
 // are zero-filled by TMA, which makes ragged edges and R tails exact.
-// Warp roles (352 threads): warps 0 and 10 issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs,
-// warps 2-9 run the epilogue; two TMEM accumulators let the epilogue of one tile overlap the MMAs of the next.
+// Warp roles: warp 0 and the last warp issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs, the
+// 8 (or, for products that store more than they load, 16) warps between them run the epilogue; two TMEM
+// accumulators let the epilogue of one tile overlap the MMAs of the next.
 // Epilogue: each thread owns one output row in TMEM; 32 columns at a time are converted, written to the warp's
 // swizzled 32 x 128-byte staging block in shared memory and handed to TMA (bulk tensor store), so that global
 // memory sees whole 128-byte lines.  The per-chunk chain (TMEM load, convert, stage, proxy fence, store) is a
@@ -36,18 +37,20 @@
 namespace cdl {
 namespace {
 
-constexpr int kEpiWarps = 8;             // two per TMEM lane quarter, each taking every other 32-column chunk
+// Epilogue warps per CTA: kEpiWarps / 4 per TMEM lane quarter, taking the 32-column chunks in turn.  Products whose
+// time is the epilogue's (two stages of loads per 256 KB of output) get twice as many, with one chunk in flight each.
+__host__ __device__ constexpr int epi_warps(bool store_heavy) { return store_heavy ? 16 : 8; }
 #ifndef CDL_G_SPLIT_PRODUCER
 #define CDL_G_SPLIT_PRODUCER 1
 #endif
 constexpr bool kSplitProducer = CDL_G_SPLIT_PRODUCER != 0;   // a second TMA warp issues the Y-operand loads
-constexpr int kThreadsTC = 64 + 32 * kEpiWarps + (kSplitProducer ? 32 : 0);
+__host__ __device__ constexpr int threads_tc(bool store_heavy) { return 64 + 32 * epi_warps(store_heavy) + (kSplitProducer ? 32 : 0); }
 // Shared memory is divided between operand stages and epilogue staging blocks (4 KB each, per epilogue warp).
 // Which of the two needs the bytes in flight depends on the shape: a long reduced dimension loads much more than
 // it stores, a short one (two stages per 128 KB of output) the opposite.
-//                                          load-heavy           store-heavy
-//   one CTA per tile  (48 KB stages)       4 stages + 1 block   3 stages + 2 blocks
-//   CTA pair per tile (32 KB stages)       6 stages + 1 block   4 stages + 3 blocks
+//                                          load-heavy                     store-heavy
+//   one CTA per tile  (48 KB stages)       4 stages, 8 epilogue warps     3 stages, 16 epilogue warps
+//   CTA pair per tile (32 KB stages)       6 stages, 8 epilogue warps     4 stages, 16 epilogue warps
 constexpr int kStagesMax = 6;
 constexpr int TM = 128;                 // output rows per tile = UMMA M
 constexpr int BR = 128;                 // bytes (= elements) of the reduced dimension per stage
@@ -204,6 +207,7 @@ __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // AND over the epilogue threads (named barrier 1)
+template <int THREADS>
 __device__ __forceinline__ bool epi_all(bool v)
 {
     uint32_t out;
@@ -213,7 +217,7 @@ __device__ __forceinline__ bool epi_all(bool v)
         "bar.red.and.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(out)
-        : "r"((uint32_t)v), "n"(32 * kEpiWarps)
+        : "r"((uint32_t)v), "n"(THREADS)
         : "memory");
     return out != 0;
 }
@@ -338,7 +342,7 @@ __device__ __forceinline__ int next_hard_index(float y, float q, float rq, float
 // the TMA loads of both CTAs count their bytes on CTA 0's "stage full" barrier; tcgen05.commit multicasts "stage
 // free" and "accumulator full" to both CTAs; the epilogues of both CTAs arrive on CTA 0's "accumulator free" barrier.
 template <bool PAIR, bool STORE_HEAVY>
-__global__ void __launch_bounds__(kThreadsTC, 1)
+__global__ void __launch_bounds__(threads_tc(STORE_HEAVY), 1)
 index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_f, const __grid_constant__ CUtensorMap map_acc,
                      const TcParams P)
@@ -353,9 +357,11 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const int lane = threadIdx.x & 31;
     volatile int *abort_flag = &abort_s;
 
+    constexpr int kEpiWarps = epi_warps(STORE_HEAVY);
+    constexpr int kChunkStep = kEpiWarps / 4;                 // warps per TMEM lane quarter
     constexpr int kStages = PAIR ? (STORE_HEAVY ? 4 : 6) : (STORE_HEAVY ? 3 : 4);
     constexpr int kStageBytes = PAIR ? kStageBytesPair : kStageBytesSingle;
-    constexpr int kOutBlocks = PAIR ? (STORE_HEAVY ? 3 : 1) : (STORE_HEAVY ? 2 : 1);      // per epilogue warp
+    constexpr int kOutBlocks = 1;                             // staging blocks per epilogue warp
     static_assert(kStages * kStageBytes + kEpiWarps * kOutBlocks * kOutWarpBytes + 1024 <= kSmemBytes, "shared memory");
     constexpr int TMU = PAIR ? 2 * TM : TM;                   // rows of a work unit's tile
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // CTA 0 of a pair issues the MMAs
@@ -622,7 +628,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
             // the epilogue warps agree on the outcome, so that either all of them or none release the accumulator
-            if (!epi_all(mbar_wait(tfull_bar(buf), tph, abort_flag))) {
+            if (!epi_all<32 * kEpiWarps>(mbar_wait(tfull_bar(buf), tph, abort_flag))) {
                 failed = true;
                 break;
             }
@@ -692,19 +698,29 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 }
             };
 
-            uint32_t va[32], vb[32];
+            uint32_t va[32];
             int ch = half;
-            if (ch < nchunks) tc_ld32(taddr + (uint32_t)(ch * 32), va);
-            while (ch < nchunks) {
-                tc_wait_ld_pin(va);
-                if (ch + 2 < nchunks) tc_ld32(taddr + (uint32_t)((ch + 2) * 32), vb);
-                emit(va, ch);
-                ch += 2;
-                if (ch < nchunks) {
-                    tc_wait_ld_pin(vb);
-                    if (ch + 2 < nchunks) tc_ld32(taddr + (uint32_t)((ch + 2) * 32), va);
-                    emit(vb, ch);
-                    ch += 2;
+            if (STORE_HEAVY) {
+                // many warps, one chunk in flight each: the other warps hide the TMEM load
+                for (; ch < nchunks; ch += kChunkStep) {
+                    tc_ld32(taddr + (uint32_t)(ch * 32), va);
+                    tc_wait_ld_pin(va);
+                    emit(va, ch);
+                }
+            } else {
+                uint32_t vb[32];
+                if (ch < nchunks) tc_ld32(taddr + (uint32_t)(ch * 32), va);
+                while (ch < nchunks) {
+                    tc_wait_ld_pin(va);
+                    if (ch + kChunkStep < nchunks) tc_ld32(taddr + (uint32_t)((ch + kChunkStep) * 32), vb);
+                    emit(va, ch);
+                    ch += kChunkStep;
+                    if (ch < nchunks) {
+                        tc_wait_ld_pin(vb);
+                        if (ch + kChunkStep < nchunks) tc_ld32(taddr + (uint32_t)((ch + kChunkStep) * 32), va);
+                        emit(vb, ch);
+                        ch += kChunkStep;
+                    }
                 }
             }
             tc_fence_before();
@@ -1043,7 +1059,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         qa[0].val.clusterDim.y = 1;
         qa[0].val.clusterDim.z = 1;
         qc.gridDim = dim3(2 * (sms / 2));
-        qc.blockDim = dim3(kThreadsTC);
+        qc.blockDim = dim3(threads_tc(false));
         qc.dynamicSmemBytes = kSmemBytes;
         qc.attrs = qa;
         qc.numAttrs = 1;
@@ -1068,7 +1084,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         at[0].val.clusterDim.y = 1;
         at[0].val.clusterDim.z = 1;
         cfg.gridDim = dim3(2u * (unsigned)(units < slots ? units : slots));
-        cfg.blockDim = dim3(kThreadsTC);
+        cfg.blockDim = dim3(threads_tc(store_heavy));
         cfg.dynamicSmemBytes = kSmemBytes;
         cfg.stream = stream;
         cfg.attrs = at;
@@ -1081,8 +1097,8 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         }
     } else {
         const int grid = (int)(units < sms ? units : sms);
-        if (store_heavy) index_gemm_tc_kernel<false, true><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
-        else index_gemm_tc_kernel<false, false><<<grid, kThreadsTC, kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        if (store_heavy) index_gemm_tc_kernel<false, true><<<grid, threads_tc(true), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        else index_gemm_tc_kernel<false, false><<<grid, threads_tc(false), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (f_out != nullptr && (splits > 1 || slabs)) {
