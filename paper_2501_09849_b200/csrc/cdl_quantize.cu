@@ -502,6 +502,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) hist_s[k] = 0u;
     if (RATE || do_hist) __syncthreads();
 
+    unsigned int *const hist_l = hist_s + (lane - P.lo * 32);    // this lane's column, indexed by level: hist_l[k * 32]
     double acc_q = 0.0, acc_a = 0.0;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -591,10 +592,11 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                             part_q2 = __ffma2_rn(gg, o.tq, part_q2);
                             part_a2 = __ffma2_rn(gg, o.ta, part_a2);
                         }
-                        packed |= (((unsigned int)o.k0[0] & 0xffu) | (((unsigned int)o.k0[1] & 0xffu) << 8)) << (16 * h);
+                        packed = h == 0 ? __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040)
+                                        : __byte_perm(packed, __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040), 0x5410);
                         if (MODE != MODE_BWD && do_hist) {
-                            hist_add(hist_s, o.k0[0] - P.lo, lane);
-                            hist_add(hist_s, o.k0[1] - P.lo, lane);
+                            atomicAdd(hist_l + o.k0[0] * 32, 1u);
+                            atomicAdd(hist_l + o.k0[1] * 32, 1u);
                         }
                     }
                 }
@@ -603,10 +605,11 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     for (int h = 0; h < 2; ++h) {
                         int k0, k1;
                         hard_pair(P, make_float2(xs[2 * h], xs[2 * h + 1]), k0, k1);
-                        packed |= (((unsigned int)k0 & 0xffu) | (((unsigned int)k1 & 0xffu) << 8)) << (16 * h);
+                        packed = h == 0 ? __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040)
+                                        : __byte_perm(packed, __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040), 0x5410);
                         if (do_hist) {
-                            hist_add(hist_s, k0 - P.lo, lane);
-                            hist_add(hist_s, k1 - P.lo, lane);
+                            atomicAdd(hist_l + k0 * 32, 1u);
+                            atomicAdd(hist_l + k1 * 32, 1u);
                         }
                     }
                 }
