@@ -76,6 +76,7 @@ int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out)
         d.A = (float)(a * 1.4426950408889634074);
         d.c1x2 = (float)(2.0 * al * q * 1.4426950408889634074);
         d.near3 = a > 12.0 ? 1 : 0;
+        d.res1 = a <= 64.0 ? 1 : 0;
         d.a2 = (float)(2.0 * a);
         d.two_aq = (float)(2.0 * al * q);
         d.q2 = (float)(q * q);

@@ -20,6 +20,7 @@ struct QuantDev {
     float A;          // alpha * q^2 * log2(e) = c1 * q
     float c1x2;       // 2 * c1
     int near3;        // alpha q^2 > 12: only the nearest level and its two neighbours carry weight (> 2^-34 relative)
+    int res1;         // alpha q^2 <= 64: theta - k q from one fused multiply-add is accurate enough for the logits
     float a2;         // 2 alpha q^2: dQ_d/dtheta = a2 * Var{J}
     float two_aq;     // 2 alpha q
     float q2;         // q^2

@@ -414,14 +414,23 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
     o.k0[0] = k0;
     o.k0[1] = k1;
     // d = x - kn q as dh + dl
-    const float2 nph = __fmul2_rn(kn, f2(-q));            // -(kn q) rounded
-    const float2 pl = __ffma2_rn(kn, f2(q), nph);         // kn q - RN(kn q), exact
-    const float2 sx = __fadd2_rn(x, nph);
-    const float2 dh = sub2(sx, pl);
-    const float2 dl = sub2(sub2(sx, dh), pl);
     // logits of the two neighbours relative to the nearest level: -alpha q (q -+ 2 d)
-    const float2 w1 = __ffma2_rn(dl, f2(-2.0f), __ffma2_rn(dh, f2(-2.0f), f2(q)));
-    const float2 wm = __ffma2_rn(dl, f2(2.0f), __ffma2_rn(dh, f2(2.0f), f2(q)));
+    float2 dh, w1, wm;
+    if (P.res1) {
+        // moderate alpha q^2: the correctly rounded residual of one fused multiply-add is accurate enough (its 2^-25 q
+        // moves a logit by at most 2 alpha q^2 2^-25 < 4e-6)
+        dh = __ffma2_rn(kn, f2(-q), x);
+        w1 = __ffma2_rn(dh, f2(-2.0f), f2(q));
+        wm = __ffma2_rn(dh, f2(2.0f), f2(q));
+    } else {
+        const float2 nph = __fmul2_rn(kn, f2(-q));            // -(kn q) rounded
+        const float2 pl = __ffma2_rn(kn, f2(q), nph);         // kn q - RN(kn q), exact
+        const float2 sx = __fadd2_rn(x, nph);
+        dh = sub2(sx, pl);
+        const float2 dl = sub2(sub2(sx, dh), pl);
+        w1 = __ffma2_rn(dl, f2(-2.0f), __ffma2_rn(dh, f2(-2.0f), f2(q)));
+        wm = __ffma2_rn(dl, f2(2.0f), __ffma2_rn(dh, f2(2.0f), f2(q)));
+    }
     const float2 a1 = __fmul2_rn(w1, f2(-P.c1)), am = __fmul2_rn(wm, f2(-P.c1));
     float2 e1 = make_float2(ex2_approx(a1.x), ex2_approx(a1.y));
     float2 em = make_float2(ex2_approx(am.x), ex2_approx(am.y));

@@ -339,3 +339,26 @@ def test_soft_histogram_and_its_entropy(torch, q, lo, hi, alpha, window):
     sh2 = torch.zeros(P.nlev, dtype=torch.int64, device="cuda")
     cdl.cdl_quantize_soft(xd, n, P, y, None, None, soft_hist=sh2)
     assert torch.equal(sh, sh2)
+
+
+@pytest.mark.parametrize("aq2", [12.5, 40.0, 63.9, 64.1, 300.0])
+@pytest.mark.parametrize("lo,hi", [(-7, 7), (0, 15)])
+def test_three_level_path_on_both_sides_of_the_residual_switch(torch, aq2, lo, hi):
+    # alpha q^2 <= 64 takes theta - k q from one fused multiply-add, above it as a two-float sum: both must hold the
+    # tolerance where the logits are most sensitive -- right at and next to the midpoints between levels, at the
+    # largest |k| -- and for large theta far outside the alphabet
+    q = 0.37
+    alpha = aq2 / (q * q)
+    rng = np.random.default_rng(int(aq2 * 10) + hi)
+    mids = (np.arange(lo, hi) + 0.5) * q
+    x = np.concatenate([mids, mids * (1 + 1e-6), mids * (1 - 1e-6), mids + 1e-4 * q, mids - 1e-4 * q,
+                        rng.uniform((lo - 1) * q, (hi + 1) * q, 4000), [1e3, -1e3, 0.0, hi * q, lo * q]]).astype(f32)
+    x = np.resize(x, 8192)
+    g = rng.normal(0, 1, x.size).astype(f32)
+    P = cdl.QuantParams(q, lo, hi, alpha)
+    y, idx, hist = run_soft(torch, x, P, True)
+    ref_idx, _ = oracle.hard(x, f32(q), lo, hi)
+    assert np.array_equal(idx, ref_idx)
+    assert_soft_close(y, oracle.soft(x, f32(q), lo, hi, f32(alpha), 0), q)
+    gx, gq, ga = run_backward(torch, x, g, P)
+    assert_backward_close(gx, gq, ga, oracle.backward(x, g, f32(q), lo, hi, f32(alpha), 0), g, q, alpha)
