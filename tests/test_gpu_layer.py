@@ -285,3 +285,40 @@ def test_step_replayed_from_a_cuda_graph_equals_the_step_launched_call_by_call(t
         assert torch.equal(step.scalars[:2], eager_scalars[:2])
         assert torch.allclose(step.scalars[2:], eager_scalars[2:], rtol=1e-9, atol=1e-12)
     assert cdl.cdl_workspace_status(step.ws, check=False) == 0
+
+
+def test_convolution_form_step_graph_equals_call_by_call(torch):
+    # the three-stream recording of the step in convolution form has its own dependencies (the forward product waits
+    # for X_idx, the activation backward pass for the data gradient): it must write what the serial step writes
+    from paper_2501_09849_b200.layer import CdlLayerStep
+    n_img, H, W, C, CO = 4, 8, 8, 128, 128
+    M, K = n_img * H * W, 9 * C
+    wq = inputs.Quantizer(0.02, -7, 7, 80.0, 0.01, 0)
+    xq = inputs.Quantizer(0.25, 0, 15, 300.0, 0.01, 5)
+    step = CdlLayerStep(torch, M, K, CO, M * C, wq, xq, q_g=1e-3, conv=cdl.ConvShape(n_img, H, W, C, 3, 3))
+    step.w.copy_(dev(torch, inputs.normal((K * CO,), 0.05, seed=6, stream=1)))
+    step.x.copy_(dev(torch, np.maximum(inputs.normal((M * C,), 1.0, seed=6, stream=2), 0).astype(f32)))
+    step.dY.copy_(dev(torch, inputs.normal((M, CO), 3e-2, seed=6, stream=3)))
+    outs = ("w_soft", "W_idx", "x_soft", "X_idx", "hist_w", "hist_x", "prob_w", "prob_x", "Y", "G_idx", "gx_in", "dW",
+            "dx", "dw")
+    step.run()
+    torch.cuda.synchronize()
+    eager = {k: getattr(step, k).clone() for k in outs}
+    eager_scalars = step.scalars.clone()
+    # the forward output and the data gradient of the serial step against the oracle's convolution
+    Xi, Wi, Gi = (eager[k].cpu().numpy() for k in ("X_idx", "W_idx", "G_idx"))
+    acc = oracle.conv_fwd(Xi.reshape(n_img, H, W, C), Wi, 3, 3, 1, 1).reshape(M, CO)
+    assert np.array_equal(eager["Y"].cpu().numpy(), scaled(acc, xq.q, wq.q))
+    accx = oracle.conv_dx(Gi.reshape(n_img, H, W, CO), Wi, (n_img, H, W, C), 3, 3, 1, 1).reshape(-1)
+    assert np.array_equal(eager["gx_in"].cpu().numpy(), scaled(accx, 1e-3, wq.q))
+    graph = step.capture()
+    for _ in range(2):
+        for k in outs:
+            getattr(step, k).zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for k in outs:
+            assert torch.equal(getattr(step, k), eager[k]), k
+        assert torch.equal(step.scalars[:2], eager_scalars[:2])
+        assert torch.allclose(step.scalars[2:], eager_scalars[2:], rtol=1e-9, atol=1e-12)
+    assert cdl.cdl_workspace_status(step.ws, check=False) == 0
