@@ -318,6 +318,10 @@ int cdl_qlinear_fwd_next(const void *A_idx, int64_t lda, const cdl_index_desc *a
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float scale = (a->q * w->q);
+    // few output channels: an HBM-bound streaming product, served by the dp4a kernels
+    if (nq.idx_out == nullptr && skinny_fwd_ok(M, N, K) && !overflow_risk(K, ra, rw) &&
+        (reinterpret_cast<uintptr_t>(acc_out) & 15u) == 0 && (reinterpret_cast<uintptr_t>(y_out) & 15u) == 0)
+        return launch_skinny_fwd(A_idx, lda, ra.is_unsigned, W_idx, ldw, M, N, K, acc_out, y_out, scale, bias, st);
     GemmOperand X{A_idx, lda, 1, ra.is_unsigned, (int)ra.absmax};
     GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
     return launch_index_gemm_tc(X, Y, M, N, K, acc_out, y_out, scale, bias, static_cast<char *>(ws) + kStatusBytes,
@@ -362,7 +366,11 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
     if (dWacc != nullptr && overflow_risk(M, ra, rg)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (want_dx) {
+    if (want_dx && skinny_dx_ok(M, N, K) && !overflow_risk(N, rg, rw)) {
+        // few reduced channels: HBM-bound, streamed by the dp4a kernel
+        rc = launch_skinny_dx(G_idx, ldg, W_idx, ldw, M, N, K, dXacc, dX, (g->q * w->q), false, st);
+        if (rc != CDL_OK) return rc;
+    } else if (want_dx) {
         // dX[m,k] = sum_n G[m,n] W[k,n]
         GemmOperand X{G_idx, ldg, 1, false, (int)rg.absmax};
         GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};

@@ -54,6 +54,14 @@ struct GemmOperand {
     int absmax;             // bound on |entry| (from the operand's declared index range)
 };
 
+// Streaming dp4a kernels for products with few output channels (N in {4, 8, 16, 32}); see cdl_gemm_skinny.cu.
+bool skinny_fwd_ok(int M, int N, int K);
+bool skinny_dx_ok(int M, int N, int K);
+int launch_skinny_fwd(const void *A, long long lda, bool a_unsigned, const void *W, long long ldw, int M, int N, int K,
+                      int32_t *acc_out, float *y_out, float scale, const float *bias, cudaStream_t stream);
+int launch_skinny_dx(const void *G, long long ldg, const void *W, long long ldw, int M, int N, int K, int32_t *acc_out,
+                     float *f_out, float scale, bool accumulate, cudaStream_t stream);
+
 int launch_gradient_digits(const float *g, long long rows, int cols, int ld, float q1, float q2, void *d1, void *d2,
                            cudaStream_t stream);
 int launch_huffman(const unsigned long long *hist, int nlev, unsigned char *lengths, unsigned long long *total_bits,
