@@ -498,14 +498,25 @@ def run_gemm(args):
         for name, fn in calls.items():
             for t in sets:
                 fn(t)
-            reps = max(4, min(40, args.steps))
+            # one pass over the buffer sets recorded as a graph: calls of a few microseconds would otherwise be
+            # timed by the host's launch path, not by the device
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    for t in sets:
+                        fn(t)
+            rounds = max(2, min(40, args.steps) // nset)
+            graph.replay()
+            torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            for i in range(reps):
-                fn(sets[i % nset])
+            for i in range(rounds):
+                graph.replay()
             e1.record(stream)
             e1.synchronize()
-            ms = e0.elapsed_time(e1) / reps
+            ms = e0.elapsed_time(e1) / (rounds * nset)
             ops = 2.0 * M * K * N
             t_tensor, t_hbm = ops / (int8_tops * 1e12), bytes_[name] / (hbm * 1e9)
             row[name] = {"ms": round(ms, 5), "int8_TOPS": round(ops / (ms * 1e-3) / 1e12, 1),

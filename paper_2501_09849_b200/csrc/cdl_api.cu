@@ -250,7 +250,10 @@ size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
         case CDL_OP_QLINEAR_FWD: return kStatusBytes + tc_gemm_scratch_bytes(M, N, K);
         case CDL_OP_QLINEAR_BWD: {
             const size_t dx = tc_gemm_scratch_bytes(M, K, N), dw = tc_gemm_scratch_bytes(K, N, M);
-            return kStatusBytes + (dx > dw ? dx : dw);
+            size_t need = dx > dw ? dx : dw;
+            const size_t skinny = skinny_dw_ok(M, N, K) ? skinny_dw_scratch_bytes(N, K) : 0;
+            if (skinny > need) need = skinny;
+            return kStatusBytes + need;
         }
         default: return 0;
     }
@@ -378,7 +381,11 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
                                   static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st);
         if (rc != CDL_OK) return rc;
     }
-    if (want_dw) {
+    if (want_dw && skinny_dw_ok(M, N, K) && !overflow_risk(M, ra, rg)) {
+        rc = launch_skinny_dw(A_idx, lda, ra.is_unsigned, G_idx, ldg, M, N, K, dWacc, dW, (g->q * a->q), false,
+                              static_cast<char *>(ws) + kStatusBytes, st);
+        if (rc != CDL_OK) return rc;
+    } else if (want_dw) {
         // dW[k,n] = sum_m A[m,k] G[m,n]
         GemmOperand X{A_idx, 1, lda, ra.is_unsigned, (int)ra.absmax};
         GemmOperand Y{G_idx, 1, ldg, false, (int)rg.absmax};

@@ -156,6 +156,181 @@ skinny_dx_kernel(const signed char *__restrict__ G, long long ldg, const signed 
     }
 }
 
+// ------------------------------------------------------------------------------------------------ dW
+// dW[k, n] = sum_m A[m, k] G[m, n]: the contraction runs over rows, so both operands are needed with four
+// consecutive rows of one column in a word.  A warp works alone on jobs of 32 rows x (16 MT columns of A): it reads
+// the rows with coalesced 4-byte loads, four rows at a time, transposes 4 x 4 byte blocks in registers (byte
+// permutes), parks the words in its own shared-memory patch and multiplies from there with the warp-level int8
+// matrix instruction (m16n8k32: 16 columns of A x 8 of G x 32 rows), sums in registers across its jobs.  The next
+// job's loads are in flight during the multiplication.  At the end the warps of a CTA add their sums in shared
+// memory and the CTA adds them to the int32 result with coalesced reductions; the last CTA to finish converts.
+constexpr int kDwWarps = 12;
+
+__device__ __forceinline__ void transpose4x4(unsigned int r0, unsigned int r1, unsigned int r2, unsigned int r3,
+                                             unsigned int (&o)[4])
+{
+    const unsigned int t0 = __byte_perm(r0, r1, 0x5140), t1 = __byte_perm(r2, r3, 0x5140);
+    const unsigned int t2 = __byte_perm(r0, r1, 0x7362), t3 = __byte_perm(r2, r3, 0x7362);
+    o[0] = __byte_perm(t0, t1, 0x5410);
+    o[1] = __byte_perm(t0, t1, 0x7632);
+    o[2] = __byte_perm(t2, t3, 0x5410);
+    o[3] = __byte_perm(t2, t3, 0x7632);
+}
+
+// D (16 x 8, int32) += A (16 x 32 bytes, row-major fragment) B (32 x 8 int8, column fragment)
+template <bool A_UNSIGNED>
+__device__ __forceinline__ void mma_k32(int (&d)[4], unsigned int a0, unsigned int a1, unsigned int a2, unsigned int a3,
+                                        unsigned int b0, unsigned int b1)
+{
+    if (A_UNSIGNED)
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct DwTail {                 // what the last CTA to finish does with the sums
+    float *f_out;
+    float scale;
+    int accumulate;
+    unsigned int *counter;      // zeroed together with the sums
+};
+
+template <int N, int MT> struct DwGeom {
+    static constexpr int NT = N >= 8 ? N / 8 : 1;           // 8-column tiles of G
+    static constexpr int NP = NT * 8;
+    static constexpr int KSL = 16 * MT;                     // columns of A per job
+    static constexpr int KS = (KSL & 31) == 8 ? KSL : ((KSL + 23) / 32 * 32 + 8);   // patch row strides in words,
+    static constexpr int GS = NP == 8 ? 8 : 40;                                     // = 8 mod 32: conflict-free
+    static constexpr int GI = (2 * N + 31) / 32;            // 4 x 4 blocks of G per lane and job
+    static constexpr int patch_words = 8 * (KS + GS);
+    static constexpr size_t smem_bytes = ((size_t)kDwWarps * patch_words + (size_t)KSL * NP) * 4;
+};
+
+template <int N, int MT, bool A_UNSIGNED>
+__global__ void __launch_bounds__(kDwWarps * 32, 1)
+skinny_dw_kernel(const unsigned char *__restrict__ A, long long lda, const signed char *__restrict__ G, long long ldg,
+                 int M, int K, int S, int32_t *__restrict__ acc_out, DwTail tail)
+{
+    using Geo = DwGeom<N, MT>;
+    constexpr int NT = Geo::NT, NP = Geo::NP, KSL = Geo::KSL, KS = Geo::KS, GS = Geo::GS, GI = Geo::GI;
+    extern __shared__ __align__(16) unsigned int smem_dw[];
+    __shared__ int is_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = lane & 3, g = lane >> 2;
+    unsigned int *At = smem_dw + warp * Geo::patch_words;       // [8][KS]: word (m4, k) = A[4 m4 .. 4 m4 + 3][k0 + k]
+    unsigned int *Gt = At + 8 * KS;                             // [8][GS]
+    int *red = reinterpret_cast<int *>(smem_dw + kDwWarps * Geo::patch_words);      // [KSL][NP]
+    for (int i = threadIdx.x; i < KSL * NP; i += kDwWarps * 32) red[i] = 0;
+    for (int i = lane; i < 8 * GS; i += 32) Gt[i] = 0u;         // columns N .. NP - 1 stay zero
+    const int slice = blockIdx.x % S, k0 = slice * KSL;
+    const long long cta_in_slice = blockIdx.x / S, ctas_per_slice = gridDim.x / S;
+    const long long ngroups = ((long long)M + 31) / 32;
+    const long long gstride = ctas_per_slice * kDwWarps;
+    int acc[MT][NT][4];
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[i][j][c] = 0;
+    unsigned int ra[MT][4], rg[GI][4];
+
+    auto fetch = [&](long long grp) {
+        const long long m0 = grp * 32;
+#pragma unroll
+        for (int j = 0; j < MT; ++j) {                          // 8 x 4 MT blocks: MT per lane
+            const int i = lane + 32 * j;
+            const int m4 = i / (4 * MT), k4 = i % (4 * MT);
+            const int k = k0 + 4 * k4;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const long long m = m0 + 4 * m4 + b;
+                ra[j][b] = (m < M && k < K) ? __ldg(reinterpret_cast<const unsigned int *>(A + m * lda + k)) : 0u;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < GI; ++j) {                          // 8 x N / 4 blocks
+            const int i = lane + 32 * j;
+            const int m4 = i / (N / 4), n4 = i % (N / 4);
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const long long m = m0 + 4 * m4 + b;
+                rg[j][b] = (i < 2 * N && m < M) ? __ldg(reinterpret_cast<const unsigned int *>(G + m * ldg + 4 * n4)) : 0u;
+            }
+        }
+    };
+
+    long long grp = cta_in_slice * kDwWarps + warp;
+    if (grp < ngroups) fetch(grp);
+    __syncthreads();                                            // red and the patches are initialised
+    for (; grp < ngroups; grp += gstride) {
+#pragma unroll
+        for (int j = 0; j < MT; ++j) {
+            const int i = lane + 32 * j;
+            const int m4 = i / (4 * MT), k4 = i % (4 * MT);
+            unsigned int o[4];
+            transpose4x4(ra[j][0], ra[j][1], ra[j][2], ra[j][3], o);
+            *reinterpret_cast<uint4 *>(At + m4 * KS + 4 * k4) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+#pragma unroll
+        for (int j = 0; j < GI; ++j) {
+            const int i = lane + 32 * j;
+            if (i < 2 * N) {
+                const int m4 = i / (N / 4), n4 = i % (N / 4);
+                unsigned int o[4];
+                transpose4x4(rg[j][0], rg[j][1], rg[j][2], rg[j][3], o);
+                *reinterpret_cast<uint4 *>(Gt + m4 * GS + 4 * n4) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        __syncwarp();
+        if (grp + gstride < ngroups) fetch(grp + gstride);      // in flight while this job is multiplied
+        unsigned int b0[NT], b1[NT];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            b0[j] = Gt[t * GS + 8 * j + g];
+            b1[j] = Gt[(t + 4) * GS + 8 * j + g];
+        }
+#pragma unroll
+        for (int i = 0; i < MT; ++i) {
+            const unsigned int a0 = At[t * KS + 16 * i + g], a1 = At[t * KS + 16 * i + g + 8];
+            const unsigned int a2 = At[(t + 4) * KS + 16 * i + g], a3 = At[(t + 4) * KS + 16 * i + g + 8];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma_k32<A_UNSIGNED>(acc[i][j], a0, a1, a2, a3, b0[j], b1[j]);
+        }
+        __syncwarp();                                           // the patch is free for the next job
+    }
+    // warps -> CTA (shared-memory adds) -> result (coalesced reductions)
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int row = 16 * i + g + (c >= 2 ? 8 : 0), col = 8 * j + 2 * t + (c & 1);
+                if (acc[i][j][c] != 0) atomicAdd(red + row * NP + col, acc[i][j][c]);
+            }
+    __syncthreads();
+    for (int i = threadIdx.x; i < KSL * N; i += kDwWarps * 32) {
+        const int row = i / N, col = i % N;
+        const int v = red[row * NP + col];
+        if (v != 0 && k0 + row < K) atomicAdd(acc_out + (long long)(k0 + row) * N + col, v);
+    }
+    if (tail.f_out == nullptr) return;
+    // the last CTA to get here turns the sums into floats
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(tail.counter, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int i = threadIdx.x; i < K * N; i += kDwWarps * 32) {
+        const float v = __fmul_rn((float)__ldcg(acc_out + i), tail.scale);
+        tail.f_out[i] = tail.accumulate ? __fadd_rn(tail.f_out[i], v) : v;
+    }
+}
+
 int grid_for(long long work_items)
 {
     const int sms = sm_count();
@@ -212,6 +387,77 @@ int launch_dx_nw(const void *G, long long ldg, const void *W, long long ldw, int
 }
 
 }  // namespace
+
+template <int N, int MT, bool A_UNSIGNED>
+int launch_dw_t(const unsigned char *a, long long lda, const signed char *g, long long ldg, int M, int K, int32_t *acc,
+                const DwTail &tail, cudaStream_t stream)
+{
+    using Geo = DwGeom<N, MT>;
+    const int sms = sm_count();
+    if (sms <= 0) return CDL_ERR_LAUNCH;
+    const int S = (K + Geo::KSL - 1) / Geo::KSL;                 // column slices of A
+    if (S > sms) return CDL_ERR_ARG;
+    if (cudaFuncSetAttribute(skinny_dw_kernel<N, MT, A_UNSIGNED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Geo::smem_bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    const long long ngroups = ((long long)M + 31) / 32;
+    long long per_slice = sms / S;                               // CTAs that share a slice: one CTA per SM in all
+    const long long useful = (ngroups + kDwWarps - 1) / kDwWarps;
+    if (per_slice > useful) per_slice = useful;
+    const int grid = (int)(per_slice * S);
+    skinny_dw_kernel<N, MT, A_UNSIGNED><<<grid, kDwWarps * 32, Geo::smem_bytes, stream>>>(a, lda, g, ldg, M, K, S, acc, tail);
+    return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
+}
+
+template <int N, int MT>
+int launch_dw_n(const void *A, long long lda, bool a_unsigned, const void *G, long long ldg, int M, int K, int32_t *acc,
+                const DwTail &tail, cudaStream_t stream)
+{
+    const unsigned char *a = static_cast<const unsigned char *>(A);
+    const signed char *g = static_cast<const signed char *>(G);
+    return a_unsigned ? launch_dw_t<N, MT, true>(a, lda, g, ldg, M, K, acc, tail, stream)
+                      : launch_dw_t<N, MT, false>(a, lda, g, ldg, M, K, acc, tail, stream);
+}
+
+bool skinny_dw_ok(int M, int N, int K)
+{
+    (void)M;
+    return (N == 4 || N == 8 || N == 16 || N == 32) && (K % 4) == 0 && K <= 2048;
+}
+
+size_t skinny_dw_scratch_bytes(int N, int K) { return ((size_t)K * N + 4) * sizeof(int32_t); }
+
+// dW (K x N floats and / or int32) from A (M x K bytes) and G (M x N int8); scratch: skinny_dw_scratch_bytes
+int launch_skinny_dw(const void *A, long long lda, bool a_unsigned, const void *G, long long ldg, int M, int N, int K,
+                     int32_t *acc_out, float *f_out, float scale, bool accumulate, void *scratch, cudaStream_t stream)
+{
+    if (scratch == nullptr) return CDL_ERR_WORKSPACE;
+    int32_t *sums = static_cast<int32_t *>(scratch);
+    DwTail tail{f_out, scale, accumulate ? 1 : 0, reinterpret_cast<unsigned int *>(sums + (size_t)K * N)};
+    int32_t *acc = acc_out != nullptr ? acc_out : sums;
+    // the sums and the CTA counter behind them start at zero
+    const size_t nsum = (size_t)K * N * sizeof(int32_t);
+    cudaError_t e;
+    if (acc_out == nullptr) {
+        e = cudaMemsetAsync(sums, 0, nsum + 4 * sizeof(int32_t), stream);
+    } else {
+        e = cudaMemsetAsync(acc_out, 0, nsum, stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(tail.counter, 0, 4 * sizeof(int32_t), stream);
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    switch (N) {
+        case 4: return launch_dw_n<4, 9>(A, lda, a_unsigned, G, ldg, M, K, acc, tail, stream);
+        case 8: return launch_dw_n<8, 9>(A, lda, a_unsigned, G, ldg, M, K, acc, tail, stream);
+        case 16: return launch_dw_n<16, 9>(A, lda, a_unsigned, G, ldg, M, K, acc, tail, stream);
+        case 32: return launch_dw_n<32, 4>(A, lda, a_unsigned, G, ldg, M, K, acc, tail, stream);
+        default: return CDL_ERR_ARG;
+    }
+}
 
 bool skinny_fwd_ok(int M, int N, int K)
 {

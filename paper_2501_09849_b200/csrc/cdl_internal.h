@@ -57,6 +57,10 @@ struct GemmOperand {
 // Streaming dp4a kernels for products with few output channels (N in {4, 8, 16, 32}); see cdl_gemm_skinny.cu.
 bool skinny_fwd_ok(int M, int N, int K);
 bool skinny_dx_ok(int M, int N, int K);
+bool skinny_dw_ok(int M, int N, int K);
+size_t skinny_dw_scratch_bytes(int N, int K);
+int launch_skinny_dw(const void *A, long long lda, bool a_unsigned, const void *G, long long ldg, int M, int N, int K,
+                     int32_t *acc_out, float *f_out, float scale, bool accumulate, void *scratch, cudaStream_t stream);
 int launch_skinny_fwd(const void *A, long long lda, bool a_unsigned, const void *W, long long ldw, int M, int N, int K,
                       int32_t *acc_out, float *y_out, float scale, const float *bias, cudaStream_t stream);
 int launch_skinny_dx(const void *G, long long ldg, const void *W, long long ldw, int M, int N, int K, int32_t *acc_out,
