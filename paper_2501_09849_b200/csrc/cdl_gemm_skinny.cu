@@ -1,12 +1,12 @@
 // Layer products whose weight matrix has few output channels (N <= 32: the 16-channel layers of CIFAR ResNets).
 // With K * N of a few thousand there are only ~10 multiply-adds per byte moved, so these products are bound by
-// HBM, not by arithmetic, and a 128-row tensor-core tile spends its time on hand-shakes: here they are streaming
-// kernels on the integer dot-product instruction (dp4a, four byte products per lane and instruction), exact in
-// int32 like the tensor-core path and with the same float epilogue.
-//   forward  Y[m, :]  = A[m, :] W        one thread per row: its A row in registers, W packed four k per word in
-//                                        shared memory and read as broadcasts
-//   dX       dA[m, :] = G[m, :] W^T      one warp per 32 rows: lane = output column (coalesced 128-byte stores), its
-//                                        W rows in registers, the G rows broadcast by shuffles
+// HBM, not by arithmetic, and a 128-row tile fed by TMA spends its time on hand-shakes: here they are streaming
+// kernels in which every warp works alone, rows go from global memory straight into the fragments of the
+// warp-level int8 matrix instruction (m16n8k32), exact in int32 like the tile path and with the same float epilogue.
+//   forward  Y[m, :]  = A[m, :] W        a warp per 16 rows, W fragments in shared memory
+//   dX       dA[m, :] = G[m, :] W^T      a warp per 16 rows, 16-byte stores; a dp4a kernel (lane = output column)
+//                                        covers K that is not a multiple of 16
+//   dW       dW       = A^T G            a warp per 32 rows, operands transposed in registers
 #include "cdl_internal.h"
 
 namespace cdl {
@@ -23,79 +23,138 @@ __device__ __forceinline__ int dot4(unsigned int a, unsigned int b, int c)
     return d;
 }
 
+// D (16 x 8, int32) += A (16 x 32 bytes, row-major fragment) B (32 x 8 int8, column fragment)
+template <bool A_UNSIGNED>
+__device__ __forceinline__ void mma_k32(int (&d)[4], unsigned int a0, unsigned int a1, unsigned int a2, unsigned int a3,
+                                        unsigned int b0, unsigned int b1)
+{
+    if (A_UNSIGNED)
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // ------------------------------------------------------------------------------------------------ forward
-// Wp[k4 * N + n] = bytes W[4 k4 .. 4 k4 + 3][n]; K a multiple of 16, N a multiple of 4, N <= 32.
-// STAGED: a warp first copies its 32 rows of A into shared memory with coalesced 16-byte loads and every lane then
-// reads its own row from there; otherwise every lane reads its row straight from global memory (rows too long to
-// stage for eight warps).
-template <int N, bool A_UNSIGNED, bool STAGED>
+// A warp takes 16 rows at a time: lane (g, t) = (lane / 4, lane % 4) reads 16 consecutive bytes of rows g and g + 8
+// per 64 columns, which are the A fragments of two m16n8k32 steps once the k positions of a step are taken in the
+// order the loads deliver them; the fragments of W are laid out in shared memory for the same order.  Output columns
+// are dealt to the 8-column tiles so that a lane ends up with 2 N / 8 consecutive columns of a row (one or two
+// 16-byte stores; a quad writes the whole row).  K a multiple of 16: after the 64-column chunks one 32- and / or one
+// 16-column piece (8- and 4-byte loads).
+__device__ __forceinline__ int fwd_kbase(int s, int t, int h, int c64, int rest)
+{
+    if (s < 2 * c64) return 64 * (s >> 1) + 16 * t + 8 * (s & 1) + 4 * h;
+    const int base = 64 * c64, r = s - 2 * c64;
+    if (rest >= 32 && r == 0) return base + 8 * t + 4 * h;
+    return h == 0 ? base + (rest >= 32 ? 32 : 0) + 4 * t : -1;     // the 16-column tail: upper half of the step empty
+}
+
+template <int N, bool A_UNSIGNED>
 __global__ void __launch_bounds__(kSkinnyThreads)
 skinny_fwd_kernel(const unsigned char *__restrict__ A, long long lda, const signed char *__restrict__ W, long long ldw,
                   int M, int K, int32_t *__restrict__ acc_out, float *__restrict__ y_out, float scale,
                   const float *__restrict__ bias)
 {
-    extern __shared__ __align__(16) unsigned int Wp[];
-    const int k4n = K / 4;
-    for (int i = threadIdx.x; i < k4n * N; i += kSkinnyThreads) {
-        const int k4 = i / N, n = i - k4 * N;
+    constexpr int NT = N >= 8 ? N / 8 : 1;
+    extern __shared__ __align__(16) unsigned int Bf[];          // [step][tile][half][lane]
+    const int c64 = K >> 6, rest = K & 63;
+    const int nsteps = 2 * c64 + (rest >= 32 ? 1 : 0) + ((rest & 31) == 16 ? 1 : 0);
+    for (int i = threadIdx.x; i < nsteps * NT * 64; i += kSkinnyThreads) {
+        const int ln = i & 31, h = (i >> 5) & 1, sj = i >> 6, j = sj % NT, s = sj / NT;
+        const int kb = fwd_kbase(s, ln & 3, h, c64, rest);
+        const int gg = ln >> 2;
+        const int col = N >= 8 ? (gg >> 1) * (2 * NT) + 2 * j + (gg & 1) : gg;
         unsigned int w = 0;
+        if (kb >= 0 && col < N) {
 #pragma unroll
-        for (int b = 0; b < 4; ++b) w |= (unsigned int)(unsigned char)W[(long long)(4 * k4 + b) * ldw + n] << (8 * b);
-        Wp[i] = w;
+            for (int b = 0; b < 4; ++b) w |= (unsigned int)(unsigned char)W[(long long)(kb + b) * ldw + col] << (8 * b);
+        }
+        Bf[i] = w;
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31, warp_in_cta = threadIdx.x >> 5;
-    const int k16 = K / 16;
-    uint4 *stage = reinterpret_cast<uint4 *>(Wp + k4n * N) + (size_t)warp_in_cta * 32 * k16;      // [32 rows][K / 16]
-    const long long stride = (long long)gridDim.x * kSkinnyThreads;
-    // whole warps iterate together (the staging copy is a warp's job); rows past M are skipped at the end
-    for (long long m0 = (long long)blockIdx.x * kSkinnyThreads + warp_in_cta * 32; m0 < M; m0 += stride) {
-        const long long m = m0 + lane;
-        if (STAGED) {
-            __syncwarp();
-            for (int i = lane; i < 32 * k16; i += 32) {
-                const int r = i / k16, c = i - r * k16;
-                if (m0 + r < M) stage[i] = __ldcs(reinterpret_cast<const uint4 *>(A + (m0 + r) * lda) + c);
-            }
-            __syncwarp();
+    const int lane = threadIdx.x & 31, t = lane & 3, g = lane >> 2;
+    const long long warp = ((long long)blockIdx.x * kSkinnyThreads + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * kSkinnyThreads) >> 5;
+    const long long ntiles = ((long long)M + 15) / 16;
+    const int cb = N >= 8 ? t * 2 * NT : 2 * t;                 // this lane's first output column
+    float bv[2 * NT];
+#pragma unroll
+    for (int q = 0; q < 2 * NT; ++q) bv[q] = (bias != nullptr && cb + q < N) ? bias[cb + q] : 0.0f;
+    for (long long tile = warp; tile < ntiles; tile += nwarps) {
+        __syncwarp();                                           // the matrix instruction wants the whole warp
+        const long long r0 = tile * 16 + g, r1 = r0 + 8;
+        const bool v0 = r0 < M, v1 = r1 < M;
+        const unsigned char *p0 = A + r0 * lda, *p1 = A + r1 * lda;
+        int acc[NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[j][c] = 0;
+        const unsigned int *bf = Bf + lane;
+#pragma unroll 2
+        for (int c = 0; c < c64; ++c) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            const uint4 x0 = v0 ? __ldcs(reinterpret_cast<const uint4 *>(p0 + 64 * c + 16 * t)) : z;
+            const uint4 x1 = v1 ? __ldcs(reinterpret_cast<const uint4 *>(p1 + 64 * c + 16 * t)) : z;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma_k32<A_UNSIGNED>(acc[j], x0.x, x1.x, x0.y, x1.y, bf[j * 64], bf[j * 64 + 32]);
+            bf += NT * 64;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma_k32<A_UNSIGNED>(acc[j], x0.z, x1.z, x0.w, x1.w, bf[j * 64], bf[j * 64 + 32]);
+            bf += NT * 64;
         }
-        if (m >= M) continue;
-        int acc[N];
+        int kb = 64 * c64;
+        if (rest >= 32) {
+            const uint2 z = make_uint2(0u, 0u);
+            const uint2 x0 = v0 ? __ldcs(reinterpret_cast<const uint2 *>(p0 + kb + 8 * t)) : z;
+            const uint2 x1 = v1 ? __ldcs(reinterpret_cast<const uint2 *>(p1 + kb + 8 * t)) : z;
 #pragma unroll
-        for (int n = 0; n < N; ++n) acc[n] = 0;
-        const uint4 *arow = STAGED ? stage + (size_t)lane * k16 : reinterpret_cast<const uint4 *>(A + m * lda);
-        for (int c = 0; c < k16; ++c) {
-            const uint4 a = STAGED ? arow[c] : __ldcs(arow + c);
-            const unsigned int aw[4] = {a.x, a.y, a.z, a.w};
+            for (int j = 0; j < NT; ++j) mma_k32<A_UNSIGNED>(acc[j], x0.x, x1.x, x0.y, x1.y, bf[j * 64], bf[j * 64 + 32]);
+            bf += NT * 64;
+            kb += 32;
+        }
+        if ((rest & 31) == 16) {
+            const unsigned int x0 = v0 ? __ldcs(reinterpret_cast<const unsigned int *>(p0 + kb + 4 * t)) : 0u;
+            const unsigned int x1 = v1 ? __ldcs(reinterpret_cast<const unsigned int *>(p1 + kb + 4 * t)) : 0u;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 *wrow = reinterpret_cast<const uint4 *>(Wp + (4 * c + j) * N);
+            for (int j = 0; j < NT; ++j) mma_k32<A_UNSIGNED>(acc[j], x0, x1, 0u, 0u, bf[j * 64], 0u);
+        }
+        if (N == 4 && t >= 2) continue;                         // columns 4 .. 7 of the only tile do not exist
 #pragma unroll
-                for (int n4 = 0; n4 < N / 4; ++n4) {
-                    const uint4 w = wrow[n4];                    // same address in every lane: a broadcast
-                    acc[4 * n4 + 0] = dot4<A_UNSIGNED>(aw[j], w.x, acc[4 * n4 + 0]);
-                    acc[4 * n4 + 1] = dot4<A_UNSIGNED>(aw[j], w.y, acc[4 * n4 + 1]);
-                    acc[4 * n4 + 2] = dot4<A_UNSIGNED>(aw[j], w.z, acc[4 * n4 + 2]);
-                    acc[4 * n4 + 3] = dot4<A_UNSIGNED>(aw[j], w.w, acc[4 * n4 + 3]);
+        for (int half = 0; half < 2; ++half) {
+            const long long r = half == 0 ? r0 : r1;
+            if (r >= M) continue;
+            int v[2 * NT];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                v[2 * j] = acc[j][2 * half];
+                v[2 * j + 1] = acc[j][2 * half + 1];
+            }
+            if (acc_out != nullptr) {
+                int *o = acc_out + r * N + cb;
+                if constexpr (2 * NT >= 4) {
+#pragma unroll
+                    for (int q = 0; q < 2 * NT; q += 4) *reinterpret_cast<int4 *>(o + q) = make_int4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                } else {
+                    *reinterpret_cast<int2 *>(o) = make_int2(v[0], v[1]);
                 }
             }
-        }
-        if (acc_out != nullptr) {
-            int4 *o = reinterpret_cast<int4 *>(acc_out + m * N);
+            if (y_out != nullptr) {
+                float f[2 * NT];
 #pragma unroll
-            for (int n4 = 0; n4 < N / 4; ++n4) o[n4] = make_int4(acc[4 * n4], acc[4 * n4 + 1], acc[4 * n4 + 2], acc[4 * n4 + 3]);
-        }
-        if (y_out != nullptr) {
-            float4 *o = reinterpret_cast<float4 *>(y_out + m * N);
-#pragma unroll
-            for (int n4 = 0; n4 < N / 4; ++n4) {
-                float f[4];
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    f[b] = __fmul_rn((float)acc[4 * n4 + b], scale);
-                    if (bias != nullptr) f[b] = __fadd_rn(f[b], bias[4 * n4 + b]);
+                for (int q = 0; q < 2 * NT; ++q) {
+                    f[q] = __fmul_rn((float)v[q], scale);
+                    if (bias != nullptr) f[q] = __fadd_rn(f[q], bv[q]);
                 }
-                __stcs(o + n4, make_float4(f[0], f[1], f[2], f[3]));
+                float *o = y_out + r * N + cb;
+                if constexpr (2 * NT >= 4) {
+#pragma unroll
+                    for (int q = 0; q < 2 * NT; q += 4) __stcs(reinterpret_cast<float4 *>(o + q), make_float4(f[q], f[q + 1], f[q + 2], f[q + 3]));
+                } else {
+                    __stcs(reinterpret_cast<float2 *>(o), make_float2(f[0], f[1]));
+                }
             }
         }
     }
@@ -156,6 +215,69 @@ skinny_dx_kernel(const signed char *__restrict__ G, long long ldg, const signed 
     }
 }
 
+// dX on the matrix instruction (K a multiple of 16): a warp takes 16 rows, its G fragment is one 4- or 8-byte load
+// per row, and every pair of 8-column tiles of the output is two instructions whose results a lane stores as 16
+// consecutive bytes per row (columns dealt to the tiles so that a quad writes 64 consecutive bytes).
+template <int N>
+__global__ void __launch_bounds__(kSkinnyThreads)
+skinny_dx_mma_kernel(const signed char *__restrict__ G, long long ldg, const signed char *__restrict__ W, long long ldw,
+                     int M, int K, int32_t *__restrict__ acc_out, float *__restrict__ f_out, float scale, int accumulate)
+{
+    constexpr int NH = N == 32 ? 2 : 1;                         // words per lane of a W fragment
+    extern __shared__ __align__(16) unsigned int Bf[];          // [tile][half][lane]
+    const int ntile = K / 8;
+    for (int i = threadIdx.x; i < ntile * NH * 32; i += kSkinnyThreads) {
+        const int ln = i & 31, h = NH == 2 ? (i >> 5) & 1 : 0, j = i / (32 * NH);
+        const int tt = ln & 3, gg = ln >> 2;
+        const int kc = 16 * (j >> 1) + 4 * (gg >> 1) + 2 * (j & 1) + (gg & 1);      // the output column behind (tile, gg)
+        const int nb = N == 32 ? 8 * tt + 4 * h : 4 * tt;
+        Bf[i] = nb < N ? *reinterpret_cast<const unsigned int *>(W + (long long)kc * ldw + nb) : 0u;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, t = lane & 3, g = lane >> 2;
+    const long long warp = ((long long)blockIdx.x * kSkinnyThreads + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * kSkinnyThreads) >> 5;
+    const long long ntiles = ((long long)M + 15) / 16;
+    for (long long tile = warp; tile < ntiles; tile += nwarps) {
+        __syncwarp();                                           // the matrix instruction wants the whole warp
+        const long long r0 = tile * 16 + g, r1 = r0 + 8;
+        const bool v0 = r0 < M, v1 = r1 < M;
+        unsigned int a0 = 0u, a1 = 0u, a2 = 0u, a3 = 0u;
+        if (N == 32) {
+            if (v0) { const uint2 x = *reinterpret_cast<const uint2 *>(G + r0 * ldg + 8 * t); a0 = x.x; a2 = x.y; }
+            if (v1) { const uint2 x = *reinterpret_cast<const uint2 *>(G + r1 * ldg + 8 * t); a1 = x.x; a3 = x.y; }
+        } else if (4 * t < N) {
+            if (v0) a0 = *reinterpret_cast<const unsigned int *>(G + r0 * ldg + 4 * t);
+            if (v1) a1 = *reinterpret_cast<const unsigned int *>(G + r1 * ldg + 4 * t);
+        }
+        const unsigned int *bf = Bf + lane;
+        for (int p = 0; p < K / 16; ++p, bf += 2 * NH * 32) {
+            int d0[4] = {0, 0, 0, 0}, d1[4] = {0, 0, 0, 0};
+            mma_k32<false>(d0, a0, a1, a2, a3, bf[0], NH == 2 ? bf[32] : 0u);
+            mma_k32<false>(d1, a0, a1, a2, a3, bf[NH * 32], NH == 2 ? bf[NH * 32 + 32] : 0u);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const long long r = half == 0 ? r0 : r1;
+                if (r >= M) continue;
+                const long long o = r * K + 16 * p + 4 * t;
+                const int v[4] = {d0[2 * half], d0[2 * half + 1], d1[2 * half], d1[2 * half + 1]};
+                if (acc_out != nullptr) *reinterpret_cast<int4 *>(acc_out + o) = make_int4(v[0], v[1], v[2], v[3]);
+                if (f_out != nullptr) {
+                    float4 f = make_float4(__fmul_rn((float)v[0], scale), __fmul_rn((float)v[1], scale),
+                                           __fmul_rn((float)v[2], scale), __fmul_rn((float)v[3], scale));
+                    float4 *fo = reinterpret_cast<float4 *>(f_out + o);
+                    if (accumulate) {
+                        const float4 c = *fo;
+                        *fo = make_float4(__fadd_rn(c.x, f.x), __fadd_rn(c.y, f.y), __fadd_rn(c.z, f.z), __fadd_rn(c.w, f.w));
+                    } else {
+                        __stcs(fo, f);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ dW
 // dW[k, n] = sum_m A[m, k] G[m, n]: the contraction runs over rows, so both operands are needed with four
 // consecutive rows of one column in a word.  A warp works alone on jobs of 32 rows x (16 MT columns of A): it reads
@@ -175,19 +297,6 @@ __device__ __forceinline__ void transpose4x4(unsigned int r0, unsigned int r1, u
     o[1] = __byte_perm(t0, t1, 0x7632);
     o[2] = __byte_perm(t2, t3, 0x5410);
     o[3] = __byte_perm(t2, t3, 0x7632);
-}
-
-// D (16 x 8, int32) += A (16 x 32 bytes, row-major fragment) B (32 x 8 int8, column fragment)
-template <bool A_UNSIGNED>
-__device__ __forceinline__ void mma_k32(int (&d)[4], unsigned int a0, unsigned int a1, unsigned int a2, unsigned int a3,
-                                        unsigned int b0, unsigned int b1)
-{
-    if (A_UNSIGNED)
-        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-    else
-        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 struct DwTail {                 // what the last CTA to finish does with the sums
@@ -340,18 +449,23 @@ int grid_for(long long work_items)
     return (int)(blocks < 1 ? 1 : blocks);
 }
 
-template <int N, bool A_UNSIGNED, bool STAGED>
+template <int N, bool A_UNSIGNED>
 int launch_fwd_t(const unsigned char *a, long long lda, const signed char *w, long long ldw, int M, int K, int32_t *acc_out,
                  float *y_out, float scale, const float *bias, cudaStream_t stream)
 {
-    const int grid = grid_for(M);
-    if (grid == 0) return CDL_ERR_LAUNCH;
-    const size_t smem = (size_t)K * N + (STAGED ? (size_t)(kSkinnyThreads / 32) * 32 * K : 0);
-    auto kern = skinny_fwd_kernel<N, A_UNSIGNED, STAGED>;
+    const int sms = sm_count();
+    if (sms <= 0) return CDL_ERR_LAUNCH;
+    constexpr int NT = N >= 8 ? N / 8 : 1;
+    const int rest = K & 63;
+    const int nsteps = 2 * (K >> 6) + (rest >= 32 ? 1 : 0) + ((rest & 31) == 16 ? 1 : 0);
+    const size_t smem = (size_t)nsteps * NT * 64 * sizeof(unsigned int);
+    auto kern = skinny_fwd_kernel<N, A_UNSIGNED>;
     if (smem > 48 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return CDL_ERR_LAUNCH;
     }
+    const long long need = (((long long)M + 15) / 16 + kSkinnyThreads / 32 - 1) / (kSkinnyThreads / 32);
+    const int grid = (int)(need < 4ll * sms ? need : 4ll * sms);
     kern<<<grid, kSkinnyThreads, smem, stream>>>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias);
     return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
 }
@@ -362,12 +476,27 @@ int launch_fwd_n(const void *A, long long lda, bool a_unsigned, const void *W, l
 {
     const unsigned char *a = static_cast<const unsigned char *>(A);
     const signed char *w = static_cast<const signed char *>(W);
-    const bool staged = (size_t)K * N + (size_t)kSkinnyThreads * K <= 96 * 1024;
-    if (a_unsigned)
-        return staged ? launch_fwd_t<N, true, true>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream)
-                      : launch_fwd_t<N, true, false>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream);
-    return staged ? launch_fwd_t<N, false, true>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream)
-                  : launch_fwd_t<N, false, false>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream);
+    return a_unsigned ? launch_fwd_t<N, true>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream)
+                      : launch_fwd_t<N, false>(a, lda, w, ldw, M, K, acc_out, y_out, scale, bias, stream);
+}
+
+template <int N>
+int launch_dx_mma(const void *G, long long ldg, const void *W, long long ldw, int M, int K, int32_t *acc_out, float *f_out,
+                  float scale, bool accumulate, cudaStream_t stream)
+{
+    const int sms = sm_count();
+    if (sms <= 0) return CDL_ERR_LAUNCH;
+    const size_t smem = (size_t)(K / 8) * (N == 32 ? 2 : 1) * 32 * sizeof(unsigned int);
+    auto kern = skinny_dx_mma_kernel<N>;
+    if (smem > 48 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    const long long need = (((long long)M + 15) / 16 + kSkinnyThreads / 32 - 1) / (kSkinnyThreads / 32);
+    const int grid = (int)(need < 6ll * sms ? need : 6ll * sms);
+    kern<<<grid, kSkinnyThreads, smem, stream>>>(static_cast<const signed char *>(G), ldg, static_cast<const signed char *>(W),
+                                                 ldw, M, K, acc_out, f_out, scale, accumulate ? 1 : 0);
+    return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
 }
 
 template <int NW>
@@ -462,7 +591,7 @@ int launch_skinny_dw(const void *A, long long lda, bool a_unsigned, const void *
 bool skinny_fwd_ok(int M, int N, int K)
 {
     (void)M;
-    return (N == 4 || N == 8 || N == 16 || N == 32) && (K % 16) == 0 && (long long)K * N <= 96 * 1024;
+    return (N == 4 || N == 8 || N == 16 || N == 32) && (K % 16) == 0 && (long long)K * (N < 8 ? 8 : N) <= 96 * 1024;
 }
 
 bool skinny_dx_ok(int M, int N, int K)
@@ -472,7 +601,7 @@ bool skinny_dx_ok(int M, int N, int K)
     return N == 4 || N == 8 || N == 16 || N == 32;
 }
 
-// Y (M x N, row pitch N) from A (M x K bytes, pitch lda, 16-byte aligned rows) and W (K x N int8, pitch ldw)
+// Y (M x N floats and / or int32) = A (M x K bytes) W (K x N int8); outputs 16-byte aligned
 int launch_skinny_fwd(const void *A, long long lda, bool a_unsigned, const void *W, long long ldw, int M, int N, int K,
                       int32_t *acc_out, float *y_out, float scale, const float *bias, cudaStream_t stream)
 {
@@ -485,10 +614,21 @@ int launch_skinny_fwd(const void *A, long long lda, bool a_unsigned, const void 
     }
 }
 
-// dA (M x K, row pitch K) from G (M x N int8, pitch ldg, 4-byte aligned rows) and W (K x N int8, pitch ldw)
+// dX (M x K) = G (M x N int8) W^T (W: K x N int8): the matrix-instruction kernel when K is a multiple of 16, its
+// fragment table fits and the outputs are 16-byte aligned, else the dp4a kernel
 int launch_skinny_dx(const void *G, long long ldg, const void *W, long long ldw, int M, int N, int K, int32_t *acc_out,
                      float *f_out, float scale, bool accumulate, cudaStream_t stream)
 {
+    const bool aligned = ((reinterpret_cast<uintptr_t>(acc_out) | reinterpret_cast<uintptr_t>(f_out)) & 15u) == 0;
+    if ((K % 16) == 0 && aligned && (long long)(K / 8) * (N == 32 ? 2 : 1) * 128 <= 96 * 1024) {
+        switch (N) {
+            case 4: return launch_dx_mma<4>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
+            case 8: return launch_dx_mma<8>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
+            case 16: return launch_dx_mma<16>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
+            case 32: return launch_dx_mma<32>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
+            default: return CDL_ERR_ARG;
+        }
+    }
     switch (N) {
         case 4: return launch_dx_nw<1>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
         case 8: return launch_dx_nw<2>(G, ldg, W, ldw, M, K, acc_out, f_out, scale, accumulate, stream);
