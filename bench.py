@@ -822,6 +822,7 @@ def main():
         roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.workload, dom))
         gemm_ms = sum(per_call_ms[c] for c in ("qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_dw"))
         quant_ms = sum(per_call_ms[c] for c in CALLS if model[c]["elems"])
+        step_bytes = sum(model[c]["bytes"] for c in CALLS)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -829,7 +830,9 @@ def main():
             "config": {"workload": args.workload, "M": M, "K": K, "N": N, "activation_elems": n_x,
                        "weight_levels": case.wq.nlev, "activation_levels": case.aq.nlev,
                        "alpha": case.wq.alpha, "rate_weight": case.wq.rate_weight, "window_x": case.aq.window,
-                       "l2": "per-step working set is several times the 126 MB L2 (inputs larger than L2)",
+                       "l2": ("per-step working set is several times the 126 MB L2 (inputs larger than L2)"
+                              if step_bytes > 2 * 126e6 else
+                              "per-step working set (%.0f MB) fits the 126 MB L2: a parity-size workload, not a bandwidth figure" % (step_bytes / 1e6)),
                        "parallelism": f"replicas x{world}, all-reduce of dW / histogram / scalars" if world > 1 else "single GPU"},
             "layer_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": 6.0 * M * K * N / (gemm_ms * 1e-3) / 1e12,
             "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": quant_elems / (quant_ms * 1e-3) / 1e9,
