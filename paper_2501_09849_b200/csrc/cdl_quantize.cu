@@ -416,7 +416,7 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
     // d = x - kn q as dh + dl
     // logits of the two neighbours relative to the nearest level: -alpha q (q -+ 2 d)
     float2 dh, w1, wm;
-    if (P.res1) {
+    if (P.res1 && MODE != MODE_SAMPLE) {   // (the sampled index keeps the two-float residual of the one-by-one path)
         // moderate alpha q^2: the correctly rounded residual of one fused multiply-add is accurate enough (its 2^-25 q
         // moves a logit by at most 2 alpha q^2 2^-25 < 4e-6)
         dh = __ffma2_rn(kn, f2(-q), x);
@@ -439,6 +439,18 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
     em.x = (kn.x > P.flo) ? em.x : 0.0f;
     em.y = (kn.y > P.flo) ? em.y : 0.0f;
     const float2 S = __fadd2_rn(__fadd2_rn(f2(1.0f), e1), em);
+    if (MODE == MODE_SAMPLE) {
+        // inversion in increasing level order: kn-1 (em), kn (1), kn+1 (e1); g carries the uniform numbers
+        const float2 gs = __fmul2_rn(g, S), cap = __fmul2_rn(S, f2(0.99999994f)), em1 = __fadd2_rn(em, f2(1.0f));
+        const float tx = fminf(gs.x, cap.x), ty = fminf(gs.y, cap.y);
+        const int s0 = k0 + ((tx >= em1.x) ? 1 : 0) - ((tx < em.x) ? 1 : 0);
+        const int s1 = k1 + ((ty >= em1.y) ? 1 : 0) - ((ty < em.y) ? 1 : 0);
+        o.k0[0] = s0;
+        o.k0[1] = s1;
+        o.y = __fmul2_rn(make_float2((float)s0, (float)s1), f2(q));
+        o.gx = o.tq = o.ta = f2(0.0f);
+        return o;
+    }
     const float2 rS = make_float2(rcp_approx(S.x), rcp_approx(S.y));
     const float2 m1 = __fmul2_rn(sub2(e1, em), rS);
     o.y = __ffma2_rn(kn, f2(q), __fmul2_rn(f2(q), m1));
@@ -586,7 +598,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 }
                 float ys[4], gxs[4];
                 unsigned int packed = 0u;
-                constexpr bool kPairs = PATH == PATH_NEAR3 && (MODE == MODE_BWD || (MODE == MODE_SOFT && !RATE));
+                constexpr bool kPairs = PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE));
                 if (kPairs) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
