@@ -25,7 +25,16 @@
 //          The window needs the exact nearest level (ties: the lower one), decided from dh + dl on a rarely
 //          taken branch.
 //   LOOP   everything else (whole index set, or another odd window): a loop over the levels within jmax
-//          steps of kn (further ones weigh < 2^-40).
+//          steps of kn (further ones weigh < 2^-40), one ex2 per level.
+//   LATTICE  whole index set, vector region of the soft and backward passes: e_j = G_j b^j with G_j = 2^(-A j^2)
+//          the same for every element (a shared-memory table that also holds j G_j, j^2 G_j, j^3 G_j) and
+//          b = 2^B per element, so a level costs a few multiply-adds and no ex2.  b^j is carried as
+//          1 + beta_j, beta_(j+1) = beta_j + (beta_j beta + beta): for small alpha q^2 b is so close to 1 that
+//          a binary32 b would lose B (its relative error, times j, would shift theta by far more than the
+//          tolerance), while beta = 2^B - 1 keeps it to full relative precision.  The four elements of a load
+//          walk the levels together on the packed instructions, the levels above and below kn separately and
+//          outwards.  Taken when the window of +-jmax levels is narrower than the index set and no rate term is
+//          asked for (1.3x the LOOP form on the soft pass, 1.4x on the backward pass).
 #include "cdl_internal.h"
 
 #include <math.h>
@@ -61,7 +70,7 @@ constexpr int kMagicBits = 0x4B400000;
 // allowed for: indices lie in [-128, 255], where an ulp is at most 2^-16; 0.5 - 2^-12 leaves 16 ulp of margin.
 constexpr float kTieGuard = 0.5f - 0.000244140625f;
 
-enum QuantPath { PATH_NEAR3 = 0, PATH_WIN5 = 1, PATH_LOOP = 2 };
+enum QuantPath { PATH_NEAR3 = 0, PATH_WIN5 = 1, PATH_LOOP = 2, PATH_LATTICE = 3 };
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
@@ -479,6 +488,151 @@ __device__ __forceinline__ PairOut quant_pair_near3(const QuantDev &P, const flo
     return o;
 }
 
+// ---- whole index set without an ex2 per level (see LATTICE in the header comment): the four elements of a
+// 128-bit load as two packed pairs that walk the levels together, so that one table load serves all four.
+struct LatPair {
+    float2 kn, dh, bu, bd;          // reference level, residual, 2^B - 1, 2^-B - 1
+    int k0, k1;
+    float2 A0, A1, A2, A3;          // sums over the levels other than kn of j^m e_j, m = 0..3
+};
+
+__device__ __forceinline__ void lattice_setup(const QuantDev &P, float2 x, LatPair &s)
+{
+    const float q = P.q;
+    // hard index (see quant_elem): reciprocal product, clamp, magic-number rounding, exact quotient near ties
+    float2 c = __fmul2_rn(x, f2(P.rq));
+    if (!P.fast_div) c = make_float2(__fdiv_rn(x.x, q), __fdiv_rn(x.y, q));
+    c.x = fminf(fmaxf(c.x, P.flo), P.fhi);
+    c.y = fminf(fmaxf(c.y, P.flo), P.fhi);
+    float2 t = __fadd2_rn(c, f2(kMagic));
+    float2 kn = __fadd2_rn(t, f2(-kMagic));
+    if (P.fast_div) {
+        const float2 df = sub2(c, kn);
+        if (fabsf(df.x) > kTieGuard || fabsf(df.y) > kTieGuard) {
+            c.x = fminf(fmaxf(__fdiv_rn(x.x, q), P.flo), P.fhi);
+            c.y = fminf(fmaxf(__fdiv_rn(x.y, q), P.flo), P.fhi);
+            t = __fadd2_rn(c, f2(kMagic));
+            kn = __fadd2_rn(t, f2(-kMagic));
+        }
+    }
+    s.kn = kn;
+    s.k0 = __float_as_int(t.x) - kMagicBits;
+    s.k1 = __float_as_int(t.y) - kMagicBits;
+    s.dh = __ffma2_rn(kn, f2(-q), x);
+    // B = 2 alpha q d log2 e, limited to +-64: beyond that the element lies far outside the index set and the
+    // levels on the side that still exists weigh < 2^-64 either way
+    float2 B = __fmul2_rn(s.dh, f2(P.c1x2));
+    B.x = fminf(fmaxf(B.x, -64.0f), 64.0f);
+    B.y = fminf(fmaxf(B.y, -64.0f), 64.0f);
+    // beta = 2^B - 1 upwards, 2^-B - 1 downwards.  |B| < 1: expm1 of a quarter of the argument by its series
+    // (|z| < 0.174, remainder < 5e-9 relative), then (1 + beta)^2 - 1 = beta (2 + beta) twice; the downward one
+    // from -beta / (1 + beta).  Otherwise from ex2 directly (b is then far enough from 1).
+    const float2 z = __fmul2_rn(B, f2(0.25f * 0.693147180559945f));
+    float2 pz = __ffma2_rn(z, f2(1.0f / 720.0f), f2(1.0f / 120.0f));
+    pz = __ffma2_rn(z, pz, f2(1.0f / 24.0f));
+    pz = __ffma2_rn(z, pz, f2(1.0f / 6.0f));
+    pz = __ffma2_rn(z, pz, f2(0.5f));
+    pz = __ffma2_rn(z, pz, f2(1.0f));
+    pz = __fmul2_rn(z, pz);
+    pz = __fmul2_rn(pz, __fadd2_rn(pz, f2(2.0f)));
+    pz = __fmul2_rn(pz, __fadd2_rn(pz, f2(2.0f)));
+    const float2 pd1 = __fadd2_rn(pz, f2(1.0f));
+    const float2 pd = __fmul2_rn(__fmul2_rn(pz, f2(-1.0f)), make_float2(rcp_approx(pd1.x), rcp_approx(pd1.y)));
+    s.bu.x = fabsf(B.x) < 1.0f ? pz.x : ex2_approx(B.x) - 1.0f;
+    s.bu.y = fabsf(B.y) < 1.0f ? pz.y : ex2_approx(B.y) - 1.0f;
+    s.bd.x = fabsf(B.x) < 1.0f ? pd.x : ex2_approx(-B.x) - 1.0f;
+    s.bd.y = fabsf(B.y) < 1.0f ? pd.y : ex2_approx(-B.y) - 1.0f;
+    s.A0 = s.A1 = s.A2 = s.A3 = f2(0.0f);
+}
+
+// adds level kn + DIR * j with weight G_j * w to the sums of one pair
+template <bool BWD, int DIR>
+__device__ __forceinline__ void lattice_add(LatPair &s, float4 ga, float4 ha, float2 w)
+{
+    s.A0 = __ffma2_rn(make_float2(ga.x, ga.y), w, s.A0);
+    s.A1 = __ffma2_rn(make_float2(DIR * ga.z, DIR * ga.w), w, s.A1);
+    if (BWD) {
+        s.A2 = __ffma2_rn(make_float2(ha.x, ha.y), w, s.A2);
+        s.A3 = __ffma2_rn(make_float2(DIR * ha.z, DIR * ha.w), w, s.A3);
+    }
+}
+
+// One side of the sums for both pairs: levels kn + DIR * j, j = 1 .. n (n0..n3 per element).
+template <bool BWD, int DIR>
+__device__ __forceinline__ void lattice_side(const float4 *__restrict__ Gtab, const float4 *__restrict__ Htab, LatPair &s0,
+                                             LatPair &s1, int n0, int n1, int n2, int n3)
+{
+    const float2 one = f2(1.0f);
+    const float2 b0 = DIR > 0 ? s0.bu : s0.bd, b1 = DIR > 0 ? s1.bu : s1.bd;
+    float2 w0 = b0, w1 = b1;               // b^j - 1
+    const int nc = min(min(n0, n1), min(n2, n3)), nm = max(max(n0, n1), max(n2, n3));
+    int j = 1;
+    for (; j <= nc; ++j) {
+        const float4 ga = Gtab[j];
+        const float4 ha = BWD ? Htab[j] : ga;
+        lattice_add<BWD, DIR>(s0, ga, ha, __fadd2_rn(w0, one));
+        lattice_add<BWD, DIR>(s1, ga, ha, __fadd2_rn(w1, one));
+        w0 = __fadd2_rn(w0, __ffma2_rn(w0, b0, b0));
+        w1 = __fadd2_rn(w1, __ffma2_rn(w1, b1, b1));
+    }
+    for (; j <= nm; ++j) {                 // elements with fewer levels on this side add zeros
+        const float4 ga = Gtab[j];
+        const float4 ha = BWD ? Htab[j] : ga;
+        float2 u0 = __fadd2_rn(w0, one), u1 = __fadd2_rn(w1, one);
+        u0.x = (j <= n0) ? u0.x : 0.0f;
+        u0.y = (j <= n1) ? u0.y : 0.0f;
+        u1.x = (j <= n2) ? u1.x : 0.0f;
+        u1.y = (j <= n3) ? u1.y : 0.0f;
+        lattice_add<BWD, DIR>(s0, ga, ha, u0);
+        lattice_add<BWD, DIR>(s1, ga, ha, u1);
+        w0 = __fadd2_rn(w0, __ffma2_rn(w0, b0, b0));
+        w1 = __fadd2_rn(w1, __ffma2_rn(w1, b1, b1));
+    }
+}
+
+template <int MODE>
+__device__ __forceinline__ PairOut lattice_finish(const QuantDev &P, const LatPair &s, float2 g)
+{
+    PairOut o;
+    const float q = P.q;
+    o.k0[0] = s.k0;
+    o.k0[1] = s.k1;
+    const float2 S = __fadd2_rn(s.A0, f2(1.0f));
+    const float2 rS = make_float2(rcp_approx(S.x), rcp_approx(S.y));
+    const float2 m1 = __fmul2_rn(s.A1, rS);
+    o.y = __ffma2_rn(s.kn, f2(q), __fmul2_rn(f2(q), m1));
+    o.gx = o.tq = o.ta = f2(0.0f);
+    if (MODE == MODE_BWD) {
+        const float2 m2 = __fmul2_rn(s.A2, rS), m3 = __fmul2_rn(s.A3, rS);
+        const float2 nm1 = __fmul2_rn(m1, f2(-1.0f));
+        const float2 varj = __ffma2_rn(nm1, m1, m2);
+        const float2 covj = __ffma2_rn(nm1, m2, m3);
+        o.gx = __fmul2_rn(g, __fmul2_rn(f2(P.a2), varj));
+        const float2 qc = __fmul2_rn(f2(q), covj);
+        const float2 dmk = __ffma2_rn(s.kn, f2(-q), s.dh);             // d - kn q
+        o.tq = __ffma2_rn(f2(P.two_aq), sub2(__fmul2_rn(dmk, varj), qc), __fadd2_rn(s.kn, m1));
+        o.ta = __fmul2_rn(f2(P.q2), sub2(__fmul2_rn(__fmul2_rn(f2(2.0f), s.dh), varj), qc));
+    }
+    return o;
+}
+
+template <int MODE>
+__device__ __forceinline__ void quant_quad_lattice(const QuantDev &P, const float4 *__restrict__ Gtab,
+                                                   const float4 *__restrict__ Htab, const float (&xs)[4],
+                                                   const float (&gs)[4], PairOut (&o)[2])
+{
+    constexpr bool kBwd = MODE == MODE_BWD;
+    LatPair s0, s1;
+    lattice_setup(P, make_float2(xs[0], xs[1]), s0);
+    lattice_setup(P, make_float2(xs[2], xs[3]), s1);
+    lattice_side<kBwd, 1>(Gtab, Htab, s0, s1, min(P.hi - s0.k0, P.jmax), min(P.hi - s0.k1, P.jmax),
+                          min(P.hi - s1.k0, P.jmax), min(P.hi - s1.k1, P.jmax));
+    lattice_side<kBwd, -1>(Gtab, Htab, s0, s1, min(s0.k0 - P.lo, P.jmax), min(s0.k1 - P.lo, P.jmax),
+                           min(s1.k0 - P.lo, P.jmax), min(s1.k1 - P.lo, P.jmax));
+    o[0] = lattice_finish<MODE>(P, s0, make_float2(gs[0], gs[1]));
+    o[1] = lattice_finish<MODE>(P, s1, make_float2(gs[2], gs[3]));
+}
+
 __device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane)
 {
     atomicAdd(&hist_s[bin * 32 + lane], 1u);
@@ -506,6 +660,21 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) mp_s[k] = 0ull;
     }
 
+    // LATTICE: (G_j, G_j, j G_j, j G_j) and (j^2 G_j, j^2 G_j, j^3 G_j, j^3 G_j), G_j = 2^(-A j^2), for the level j steps
+    // from the nearest one; every entry twice so that a 128-bit load yields two packed operands
+    __shared__ float4 Gtab[PATH == PATH_LATTICE ? CDL_MAX_LEVELS : 1];
+    __shared__ float4 Htab[(PATH == PATH_LATTICE && MODE == MODE_BWD) ? CDL_MAX_LEVELS : 1];
+    if (PATH == PATH_LATTICE) {
+        for (int j = threadIdx.x; j < CDL_MAX_LEVELS; j += kThreads) {
+            const float jf = (float)j;
+            const float G = exp2f(__fmul_rn(__fmul_rn(-P.A, jf), jf)), jG = __fmul_rn(jf, G), j2G = __fmul_rn(jf, jG);
+            Gtab[j] = make_float4(G, G, jG, jG);
+            if (MODE == MODE_BWD) {
+                const float j3G = __fmul_rn(jf, j2G);
+                Htab[j] = make_float4(j2G, j2G, j3G, j3G);
+            }
+        }
+    }
     constexpr bool kPairRate = MODE == MODE_BWD && RATE && PATH == PATH_NEAR3;
     __shared__ float2 Dtab[kPairRate ? CDL_MAX_LEVELS : 1];     // (L[k+1] - L[k], L[k-1] - L[k]), clamped at the ends
     if (MODE == MODE_BWD && RATE) {
@@ -521,7 +690,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     }
     if (do_hist)
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) hist_s[k] = 0u;
-    if (RATE || do_hist) __syncthreads();
+    if (RATE || do_hist || PATH == PATH_LATTICE) __syncthreads();
 
     unsigned int *const hist_l = hist_s + (lane - P.lo * 32);    // this lane's column, indexed by level: hist_l[k * 32]
     double acc_q = 0.0, acc_a = 0.0;
@@ -598,12 +767,15 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 }
                 float ys[4], gxs[4];
                 unsigned int packed = 0u;
-                constexpr bool kPairs = PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE));
+                constexpr bool kPairs = (PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE))) ||
+                                        (PATH == PATH_LATTICE && !RATE && (MODE == MODE_BWD || MODE == MODE_SOFT));
                 if (kPairs) {
+                    PairOut quad[2];
+                    if (PATH == PATH_LATTICE) quant_quad_lattice<MODE>(P, Gtab, Htab, xs, gs, quad);
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const PairOut o = quant_pair_near3<MODE, RATE>(P, Dtab, make_float2(xs[2 * h], xs[2 * h + 1]),
-                                                                       make_float2(gs[2 * h], gs[2 * h + 1]));
+                        const float2 xp = make_float2(xs[2 * h], xs[2 * h + 1]), gp = make_float2(gs[2 * h], gs[2 * h + 1]);
+                        const PairOut o = PATH == PATH_LATTICE ? quad[h] : quant_pair_near3<MODE, RATE>(P, Dtab, xp, gp);
                         ys[2 * h] = o.y.x;
                         ys[2 * h + 1] = o.y.y;
                         gxs[2 * h] = o.gx.x;
@@ -795,6 +967,12 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     unsigned char *ib = static_cast<unsigned char *>(idx);
     const int path = qd.near3 ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
     const bool rate = (mode == MODE_BWD) && qd.level_prob != nullptr && qd.rate_c != 0.0f;
+    // Whole index set, levels within jmax steps on both sides for most elements (2 jmax + 1 < nlev), vector region
+    // present, no soft histogram and no rate term: the table form of the level sums.  (When the index set is
+    // narrower than the window, an element's levels lie mostly on one side of it, a warp walks both sides to the
+    // longest lane's end, and the form loses what it gains; with the rate term it was no faster either.)
+    const bool lattice = path == PATH_LOOP && qd.window == 0 && n4 > 0 && 2 * qd.jmax + 1 < qd.nlev && !rate &&
+                         ((mode == MODE_SOFT && soft_hist == nullptr) || mode == MODE_BWD);
 #define CDL_Q(M, PTH, RT) \
     launch_t<M, PTH, RT>(qd, x, grad_out, n, head, n4, y, ib, hist, grad_x, grad_q, grad_alpha, soft_hist, stream)
     switch (mode) {
@@ -805,6 +983,7 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
                 return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, true)
                      : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, true)
                                          : CDL_Q(MODE_SOFT, PATH_LOOP, true);
+            if (lattice) return CDL_Q(MODE_SOFT, PATH_LATTICE, false);
             return path == PATH_NEAR3 ? CDL_Q(MODE_SOFT, PATH_NEAR3, false)
                  : path == PATH_WIN5 ? CDL_Q(MODE_SOFT, PATH_WIN5, false)
                                      : CDL_Q(MODE_SOFT, PATH_LOOP, false);
@@ -813,6 +992,7 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
                  : path == PATH_WIN5 ? CDL_Q(MODE_SAMPLE, PATH_WIN5, false)
                                      : CDL_Q(MODE_SAMPLE, PATH_LOOP, false);
         case MODE_BWD:
+            if (lattice) return CDL_Q(MODE_BWD, PATH_LATTICE, false);
             if (rate)
                 return path == PATH_NEAR3 ? CDL_Q(MODE_BWD, PATH_NEAR3, true)
                      : path == PATH_WIN5 ? CDL_Q(MODE_BWD, PATH_WIN5, true)

@@ -362,3 +362,40 @@ def test_three_level_path_on_both_sides_of_the_residual_switch(torch, aq2, lo, h
     assert_soft_close(y, oracle.soft(x, f32(q), lo, hi, f32(alpha), 0), q)
     gx, gq, ga = run_backward(torch, x, g, P)
     assert_backward_close(gx, gq, ga, oracle.backward(x, g, f32(q), lo, hi, f32(alpha), 0), g, q, alpha)
+
+
+# ------------------------------------------------------- whole index set, window narrower than the index set
+@pytest.mark.parametrize("lo,hi,q,alpha", [
+    (-32, 31, 0.05, 20.0),      # alpha q^2 log2 e = 0.072: powers of b carried as 1 + beta_j
+    (-32, 31, 0.05, 60.0),      # 0.216: powers of b by repeated multiplication
+    (0, 63, 0.06, 25.0),        # unsigned index set with half of the data at its lower edge
+    (-128, 127, 0.03, 30.0),    # the widest index set, 0.039
+])
+def test_table_form_of_the_level_sums(torch, lo, hi, q, alpha):
+    # The soft and backward passes over the whole index set when levels further than jmax steps from the nearest
+    # one carry no weight and 2 jmax + 1 < nlev: level weights G_j b^j from a table and a recurrence instead of
+    # one exponential per level.  Data: a normal/Laplace mixture wide enough that some elements sit at the edges
+    # of the index set (levels on one side only) and far outside it; rate term with non-uniform level
+    # probabilities; an element count that leaves a scalar tail.
+    n = (1 << 17) + 3
+    x = (inputs.normal_laplace_mixture((n,), seed=lo + 300) * f32(0.45 * hi * q)).astype(f32)
+    if lo == 0:
+        x = np.maximum(x, f32(0.0)) + (x < 0) * f32(-0.02) * (np.arange(n) % 7 == 0)
+        x = x.astype(f32)
+    g = inputs.normal((n,), 1.0, seed=hi + 400)
+    nlev = hi - lo + 1
+    ref_idx, ref_hist = oracle.hard(x, f32(q), lo, hi)
+    P = cdl.QuantParams(q, lo, hi, alpha)
+    y, idx, hist = run_soft(torch, x, P)
+    assert np.array_equal(idx, ref_idx) and np.array_equal(hist, ref_hist)
+    assert int(ref_hist[0]) > 0 and int(ref_hist[-1]) > 0          # both edges of the index set are reached
+    assert_soft_close(y, oracle.soft(x, f32(q), lo, hi, f32(alpha)), q)
+    gx, gq, ga = run_backward(torch, x, g, P)
+    assert_backward_close(gx, gq, ga, oracle.backward(x, g, f32(q), lo, hi, f32(alpha)), g, q, alpha)
+    # rate term: probabilities from the tensor's own histogram, floored so that empty levels stay finite
+    probs = (ref_hist.astype(np.float64) + 1.0) / float(ref_hist.sum() + nlev)
+    probs32 = probs.astype(f32).astype(np.float64)
+    Pr = cdl.QuantParams(q, lo, hi, alpha, 0.02, dev(torch, probs.astype(f32)))
+    gx, gq, ga = run_backward(torch, x, g, Pr)
+    ref = oracle.backward(x, g, f32(q), lo, hi, f32(alpha), 0, f32(0.02), probs32)
+    assert_backward_close(gx, gq, ga, ref, g, q, alpha, 0.02, probs32)
