@@ -600,7 +600,8 @@ __device__ __forceinline__ PairOut lattice_finish(const QuantDev &P, const LatPa
     const float2 S = __fadd2_rn(s.A0, f2(1.0f));
     const float2 rS = make_float2(rcp_approx(S.x), rcp_approx(S.y));
     const float2 m1 = __fmul2_rn(s.A1, rS);
-    o.y = __ffma2_rn(s.kn, f2(q), __fmul2_rn(f2(q), m1));
+    // (0 * residual: zero for finite input; a NaN or infinite input, whose B was clamped above, still gives NaN)
+    o.y = __ffma2_rn(s.kn, f2(q), __ffma2_rn(f2(q), m1, __fmul2_rn(s.dh, f2(0.0f))));
     o.gx = o.tq = o.ta = f2(0.0f);
     if (MODE == MODE_BWD) {
         const float2 m2 = __fmul2_rn(s.A2, rS), m3 = __fmul2_rn(s.A3, rS);

@@ -399,3 +399,19 @@ def test_table_form_of_the_level_sums(torch, lo, hi, q, alpha):
     gx, gq, ga = run_backward(torch, x, g, Pr)
     ref = oracle.backward(x, g, f32(q), lo, hi, f32(alpha), 0, f32(0.02), probs32)
     assert_backward_close(gx, gq, ga, ref, g, q, alpha, 0.02, probs32)
+
+
+def test_table_form_non_finite_inputs_give_nan_and_leave_their_neighbours_alone(torch):
+    # the soft value of a NaN or infinite element is NaN (the header's contract); the three finite elements
+    # that share its 128-bit load and walk the levels with it are unaffected
+    lo, hi, q, alpha = -32, 31, 0.05, 20.0
+    x = (inputs.normal((4096,), 0.5, seed=77)).astype(f32)
+    bad = {5: np.nan, 130: np.inf, 2051: -np.inf}
+    for i, v in bad.items():
+        x[i] = v
+    y, idx, _ = run_soft(torch, x, cdl.QuantParams(q, lo, hi, alpha))
+    assert all(np.isnan(y[i]) for i in bad)
+    assert [int(idx[i]) for i in bad] == [lo, hi, lo]
+    ok = np.ones(x.size, dtype=bool)
+    ok[list(bad)] = False
+    assert_soft_close(y[ok], oracle.soft(x[ok], f32(q), lo, hi, f32(alpha)), q)
