@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
     ap.add_argument("--sweep-max-log2n", type=int, default=28)
+    ap.add_argument("--sweep-point", type=float, nargs=3, metavar=("L", "ALPHA", "LOG2N"),
+                    help="with --sweep: only this point of the grid (any L <= 127, any alpha), e.g. for a profiler capture")
     ap.add_argument("--gemm", type=int, nargs=3, metavar=("M", "K", "N"), action="append",
                     help="index-GEMM-only timing of the forward, dX and dW products for this shape (repeatable)")
     return ap.parse_args()
@@ -379,6 +381,11 @@ def run_sweep(args):
     pk, pk_kind = peaks()
     hbm = float(pk["hbm_gbs"])
     gen = torch.Generator(device="cuda").manual_seed(5)
+    grid_n = list(range(20, args.sweep_max_log2n + 1, 2))
+    grid_L, grid_alpha = (1, 3, 7, 15, 127), (1.0, 100.0, 1e4)
+    if args.sweep_point:
+        grid_L, grid_alpha, grid_n = (int(args.sweep_point[0]),), (float(args.sweep_point[1]),), [int(args.sweep_point[2])]
+        args.sweep_max_log2n = grid_n[0]
     nmax = 1 << args.sweep_max_log2n
     pick = torch.rand(nmax, device="cuda", generator=gen) < 0.5
     xn = torch.randn(nmax, device="cuda", generator=gen)
@@ -415,13 +422,13 @@ def run_sweep(args):
         return statistics.median(ts)
 
     rows = []
-    for log2n in range(20, args.sweep_max_log2n + 1, 2):
+    for log2n in grid_n:
         n = 1 << log2n
-        for L in (1, 3, 7, 15, 127):
+        for L in grid_L:
             hist = torch.zeros(2 * L + 1, dtype=torch.int64, device="cuda")
             lp = torch.full((2 * L + 1,), 1.0 / (2 * L + 1), dtype=torch.float32, device="cuda")
             lp[L] *= 1.5
-            for alpha in (1.0, 100.0, 1e4):
+            for alpha in grid_alpha:
                 P = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01)
                 Pr = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01, lp)
 
@@ -444,7 +451,7 @@ def run_sweep(args):
                           "soft_idx_hist": (9, mk("soft_idx_hist")), "sample_hist": (5, mk("sample_hist")),
                           "backward": (12, mk("backward")),
                           "backward_rate": (12, mk("backward", Pr))}
-                if alpha != 1.0:
+                if alpha != grid_alpha[0]:
                     passes.pop("hard"), passes.pop("hard_hist")      # the hard passes do not depend on alpha
                 for name, (bpe, make) in passes.items():
                     ms = timed(make, n)

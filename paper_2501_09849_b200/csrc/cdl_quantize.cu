@@ -34,7 +34,8 @@
 //          tolerance), while beta = 2^B - 1 keeps it to full relative precision.  The four elements of a load
 //          walk the levels together on the packed instructions, the levels above and below kn separately and
 //          outwards.  Taken when the window of +-jmax levels is narrower than the index set and no rate term is
-//          asked for (1.3x the LOOP form on the soft pass, 1.4x on the backward pass).
+//          asked for, by the warps all of whose elements have jmax levels on either side (the others take LOOP);
+//          1.3x the LOOP form on the soft pass, 1.4x on the backward pass.
 #include "cdl_internal.h"
 
 #include <math.h>
@@ -496,10 +497,10 @@ struct LatPair {
     float2 A0, A1, A2, A3;          // sums over the levels other than kn of j^m e_j, m = 0..3
 };
 
-__device__ __forceinline__ void lattice_setup(const QuantDev &P, float2 x, LatPair &s)
+// hard indices of a pair (see quant_elem: reciprocal product, clamp, magic-number rounding, exact quotient near ties)
+__device__ __forceinline__ void lattice_index(const QuantDev &P, float2 x, LatPair &s)
 {
     const float q = P.q;
-    // hard index (see quant_elem): reciprocal product, clamp, magic-number rounding, exact quotient near ties
     float2 c = __fmul2_rn(x, f2(P.rq));
     if (!P.fast_div) c = make_float2(__fdiv_rn(x.x, q), __fdiv_rn(x.y, q));
     c.x = fminf(fmaxf(c.x, P.flo), P.fhi);
@@ -518,6 +519,12 @@ __device__ __forceinline__ void lattice_setup(const QuantDev &P, float2 x, LatPa
     s.kn = kn;
     s.k0 = __float_as_int(t.x) - kMagicBits;
     s.k1 = __float_as_int(t.y) - kMagicBits;
+}
+
+__device__ __forceinline__ void lattice_setup(const QuantDev &P, float2 x, LatPair &s)
+{
+    const float q = P.q;
+    const float2 kn = s.kn;
     s.dh = __ffma2_rn(kn, f2(-q), x);
     // B = 2 alpha q d log2 e, limited to +-64: beyond that the element lies far outside the index set and the
     // levels on the side that still exists weigh < 2^-64 either way
@@ -557,34 +564,19 @@ __device__ __forceinline__ void lattice_add(LatPair &s, float4 ga, float4 ha, fl
     }
 }
 
-// One side of the sums for both pairs: levels kn + DIR * j, j = 1 .. n (n0..n3 per element).
+// One side of the sums for both pairs: levels kn + DIR * j, j = 1 .. jmax (all of them inside the index set).
 template <bool BWD, int DIR>
 __device__ __forceinline__ void lattice_side(const float4 *__restrict__ Gtab, const float4 *__restrict__ Htab, LatPair &s0,
-                                             LatPair &s1, int n0, int n1, int n2, int n3)
+                                             LatPair &s1, int jmax)
 {
     const float2 one = f2(1.0f);
     const float2 b0 = DIR > 0 ? s0.bu : s0.bd, b1 = DIR > 0 ? s1.bu : s1.bd;
     float2 w0 = b0, w1 = b1;               // b^j - 1
-    const int nc = min(min(n0, n1), min(n2, n3)), nm = max(max(n0, n1), max(n2, n3));
-    int j = 1;
-    for (; j <= nc; ++j) {
+    for (int j = 1; j <= jmax; ++j) {
         const float4 ga = Gtab[j];
         const float4 ha = BWD ? Htab[j] : ga;
         lattice_add<BWD, DIR>(s0, ga, ha, __fadd2_rn(w0, one));
         lattice_add<BWD, DIR>(s1, ga, ha, __fadd2_rn(w1, one));
-        w0 = __fadd2_rn(w0, __ffma2_rn(w0, b0, b0));
-        w1 = __fadd2_rn(w1, __ffma2_rn(w1, b1, b1));
-    }
-    for (; j <= nm; ++j) {                 // elements with fewer levels on this side add zeros
-        const float4 ga = Gtab[j];
-        const float4 ha = BWD ? Htab[j] : ga;
-        float2 u0 = __fadd2_rn(w0, one), u1 = __fadd2_rn(w1, one);
-        u0.x = (j <= n0) ? u0.x : 0.0f;
-        u0.y = (j <= n1) ? u0.y : 0.0f;
-        u1.x = (j <= n2) ? u1.x : 0.0f;
-        u1.y = (j <= n3) ? u1.y : 0.0f;
-        lattice_add<BWD, DIR>(s0, ga, ha, u0);
-        lattice_add<BWD, DIR>(s1, ga, ha, u1);
         w0 = __fadd2_rn(w0, __ffma2_rn(w0, b0, b0));
         w1 = __fadd2_rn(w1, __ffma2_rn(w1, b1, b1));
     }
@@ -617,19 +609,17 @@ __device__ __forceinline__ PairOut lattice_finish(const QuantDev &P, const LatPa
     return o;
 }
 
+// the four elements of a load whose hard indices s0, s1 already hold; all four have jmax levels on either side
 template <int MODE>
 __device__ __forceinline__ void quant_quad_lattice(const QuantDev &P, const float4 *__restrict__ Gtab,
                                                    const float4 *__restrict__ Htab, const float (&xs)[4],
-                                                   const float (&gs)[4], PairOut (&o)[2])
+                                                   const float (&gs)[4], LatPair &s0, LatPair &s1, PairOut (&o)[2])
 {
     constexpr bool kBwd = MODE == MODE_BWD;
-    LatPair s0, s1;
     lattice_setup(P, make_float2(xs[0], xs[1]), s0);
     lattice_setup(P, make_float2(xs[2], xs[3]), s1);
-    lattice_side<kBwd, 1>(Gtab, Htab, s0, s1, min(P.hi - s0.k0, P.jmax), min(P.hi - s0.k1, P.jmax),
-                          min(P.hi - s1.k0, P.jmax), min(P.hi - s1.k1, P.jmax));
-    lattice_side<kBwd, -1>(Gtab, Htab, s0, s1, min(s0.k0 - P.lo, P.jmax), min(s0.k1 - P.lo, P.jmax),
-                           min(s1.k0 - P.lo, P.jmax), min(s1.k1 - P.lo, P.jmax));
+    lattice_side<kBwd, 1>(Gtab, Htab, s0, s1, P.jmax);
+    lattice_side<kBwd, -1>(Gtab, Htab, s0, s1, P.jmax);
     o[0] = lattice_finish<MODE>(P, s0, make_float2(gs[0], gs[1]));
     o[1] = lattice_finish<MODE>(P, s1, make_float2(gs[2], gs[3]));
 }
@@ -770,9 +760,22 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 unsigned int packed = 0u;
                 constexpr bool kPairs = (PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE))) ||
                                         (PATH == PATH_LATTICE && !RATE && (MODE == MODE_BWD || MODE == MODE_SOFT));
-                if (kPairs) {
-                    PairOut quad[2];
-                    if (PATH == PATH_LATTICE) quant_quad_lattice<MODE>(P, Gtab, Htab, xs, gs, quad);
+                // LATTICE: the table form serves a warp all of whose elements have jmax levels on either side of
+                // their nearest one; a warp with an element near the edge of the index set (or outside it) takes
+                // the level loop, which visits exactly each element's levels
+                bool use_pairs = kPairs;
+                PairOut quad[2];
+                if (PATH == PATH_LATTICE && kPairs) {
+                    LatPair s0, s1;
+                    lattice_index(P, make_float2(xs[0], xs[1]), s0);
+                    lattice_index(P, make_float2(xs[2], xs[3]), s1);
+                    const int klo = P.lo + P.jmax, khi = P.hi - P.jmax;
+                    const bool inner = min(min(s0.k0, s0.k1), min(s1.k0, s1.k1)) >= klo &&
+                                       max(max(s0.k0, s0.k1), max(s1.k0, s1.k1)) <= khi;
+                    use_pairs = __all_sync(__activemask(), inner);
+                    if (use_pairs) quant_quad_lattice<MODE>(P, Gtab, Htab, xs, gs, s0, s1, quad);
+                }
+                if (kPairs && use_pairs) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const float2 xp = make_float2(xs[2 * h], xs[2 * h + 1]), gp = make_float2(gs[2 * h], gs[2 * h + 1]);
@@ -808,7 +811,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     }
                 }
 #pragma unroll
-                for (int c = 0; c < ((kPairs || MODE == MODE_HARD) ? 0 : 4); ++c) {
+                for (int c = 0; c < (((kPairs && PATH != PATH_LATTICE) || MODE == MODE_HARD) ? 0 : 4); ++c) {
+                    if (kPairs && use_pairs) break;      // (only LATTICE decides this at run time; the bound stays constant)
                     const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
                     ys[c] = o.y;
                     gxs[c] = o.gx;
@@ -968,11 +972,13 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     unsigned char *ib = static_cast<unsigned char *>(idx);
     const int path = qd.near3 ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
     const bool rate = (mode == MODE_BWD) && qd.level_prob != nullptr && qd.rate_c != 0.0f;
-    // Whole index set, levels within jmax steps on both sides for most elements (2 jmax + 1 < nlev), vector region
-    // present, no soft histogram and no rate term: the table form of the level sums.  (When the index set is
-    // narrower than the window, an element's levels lie mostly on one side of it, a warp walks both sides to the
-    // longest lane's end, and the form loses what it gains; with the rate term it was no faster either.)
-    const bool lattice = path == PATH_LOOP && qd.window == 0 && n4 > 0 && 2 * qd.jmax + 1 < qd.nlev && !rate &&
+    // Whole index set, a window of +-jmax levels that is narrower than the index set and wide enough to pay for the
+    // per-element set-up (jmax >= 8), vector region present, no soft histogram and no rate term: the table form of
+    // the level sums for the warps whose elements all lie jmax levels inside the index set.  (Measured: with the
+    // rate term - two more per-lane table loads per level - it was no faster; letting elements near the edges take
+    // part, with per-element level counts and masks, made a warp walk both sides to its longest lane's end and
+    // lost more than it gained on heavy-tailed data.)
+    const bool lattice = path == PATH_LOOP && qd.window == 0 && n4 > 0 && qd.jmax >= 8 && 2 * qd.jmax + 1 < qd.nlev && !rate &&
                          ((mode == MODE_SOFT && soft_hist == nullptr) || mode == MODE_BWD);
 #define CDL_Q(M, PTH, RT) \
     launch_t<M, PTH, RT>(qd, x, grad_out, n, head, n4, y, ib, hist, grad_x, grad_q, grad_alpha, soft_hist, stream)

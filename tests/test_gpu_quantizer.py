@@ -374,14 +374,19 @@ def test_three_level_path_on_both_sides_of_the_residual_switch(torch, aq2, lo, h
 def test_table_form_of_the_level_sums(torch, lo, hi, q, alpha):
     # The soft and backward passes over the whole index set when levels further than jmax steps from the nearest
     # one carry no weight and 2 jmax + 1 < nlev: level weights G_j b^j from a table and a recurrence instead of
-    # one exponential per level.  Data: a normal/Laplace mixture wide enough that some elements sit at the edges
-    # of the index set (levels on one side only) and far outside it; rate term with non-uniform level
+    # one exponential per level, for the warps whose elements all lie jmax levels inside the index set.  Data:
+    # half of the tensor near the middle of the index set, half a normal/Laplace mixture wide enough that some
+    # elements sit at the edges (levels on one side only) and far outside; rate term with non-uniform level
     # probabilities; an element count that leaves a scalar tail.
     n = (1 << 17) + 3
     x = (inputs.normal_laplace_mixture((n,), seed=lo + 300) * f32(0.45 * hi * q)).astype(f32)
     if lo == 0:
         x = np.maximum(x, f32(0.0)) + (x < 0) * f32(-0.02) * (np.arange(n) % 7 == 0)
         x = x.astype(f32)
+    # first half: within three levels of the middle of the index set, so that whole warps are far from its edges
+    # (the table form is taken warp by warp); second half: the wide data, edges and outliers included
+    mid = 0.5 * (lo + hi) * q
+    x[: n // 2] = (mid + np.clip(inputs.normal((n // 2,), 1.5 * q, seed=hi + 500), -3.0 * q, 3.0 * q)).astype(f32)
     g = inputs.normal((n,), 1.0, seed=hi + 400)
     nlev = hi - lo + 1
     ref_idx, ref_hist = oracle.hard(x, f32(q), lo, hi)
@@ -402,10 +407,10 @@ def test_table_form_of_the_level_sums(torch, lo, hi, q, alpha):
 
 
 def test_table_form_non_finite_inputs_give_nan_and_leave_their_neighbours_alone(torch):
-    # the soft value of a NaN or infinite element is NaN (the header's contract); the three finite elements
-    # that share its 128-bit load and walk the levels with it are unaffected
+    # the soft value of a NaN or infinite element is NaN (the header's contract); the finite elements of its
+    # warp, which takes the level loop because of it while the other warps take the table form, are unaffected
     lo, hi, q, alpha = -32, 31, 0.05, 20.0
-    x = (inputs.normal((4096,), 0.5, seed=77)).astype(f32)
+    x = np.clip(inputs.normal((4096,), 0.1, seed=77), -0.2, 0.2).astype(f32)     # |index| <= 4: far from the edges
     bad = {5: np.nan, 130: np.inf, 2051: -np.inf}
     for i, v in bad.items():
         x[i] = v
