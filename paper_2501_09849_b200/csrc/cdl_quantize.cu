@@ -15,7 +15,7 @@
 //   rate term   = rate_weight * (-2 alpha q) * Cov(L, J),  L = log2 of the level probability.
 // The re-centred forms equal the printed ones (expand X = q (kn + J)) without their cancellation.
 //
-// Three evaluation paths, chosen per launch from alpha q^2 and the window (both uniform over the tensor):
+// Four evaluation paths, chosen per launch from alpha q^2 and the window (both uniform over the tensor):
 //   NEAR3  alpha q^2 > 12: levels two or more steps from the nearest one weigh < e^-24; only kn-1, kn, kn+1 are
 //          summed.  Here d must be exact next to the midpoints (dQ_d/dtheta ~ alpha q^2 / 2 there), so d is
 //          carried as an unevaluated sum dh + dl of two floats: k0 q is split exactly with one fma and
