@@ -839,7 +839,7 @@ def main():
                        "alpha": case.wq.alpha, "rate_weight": case.wq.rate_weight, "window_x": case.aq.window,
                        "l2": ("per-step working set is several times the 126 MB L2 (inputs larger than L2)"
                               if step_bytes > 2 * 126e6 else
-                              "per-step working set (%.0f MB) fits the 126 MB L2: a parity-size workload, not a bandwidth figure" % (step_bytes / 1e6)),
+                              "a step moves %.0f MB in all, of the order of the 126 MB L2: a parity-size workload, not a bandwidth figure" % (step_bytes / 1e6)),
                        "parallelism": f"replicas x{world}, all-reduce of dW / histogram / scalars" if world > 1 else "single GPU"},
             "layer_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": 6.0 * M * K * N / (gemm_ms * 1e-3) / 1e12,
             "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": quant_elems / (quant_ms * 1e-3) / 1e9,
