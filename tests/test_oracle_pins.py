@@ -292,6 +292,55 @@ def test_backward_is_the_gradient_proxy_of_the_partials():
     assert out["abs_alpha"] == pytest.approx(math.fsum(np.abs(gd * dal)), rel=1e-12)
 
 
+def test_backward_term_magnitude_scales_two_level_closed_form():
+    # mag_q / mag_alpha (the floors of the reduced-sum tolerances) on levels {0, q}, where every moment is a
+    # logistic expression: E = q s, Var = q^2 s (1 - s), Skew_u = E X^3 - E X E X^2 = q^3 s (1 - s),
+    # s = sigma(alpha q (2 theta - q)).  A dropped 1/q, a missing term or a lost absolute value fails here.
+    q, alpha = f32(0.5), f32(6.0)
+    x = np.linspace(-0.5, 1.0, 31).astype(f32)
+    g = inputs.normal((31,), 1.0, seed=21)
+    out = oracle.backward(x, g, q, 0, 1, alpha)
+    qq, al, th, ag = float(q), float(alpha), x.astype(np.float64), np.abs(g.astype(np.float64))
+    s = 1.0 / (1.0 + np.exp(-al * qq * (2.0 * th - qq)))
+    v = s * (1.0 - s)
+    mag_q = math.fsum(ag * (qq * s + np.abs(2.0 * al * th) * qq * qq * v + 2.0 * al * qq ** 3 * v) / qq)
+    mag_alpha = math.fsum(ag * (np.abs(2.0 * th) * qq * qq * v + qq ** 3 * v))
+    assert out["mag_q"] == pytest.approx(mag_q, rel=1e-11)
+    assert out["mag_alpha"] == pytest.approx(mag_alpha, rel=1e-11)
+    # the three terms have mixed signs on this grid (theta < 0 and theta > 0), so the scales strictly exceed
+    # the sums of |g * partial| and those exceed the signed sums
+    assert out["mag_q"] > out["abs_q"] > abs(out["grad_q"])
+    assert out["mag_alpha"] > out["abs_alpha"] > abs(out["grad_alpha"])
+
+
+@pytest.mark.parametrize("window", (0, 5))
+def test_backward_term_magnitude_scales_from_the_cpmf(window):
+    # General alphabets: the three terms of Eq. (9b) and the two of dQ_d/dalpha rebuilt from the CPMF itself
+    # (moments taken with numpy), and the identities  term sums = partials  that tie them to Lemma 1.
+    x = inputs.normal((257,), 0.08, seed=12)
+    g = inputs.normal((257,), 1.0, seed=13)
+    q, lo, hi, al = f32(0.02), -7, 7, f32(50.0)
+    out = oracle.backward(x, g, q, lo, hi, al, window)
+    _, dq, dal, _ = oracle.partials(x, q, lo, hi, al, window)
+    qq, a = float(q), float(al)
+    lev = np.arange(lo, hi + 1, dtype=np.float64) * qq
+    mq, ma = [], []
+    for e in range(x.size):
+        th, ge = float(x[e]), abs(float(g[e]))
+        P = oracle.cpmf(th, qq, lo, hi, a, window)
+        E = float(P @ lev)
+        var = float(P @ (lev - E) ** 2)
+        sk = float(P @ lev ** 3) - E * float(P @ lev ** 2)
+        t_q = (E, 2.0 * a * th * var, -2.0 * a * sk)
+        t_a = (2.0 * th * var, -sk)
+        assert sum(t_q) / qq == pytest.approx(dq[e], rel=1e-9, abs=1e-12)
+        assert sum(t_a) == pytest.approx(dal[e], rel=1e-9, abs=1e-15)
+        mq.append(ge * sum(abs(t) for t in t_q) / qq)
+        ma.append(ge * sum(abs(t) for t in t_a))
+    assert out["mag_q"] == pytest.approx(math.fsum(mq), rel=1e-11)
+    assert out["mag_alpha"] == pytest.approx(math.fsum(ma), rel=1e-11)
+
+
 def test_backward_zero_rate_weight_and_uniform_probabilities_add_nothing():
     x = inputs.normal((300,), 0.06, seed=8)
     g = inputs.normal((300,), 1.0, seed=9)
