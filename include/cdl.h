@@ -11,9 +11,12 @@
  * Conventions common to every entry point
  *  - Pointers marked [dev] are device memory owned by the caller; [host] are
  *    host memory read during the call only.  The library allocates no device
- *    memory, keeps no state between calls (the built-in scratch of
- *    cdl_qlinear_bwd_dw_noalloc excepted) and never synchronises the device
- *    (cdl_workspace_status excepted): work is enqueued on `stream` (a
+ *    memory and never synchronises the device (cdl_workspace_status and
+ *    cdl_noalloc_status excepted).  What it keeps between calls is per-device
+ *    bookkeeping only (device properties, kernel attributes set once, the
+ *    address and contents of the built-in scratch of
+ *    cdl_qlinear_bwd_dw_noalloc): no result depends on earlier calls.
+ *    Work is enqueued on `stream` (a
  *    cudaStream_t passed as void*; NULL is the legacy default stream) and
  *    outputs are valid once the stream reaches it.
  *  - All matrices are row-major; leading dimensions are in elements.
@@ -277,19 +280,28 @@ size_t cdl_qlinear_bwd_fp_workspace_bytes(int32_t M, int32_t N, int32_t K);
  *   G_idx [dev] M x N int8 (ld ldg), A_idx [dev] M x K bytes (ld lda), dW [dev] K x N floats; alignment and
  *   leading-dimension rules as for cdl_qlinear_bwd.  The caller still owns inputs and output.
  *
- * Limit: K * N <= CDL_NOALLOC_MAX_DW_ELEMS, otherwise CDL_ERR_TOO_LARGE and nothing is launched.
+ * Limits: K * N <= CDL_NOALLOC_MAX_DW_ELEMS, otherwise CDL_ERR_TOO_LARGE; and M * max|a| * max|g| < 2^31 for the
+ * declared index ranges (the sum over M must fit the int32 accumulators: there is no room here for the per-part
+ * slabs with which cdl_qlinear_bwd sums longer reductions in int64), otherwise CDL_ERR_OVERFLOW_RISK - for
+ * indices 0..15 against -127..127 that is M <= 1,127,287 rows.  In both cases nothing is launched.  Within the
+ * limits the values are those of cdl_qlinear_bwd, bit for bit.
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  * Set-up: the first call on each device (with that device current) looks up the array's device address;
  * make that first call before any stream capture begins.
  * Sharing: all calls on a device use the same array, which still holds the previous call's contents; the
  * call clears what it needs before use.  Two calls whose GPU work can overlap (different streams, no
- * dependency) race on it: serialise them.  A device-side timeout is recorded only in the library's own
- * status word and is not reported by this entry point.
+ * dependency) race on it: serialise them.  A bounded device-side wait that expires is recorded in the array's
+ * status block; cdl_noalloc_status reads it.
  */
 #define CDL_NOALLOC_MAX_DW_ELEMS (1 << 20)
 int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
                                const void *A_idx, int64_t lda, const cdl_index_desc *a,
                                int32_t M, int32_t N, int32_t K, float *dW, void *stream);
+
+/* cdl_workspace_status for the built-in scratch of cdl_qlinear_bwd_dw_noalloc on the current device: synchronises
+ * `stream`, returns CDL_ERR_TIMEOUT (and clears the record) when a wait of such a call gave up, else CDL_OK.
+ * Allocates nothing.  (No counterpart in the paper.) */
+int cdl_noalloc_status(void *stream);
 
 /*
  * The same three layer products for a convolutional layer (the layers of the paper's networks, Sec. VI-C and
@@ -351,8 +363,9 @@ size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K);
 
 /* Synchronises `stream` and reports whether a bounded device-side wait of a GEMM call that used this workspace
  * gave up: CDL_ERR_TIMEOUT (the outputs of that call are then undefined; the record is cleared by this call) or
- * CDL_OK.  The GEMM calls never touch the first word of a workspace unless a wait expires, in which case they
- * store CDL_ERR_TIMEOUT there and it stays until read here; any other content (a fresh allocation) reads as OK. */
+ * CDL_OK.  The GEMM calls never touch the status block (the first 16 bytes of a workspace) unless a wait expires, in
+ * which case they store a record there - CDL_ERR_TIMEOUT followed by two tag words - that stays until read here;
+ * any other content, such as whatever a fresh or recycled allocation holds, reads as OK. */
 int cdl_workspace_status(void *ws, void *stream);
 
 /* Static, NUL-terminated description of a status code. */

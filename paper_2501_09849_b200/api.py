@@ -12,7 +12,7 @@ from pathlib import Path
 __all__ = [
     "CdlError", "QuantParams", "IndexDesc", "library_path", "load_library",
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
-    "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc",
+    "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_noalloc_status",
     "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
     "cdl_huffman_lengths", "cdl_qconv_bwd_fp", "cdl_qconv_bwd_fp_workspace_bytes", "cdl_qlinear_bwd_fp", "cdl_qlinear_bwd_fp_workspace_bytes", "cdl_qlinear_fwd_next", "cdl_qconv_fwd_next", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
@@ -117,6 +117,8 @@ def load_library():
     lib.cdl_workspace_bytes.argtypes = [I32, I32, I32, I32]
     lib.cdl_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_status.argtypes = [P, P]
+    lib.cdl_noalloc_status.argtypes = [P]
+    lib.cdl_noalloc_status.restype = C.c_int
     for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample", "cdl_index_entropy",
                  "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status",
                  "cdl_qconv_fwd", "cdl_qconv_bwd"):
@@ -323,3 +325,10 @@ def cdl_qlinear_bwd_dw_noalloc(G_idx, ldg, g: IndexDesc, A_idx, lda, a: IndexDes
     rc = load_library().cdl_qlinear_bwd_dw_noalloc(_ptr(G_idx), ldg, C.byref(gc), _ptr(A_idx), lda, C.byref(ac), M, N, K,
                                                    _ptr(dW), _stream(stream))
     return _check(rc, "cdl_qlinear_bwd_dw_noalloc", check)
+
+
+def cdl_noalloc_status(stream=None, check=True):
+    """Synchronises the stream and reports a device-side timeout of the last cdl_qlinear_bwd_dw_noalloc call on the
+    current device (the record lives in the library's built-in scratch); allocates nothing."""
+    rc = load_library().cdl_noalloc_status(_stream(stream))
+    return _check(rc, "cdl_noalloc_status", check)

@@ -42,7 +42,6 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     cmd = [nvcc, *NVCC_FLAGS, "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("CDL_EXTRA_NVCC_FLAGS", "").split()
     cmd += ["-o", str(tmp), *map(str, sources())]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)

@@ -34,6 +34,21 @@ int check_device()
     return g_dev_ok[dev] == 1 ? CDL_OK : CDL_ERR_UNSUPPORTED;
 }
 
+int read_status_block(void *block, cudaStream_t st)
+{
+    int32_t words[3] = {0, 0, 0};
+    if (cudaMemcpyAsync(words, block, sizeof words, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    // kernels write nothing but a complete record into the block; anything else (a fresh allocation) is "no record"
+    if (words[0] != CDL_ERR_TIMEOUT || (unsigned int)words[1] != kStatusTag1 || (unsigned int)words[2] != kStatusTag2)
+        return CDL_OK;
+    if (cudaMemsetAsync(block, 0, sizeof words, st) != cudaSuccess) (void)cudaGetLastError();
+    return CDL_ERR_TIMEOUT;
+}
+
 int sm_count()
 {
     int dev = 0;
@@ -262,16 +277,7 @@ size_t cdl_workspace_bytes(int32_t op, int32_t M, int32_t N, int32_t K)
 int cdl_workspace_status(void *ws, void *stream)
 {
     if (ws == nullptr) return CDL_ERR_WORKSPACE;
-    int32_t word = 0;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(&word, ws, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return CDL_ERR_LAUNCH;
-    }
-    if (word != CDL_ERR_TIMEOUT) return CDL_OK;     // kernels write nothing but this code into the word
-    if (cudaMemsetAsync(ws, 0, sizeof word, st) != cudaSuccess) (void)cudaGetLastError();
-    return CDL_ERR_TIMEOUT;
+    return read_status_block(ws, static_cast<cudaStream_t>(stream));
 }
 
 namespace {
@@ -469,6 +475,39 @@ int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx,
                               stream);
 }
 
+namespace {
+// Argument checks of the backward convolution products (everything but the workspace): CDL_OK, or the status the
+// entry point returns before anything is enqueued.
+int check_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
+                    const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
+                    const int32_t *dXacc, const float *dX, const int32_t *dWacc, const float *dW, int64_t *M_out,
+                    int *taps_out, cdl::IndexRange *rg, cdl::IndexRange *rx, cdl::IndexRange *rw)
+{
+    using namespace cdl;
+    const bool want_dx = dXacc != nullptr || dX != nullptr;
+    const bool want_dw = dWacc != nullptr || dW != nullptr;
+    if (G_idx == nullptr || !conv_dims(shape, C_out, M_out, taps_out)) return CDL_ERR_ARG;
+    if (!want_dx && !want_dw) return CDL_ERR_ARG;
+    if ((want_dx && W_idx == nullptr) || (want_dw && X_idx == nullptr)) return CDL_ERR_ARG;
+    if (want_dx && ldw < C_out) return CDL_ERR_ARG;
+    int rc;
+    if ((rc = index_range(g, rg)) != CDL_OK) return rc;
+    if (rg->is_unsigned && g->hi > 127) return CDL_ERR_RANGE;
+    if (want_dw && (rc = index_range(x, rx)) != CDL_OK) return rc;
+    if (want_dx) {
+        if ((rc = index_range(w, rw)) != CDL_OK) return rc;
+        if (rw->is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+    }
+    if (reinterpret_cast<uintptr_t>(G_idx) & 15u) return CDL_ERR_ALIGN;
+    if (want_dw && (reinterpret_cast<uintptr_t>(X_idx) & 15u)) return CDL_ERR_ALIGN;
+    if (want_dx && ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))) return CDL_ERR_ALIGN;
+    if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    if (dXacc != nullptr && overflow_risk((int64_t)*taps_out * C_out, *rg, *rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (dWacc != nullptr && overflow_risk(*M_out, *rx, *rg)) return CDL_ERR_OVERFLOW_RISK;
+    return CDL_OK;
+}
+}  // namespace
+
 int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
                   const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
                   int32_t *dXacc, float *dX, int32_t *dWacc, float *dW, void *ws, size_t ws_bytes, void *stream)
@@ -477,27 +516,11 @@ int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx,
     const bool want_dw = dWacc != nullptr || dW != nullptr;
     int64_t M;
     int taps;
-    if (G_idx == nullptr || !conv_dims(shape, C_out, &M, &taps)) return CDL_ERR_ARG;
-    if (!want_dx && !want_dw) return CDL_ERR_ARG;
-    if ((want_dx && W_idx == nullptr) || (want_dw && X_idx == nullptr)) return CDL_ERR_ARG;
-    if (want_dx && ldw < C_out) return CDL_ERR_ARG;
     IndexRange rg, rx{false, 0}, rw{false, 0};
-    int rc;
-    if ((rc = index_range(g, &rg)) != CDL_OK) return rc;
-    if (rg.is_unsigned && g->hi > 127) return CDL_ERR_RANGE;
-    if (want_dw && (rc = index_range(x, &rx)) != CDL_OK) return rc;
-    if (want_dx) {
-        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
-        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
-    }
-    if (reinterpret_cast<uintptr_t>(G_idx) & 15u) return CDL_ERR_ALIGN;
-    if (want_dw && (reinterpret_cast<uintptr_t>(X_idx) & 15u)) return CDL_ERR_ALIGN;
-    if (want_dx && ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))) return CDL_ERR_ALIGN;
-    if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    int rc = check_qconv_bwd(G_idx, g, X_idx, x, W_idx, ldw, w, shape, C_out, dXacc, dX, dWacc, dW, &M, &taps, &rg, &rx, &rw);
+    if (rc != CDL_OK) return rc;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_workspace_bytes(shape, C_out))
         return CDL_ERR_WORKSPACE;
-    if (dXacc != nullptr && overflow_risk((int64_t)taps * C_out, rg, rw)) return CDL_ERR_OVERFLOW_RISK;
-    if (dWacc != nullptr && overflow_risk(M, rx, rg)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (want_dx) {
@@ -544,13 +567,27 @@ int cdl_qlinear_bwd_fp(const float *G, float g_absmax, const void *A_idx, int64_
     if (bad_f32_ptr(G)) return CDL_ERR_ALIGN;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qlinear_bwd_fp_workspace_bytes(M, N, K))
         return CDL_ERR_WORKSPACE;
+    // every argument is checked before the first operation is enqueued
+    IndexRange rg{false, 127}, ra{false, 0}, rw{false, 0};
+    int rc;
+    if (dW != nullptr && (rc = index_range(a, &ra)) != CDL_OK) return rc;
+    if (dX != nullptr) {
+        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
+        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
+        if (ldw < N) return CDL_ERR_ARG;
+        if ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u)) return CDL_ERR_ALIGN;
+    }
+    if (dW != nullptr) {
+        if (lda < K) return CDL_ERR_ARG;
+        if ((lda & 15) || (reinterpret_cast<uintptr_t>(A_idx) & 15u)) return CDL_ERR_ALIGN;
+    }
+    if (bad_f32_ptr(dX) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
+    if ((rc = check_device()) != CDL_OK) return rc;
     const float q1 = g_absmax / 127.0f, q2 = q1 / 254.0f;
     const int64_t ldg = ld16(N);
     const size_t base = align256(cdl_workspace_bytes(CDL_OP_QLINEAR_BWD, M, N, K));
     const size_t plane = align256((size_t)M * (size_t)ldg);
     char *d1 = static_cast<char *>(ws) + base, *d2 = d1 + plane;
-    int rc = check_device();
-    if (rc != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ldg != N) {      // the pad columns are operands of the TMA loads: keep them defined
         if (cudaMemsetAsync(d1, 0, 2 * plane, st) != cudaSuccess) {
@@ -561,15 +598,6 @@ int cdl_qlinear_bwd_fp(const float *G, float g_absmax, const void *A_idx, int64_
     if ((rc = launch_gradient_digits(G, M, N, (int)ldg, q1, q2, d1, d2, st)) != CDL_OK) return rc;
     const cdl_index_desc g1{q1, -127, 127}, g2{q2, -127, 127};
     // first digit stores, second digit adds: dX = RN(RN(acc1 s1) + RN(acc2 s2))
-    IndexRange rg{false, 127}, ra{false, 0}, rw{false, 0};
-    if (dW != nullptr && (rc = index_range(a, &ra)) != CDL_OK) return rc;
-    if (dX != nullptr) {
-        if ((rc = index_range(w, &rw)) != CDL_OK) return rc;
-        if (rw.is_unsigned && w->hi > 127) return CDL_ERR_RANGE;
-        if ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u) || ldw < N) return CDL_ERR_ALIGN;
-    }
-    if (dW != nullptr && ((lda & 15) || (reinterpret_cast<uintptr_t>(A_idx) & 15u) || lda < K)) return CDL_ERR_ALIGN;
-    if (bad_f32_ptr(dX) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
     char *scratch = static_cast<char *>(ws) + kStatusBytes;
     for (int pass = 0; pass < 2; ++pass) {
         const char *dig = pass == 0 ? d1 : d2;
@@ -615,8 +643,18 @@ int cdl_qconv_bwd_fp(const float *G, float g_absmax, const void *X_idx, const cd
     const size_t base = align256(cdl_qconv_workspace_bytes(shape, C_out));
     const size_t plane = align256((size_t)M * (size_t)C_out);
     char *d1 = static_cast<char *>(ws) + base, *d2 = d1 + plane;
-    int rc = check_device();
-    if (rc != CDL_OK) return rc;
+    // every argument is checked before the first operation is enqueued (the digit planes stand in for G_idx)
+    int rc;
+    {
+        const cdl_index_desc gd{q1, -127, 127};
+        IndexRange cg_, cx_{false, 0}, cw_{false, 0};
+        int64_t M2;
+        int taps2;
+        if (!(q1 > 0.0f) || !(q2 > 0.0f)) return CDL_ERR_RANGE;
+        rc = check_qconv_bwd(d1, &gd, X_idx, x, W_idx, ldw, w, shape, C_out, nullptr, dX, nullptr, dW, &M2, &taps2, &cg_, &cx_, &cw_);
+        if (rc != CDL_OK) return rc;
+    }
+    if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((rc = launch_gradient_digits(G, M, C_out, C_out, q1, q2, d1, d2, st)) != CDL_OK) return rc;
     // each digit plane is a gradient index tensor of its own step: the first pass stores, the second adds.  The

@@ -32,7 +32,10 @@
 // Every wait is bounded: on expiry the kernel records CDL_ERR_TIMEOUT in the status word and winds down.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "cdl_internal.h"
+#include "cdl_wait.cuh"
 
 namespace cdl {
 namespace {
@@ -40,10 +43,7 @@ namespace {
 // Epilogue warps per CTA: kEpiWarps / 4 per TMEM lane quarter, taking the 32-column chunks in turn.  Products whose
 // time is the epilogue's (two stages of loads per 256 KB of output) get twice as many, with one chunk in flight each.
 __host__ __device__ constexpr int epi_warps(bool store_heavy) { return store_heavy ? 16 : 8; }
-#ifndef CDL_G_SPLIT_PRODUCER
-#define CDL_G_SPLIT_PRODUCER 1
-#endif
-constexpr bool kSplitProducer = CDL_G_SPLIT_PRODUCER != 0;   // a second TMA warp issues the Y-operand loads
+constexpr bool kSplitProducer = true;   // a second TMA warp issues the Y-operand loads
 __host__ __device__ constexpr int threads_tc(bool store_heavy) { return 64 + 32 * epi_warps(store_heavy) + (kSplitProducer ? 32 : 0); }
 // Shared memory is divided between operand stages and epilogue staging blocks (4 KB each, per epilogue warp).
 // Which of the two needs the bytes in flight depends on the shape: a long reduced dimension loads much more than
@@ -63,13 +63,7 @@ constexpr int kOutWarpBytes = 32 * 128;  // epilogue staging block of one warp: 
 // allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
 constexpr int kSmemBytes = 232448 - 1024;
 constexpr int kPlanSMs = 148;           // B200: splits are planned for this count so that workspace sizes are fixed
-constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s
-#ifndef CDL_G_TRYWAIT_HINT_NS
-#define CDL_G_TRYWAIT_HINT_NS 20000
-#endif
-// Upper bound, in nanoseconds, on how long one try_wait may keep its thread suspended while the phase is pending:
-// a suspended poller leaves the issue slots of its scheduler to the epilogue warps that share it.
-constexpr unsigned int kTryWaitHintNs = CDL_G_TRYWAIT_HINT_NS;
+constexpr unsigned long long kWaitNs = 2000000000ull;  // limit of every device-side wait: 2 s
 
 struct TcParams {
     int I, J, R;            // rows the tiling runs over, output columns, reduced extent of the tiling
@@ -86,6 +80,7 @@ struct TcParams {
     int f_acc;              // 1: the float output is added to what f_out holds (one binary32 addition per element)
     const float *bias;
     int *status;
+    unsigned long long wait_ns;   // limit of each mbarrier wait
     int tma_f, tma_acc;     // the float / int32 output goes through shared memory and TMA
     // Implicit patch matrix (convolution): the X operand is gathered by TMA im2col loads from an [N,H,W,C] index
     // tensor instead of being read from a stored matrix.
@@ -105,51 +100,6 @@ struct TcParams {
 };
 
 // ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(kTryWaitHintNs)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: false when the barrier did not complete within kWaitNs or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    for (int fast = 0; fast < 64; ++fast)
-        if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag != 0) return false;
-        if (global_ns() - t0 > kWaitNs) return false;
-    }
-}
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
     asm volatile(
@@ -444,7 +394,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 for (int rb = rb0; rb < rb1; ++rb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.wait_ns)) {
                         failed = true;
                         break;
                     }
@@ -508,7 +458,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
             if (failed) {
                 abort_s = 1;
-                atomicExch(P.status, CDL_ERR_TIMEOUT);
+                record_timeout(P.status);
             }
         }
     } else if (warp == 1) {
@@ -521,7 +471,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
                 const int buf = tcount & 1;
                 const uint32_t tph = (tcount >> 1) & 1u;
-                if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag)) {
+                if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, P.wait_ns)) {
                     failed = true;
                     break;
                 }
@@ -530,7 +480,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 for (int rb = rb0; rb < rb1; ++rb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, P.wait_ns)) {
                         failed = true;
                         break;
                     }
@@ -561,7 +511,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
             if (failed) {
                 abort_s = 1;
-                atomicExch(P.status, CDL_ERR_TIMEOUT);
+                record_timeout(P.status);
             }
         }
     } else {
@@ -628,7 +578,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
             // the epilogue warps agree on the outcome, so that either all of them or none release the accumulator
-            if (!epi_all<32 * kEpiWarps>(mbar_wait(tfull_bar(buf), tph, abort_flag))) {
+            if (!epi_all<32 * kEpiWarps>(mbar_wait(tfull_bar(buf), tph, abort_flag, P.wait_ns))) {
                 failed = true;
                 break;
             }
@@ -733,7 +683,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (lane == 0) bulk_wait_all();             // staged blocks are out before shared memory goes away
         if (failed && lane == 0) {
             abort_s = 1;
-            atomicExch(P.status, CDL_ERR_TIMEOUT);
+            record_timeout(P.status);
         }
     }
 
@@ -997,6 +947,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.f_acc = accumulate_f ? 1 : 0;
     P.bias = bias;
     P.status = status;
+    P.wait_ns = kWaitNs;
     P.f_out = f_out;
     P.acc_out = acc_out;
     const long long n_out = (long long)I * J;
@@ -1123,7 +1074,7 @@ namespace {
 constexpr size_t kStaticStatusBytes = 256;
 constexpr size_t kStaticAccElems = CDL_NOALLOC_MAX_DW_ELEMS;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticStatusBytes + kStaticAccElems * sizeof(int32_t)];
-unsigned char *g_static_ptr[64];   // device address of g_static_scratch, per device
+std::atomic<unsigned char *> g_static_ptr[64];   // device address of g_static_scratch, per device
 }  // namespace
 
 extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const cdl_index_desc *g, const void *A_idx,
@@ -1149,16 +1100,18 @@ extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const 
     if (rc != CDL_OK) return rc;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
-    if (g_static_ptr[dev] == nullptr) {
-        // one-time set-up for this device (the device is current): resolve the array's device address
+    unsigned char *base = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (base == nullptr) {
+        // one-time set-up for this device (the device is current): resolve the array's device address; threads
+        // that race here all obtain the same address
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
             (void)cudaGetLastError();
             return CDL_ERR_LAUNCH;
         }
-        g_static_ptr[dev] = static_cast<unsigned char *>(p);
+        base = static_cast<unsigned char *>(p);
+        g_static_ptr[dev].store(base, std::memory_order_release);
     }
-    unsigned char *base = g_static_ptr[dev];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: clear the status word here; the accumulation buffer is
     // cleared by the launcher whenever the reduction is split
@@ -1170,4 +1123,14 @@ extern "C" int cdl_qlinear_bwd_dw_noalloc(const void *G_idx, int64_t ldg, const 
     GemmOperand Y{G_idx, 1, ldg, false, (int)gmax};
     return launch_index_gemm_tc(X, Y, K, N, M, nullptr, dW, g->q * a->q, nullptr, base + kStaticStatusBytes,
                                 reinterpret_cast<int *>(base), st, nullptr, nullptr, false, true);
+}
+
+extern "C" int cdl_noalloc_status(void *stream)
+{
+    using namespace cdl;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
+    unsigned char *base = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (base == nullptr) return CDL_OK;        // cdl_qlinear_bwd_dw_noalloc has not run on this device
+    return read_status_block(base, static_cast<cudaStream_t>(stream));
 }

@@ -34,6 +34,12 @@ struct QuantDev {
 
 enum QuantMode { MODE_HARD = 0, MODE_SOFT = 1, MODE_BWD = 2, MODE_SAMPLE = 3 };
 
+// A status block (first 16 bytes of a workspace, or of the built-in scratch) holds a timeout record when its first
+// word is CDL_ERR_TIMEOUT and the next two are these tags.
+constexpr unsigned int kStatusTag1 = 0x43444C54u, kStatusTag2 = 0x6F757421u;
+// Synchronises the stream, reads the block, clears a record if there is one; CDL_OK, CDL_ERR_TIMEOUT or CDL_ERR_LAUNCH.
+int read_status_block(void *block, cudaStream_t stream);
+
 int check_device();   // CDL_OK, CDL_ERR_UNSUPPORTED or CDL_ERR_LAUNCH
 int sm_count();       // multiprocessors of the current device (0 on error)
 int make_quant_dev(const cdl_quant_params *p, bool need_alpha, QuantDev *out);

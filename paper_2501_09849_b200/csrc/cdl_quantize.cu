@@ -43,28 +43,11 @@
 namespace cdl {
 namespace {
 
-// Launch shape (overridable at build time for tuning runs)
-#ifndef CDL_Q_THREADS
-#define CDL_Q_THREADS 256
-#endif
-#ifndef CDL_Q_BATCH
-#define CDL_Q_BATCH 2
-#endif
-#ifndef CDL_Q_MINBLOCKS
-#define CDL_Q_MINBLOCKS 1
-#endif
-#ifndef CDL_Q_PREFETCH
-#define CDL_Q_PREFETCH 0     // 1: the loads of the next iteration are issued before the arithmetic of this one
-#endif
-#ifdef CDL_Q_PLAIN_LDST
-#define CDL_LD(p) (*(p))
-#define CDL_ST(p, v) (*(p) = (v))
-#else
+constexpr int kThreads = 256;
+constexpr int kBatch = 2;            // float4 loads in flight per thread
+// streaming accesses: every element is touched once, so loads and stores bypass the usual cache retention
 #define CDL_LD(p) __ldcs(p)
 #define CDL_ST(p, v) __stcs(p, v)
-#endif
-constexpr int kThreads = CDL_Q_THREADS;
-constexpr int kBatch = CDL_Q_BATCH;  // float4 loads in flight per thread
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
 // |quotient - nearest integer| above this may be a rounding tie once the 3-ulp error of the reciprocal product is
@@ -632,7 +615,7 @@ __device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane
 // Vector region: elements [head, head + 4 n4); the remaining head + tail elements are done one by one.
 // When the pointers do not allow 128-bit access the host passes n4 = 0 and everything is scalar.
 template <int MODE, int PATH, bool RATE>
-__global__ void __launch_bounds__(kThreads, CDL_Q_MINBLOCKS)
+__global__ void __launch_bounds__(kThreads)
 quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__restrict__ g, int64_t n,
                 int64_t head, int64_t n4, float *__restrict__ y, unsigned char *__restrict__ idx,
                 unsigned long long *__restrict__ hist, float *__restrict__ gx,
@@ -694,31 +677,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     float4 *gx4 = reinterpret_cast<float4 *>(gx + head);
     unsigned int *idx4 = reinterpret_cast<unsigned int *>(idx + head);
 
-#if CDL_Q_PREFETCH
-    float4 xn[kBatch], gn[kBatch];
-#pragma unroll
-    for (int b = 0; b < kBatch; ++b) {
-        const int64_t i = tid + b * stride;
-        if (i < n4) {
-            xn[b] = CDL_LD(x4 + i);
-            if (MODE == MODE_BWD) gn[b] = CDL_LD(g4 + i);
-        }
-    }
-#endif
     for (int64_t base = tid; base < n4; base += stride * kBatch) {
         float4 xv[kBatch], gv[kBatch];
-#if CDL_Q_PREFETCH
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            xv[b] = xn[b];
-            if (MODE == MODE_BWD) gv[b] = gn[b];
-            const int64_t i = base + stride * kBatch + b * stride;
-            if (i < n4) {
-                xn[b] = CDL_LD(x4 + i);
-                if (MODE == MODE_BWD) gn[b] = CDL_LD(g4 + i);
-            }
-        }
-#else
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             const int64_t i = base + b * stride;
@@ -727,7 +687,6 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                 if (MODE == MODE_BWD) gv[b] = CDL_LD(g4 + i);
             }
         }
-#endif
         float part_q = 0.0f, part_a = 0.0f;
         float2 part_q2 = make_float2(0.0f, 0.0f), part_a2 = make_float2(0.0f, 0.0f);    // pair path: two running sums each
 #pragma unroll
@@ -970,7 +929,10 @@ int launch_quantize(int mode, const float *x, const float *grad_out, int64_t n, 
     if (n4 == 0) head = 0;
 
     unsigned char *ib = static_cast<unsigned char *>(idx);
-    const int path = qd.near3 ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
+    // NEAR3 sums the nearest level and its two neighbours whatever the window: right for the whole index set and for
+    // any window of three or more (what it leaves out weighs < e^-24), wrong for a window of one, which keeps the
+    // nearest level alone (zero variance and gradient): that one takes the level loop, which honours the window.
+    const int path = (qd.near3 && qd.window != 1) ? PATH_NEAR3 : (qd.window == 5 ? PATH_WIN5 : PATH_LOOP);
     const bool rate = (mode == MODE_BWD) && qd.level_prob != nullptr && qd.rate_c != 0.0f;
     // Whole index set, a window of +-jmax levels that is narrower than the index set and wide enough to pay for the
     // per-element set-up (jmax >= 8), vector region present, no soft histogram and no rate term: the table form of

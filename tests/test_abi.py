@@ -114,6 +114,33 @@ def test_qlinear_argument_errors_need_no_device(lib):
              ws_bytes=cdl.cdl_workspace_bytes(2, M, 128, 256), check=False) == OVF
 
 
+def test_real_gradient_products_check_every_argument_before_enqueueing(lib):
+    # Without a device any enqueue attempt would come back as a launch error: a range / alignment / argument status
+    # therefore shows that the check ran before the first memset or kernel launch.
+    D = cdl.IndexDesc
+    p, ws = 0x10000, 0x20000
+    a, w = D(0.25, 0, 15), D(0.02, -7, 7)
+    M, N, K = 64, 120, 256                     # N not a multiple of 16: the digit planes would be cleared first
+    nb = cdl.cdl_qlinear_bwd_fp_workspace_bytes(M, N, K)
+    f = cdl.cdl_qlinear_bwd_fp
+    assert f(p, 1.0, p, 256, D(0.25, 0, 300), p, 128, w, M, N, K, dW=p, ws=ws, ws_bytes=nb, check=False) == RANGE
+    assert f(p, 1.0, p, 256, D(0.25, 5, 1), p, 128, w, M, N, K, dW=p, ws=ws, ws_bytes=nb, check=False) == RANGE
+    assert f(p, 1.0, p, 264, a, p, 128, w, M, N, K, dW=p, ws=ws, ws_bytes=nb, check=False) == ALIGN      # lda % 16
+    assert f(p, 1.0, p, 240, a, p, 128, w, M, N, K, dW=p, ws=ws, ws_bytes=nb, check=False) == ARG        # lda < K
+    assert f(p, 1.0, p, 256, a, p, 128, D(0.02, 0, 200), M, N, K, dX=p, ws=ws, ws_bytes=nb, check=False) == RANGE
+    assert f(p, 1.0, p, 256, a, p + 8, 128, w, M, N, K, dX=p, ws=ws, ws_bytes=nb, check=False) == ALIGN
+    assert f(p, 1.0, p, 256, a, p, 112, w, M, N, K, dX=p, ws=ws, ws_bytes=nb, check=False) == ARG        # ldw < N
+    assert f(p, 1.0, p, 256, a, p, 128, w, M, N, K, dX=p + 2, ws=ws, ws_bytes=nb, check=False) == ALIGN
+    shape = cdl.ConvShape(2, 8, 8, 64, 3, 3)
+    nc = cdl.cdl_qconv_bwd_fp_workspace_bytes(shape, 64)
+    c = cdl.cdl_qconv_bwd_fp
+    assert c(p, 1.0, p, D(0.25, 0, 300), p, 64, w, shape, 64, dW=p, ws=ws, ws_bytes=nc, check=False) == RANGE
+    assert c(p, 1.0, p + 4, a, p, 64, w, shape, 64, dW=p, ws=ws, ws_bytes=nc, check=False) == ALIGN
+    assert c(p, 1.0, p, a, p, 72, w, shape, 64, dX=p, ws=ws, ws_bytes=nc, check=False) == ALIGN          # ldw % 16
+    assert c(p, 1.0, p, a, p, 48, w, shape, 64, dX=p, ws=ws, ws_bytes=nc, check=False) == ARG            # ldw < C_out
+    assert c(p, 1.0, p, a, p, 64, D(0.02, 0, 200), shape, 64, dX=p, ws=ws, ws_bytes=nc, check=False) == RANGE
+
+
 def test_missing_library_raises_instead_of_falling_back(monkeypatch, tmp_path):
     from paper_2501_09849_b200 import api
     monkeypatch.setattr(api, "_LIB", None)

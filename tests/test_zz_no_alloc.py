@@ -33,7 +33,7 @@ def test_noalloc_dw_matches_regular_entry_point_twice_in_a_row():
         for repeat in range(2):
             out = torch.full((K, N), -2.0, dtype=torch.float32, device="cuda")
             cdl.cdl_qlinear_bwd_dw_noalloc(G, N, g, A, K, a, M, N, K, out)
-            torch.cuda.synchronize()
+            assert cdl.cdl_noalloc_status() == 0          # synchronises; no device-side wait gave up
             assert torch.equal(out, ref), (M, K, N, repeat)
         # and against plain integer arithmetic on the host, so that both being wrong together cannot pass
         acc = A.cpu().numpy().astype(np.int64).T @ G.cpu().numpy().astype(np.int64)
@@ -50,3 +50,16 @@ def test_noalloc_dw_rejects_sizes_beyond_its_static_scratch():
     buf = torch.zeros(16, dtype=torch.uint8, device="cuda")
     rc = cdl.cdl_qlinear_bwd_dw_noalloc(buf, N, g, buf, K, a, M, N, K, buf, check=False)
     assert rc == -9 and "built-in scratch" in cdl.cdl_strerror(rc)
+
+
+def test_noalloc_dw_rejects_reductions_too_long_for_int32():
+    # cdl_qlinear_bwd cuts such a reduction into exact parts and sums them in int64 slabs; the built-in scratch has
+    # no room for slabs, so the entry point refuses (documented limit M * max|a| * max|g| < 2^31)
+    import torch
+    cdl.load_library()
+    a, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(1e-3, -127, 127)
+    buf = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    M_ok, M_bad = (1 << 31) // (15 * 127) - 16, ((1 << 31) // (15 * 127) // 16 + 1) * 16
+    assert M_bad * 15 * 127 >= 1 << 31 > M_ok * 15 * 127
+    rc = cdl.cdl_qlinear_bwd_dw_noalloc(buf, 16, g, buf, 16, a, M_bad, 16, 16, buf, check=False)
+    assert rc == -5 and "overflow" in cdl.cdl_strerror(rc)
