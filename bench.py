@@ -8,13 +8,17 @@ backward index GEMMs, and the analytic quantizer backward for activations and we
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl cdl|reference]
 
 Prints ONE JSON line (rank 0).  `value` counts the tensor elements that went through a quantizer pass per
-second of whole-step time, summed over ranks (each rank runs its own batch: weak scaling).
+second of whole-step time, summed over ranks (each rank runs its own batch: weak scaling).  On one GPU the same
+line also carries the rest of the metric: `sweep` (quantizer passes alone, 2^28 / 2^30 elements and the layer's own
+tensor size), `gemm` (the index GEMMs alone on the tensor-bound shapes) and `network` (the whole ResNet-18 step).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -29,16 +33,13 @@ if str(ROOT) not in sys.path:
 METRIC = "quantizer Gelem/s (% of HBM peak); CDL layer fwd+bwd ms and int8 TOPS"
 UNIT = "Gelem/s"
 G_STD = 1e-2                 # standard deviation of the synthetic dL/dY
-CPU_BASELINE_SECONDS = 20.0   # host time the cpu_baseline leg may spend (it samples the step to fit)
+CPU_BASELINE_SECONDS = 14.0   # host time the all-threads leg of cpu_baseline may spend (it samples the step to fit)
+CPU_BASELINE_SECONDS_1T = 8.0  # and the one-thread leg
 INT8_OVER_BF16 = 2.0         # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture, keyed by
-# (workload, call); None until captured for the current kernel.
-NCU_TRAFFIC_BYTES = {
-    # profiles/index_gemm_tc_resnet18_layer3_conv.md: 13.5 MB read + 402.6 MB written while the kernel ran (the
-    # write-back of the 462 MB output continues after it ends)
-    ("resnet18_layer3_conv", "qlinear_bwd_dx"): 416.1e6,
-}
+BURST_REGION_SECONDS = 1.0   # a timed region shorter than this runs at burst clocks: the burst tensor peak applies
+BYTES_PER_ELEM = {"hard": 5, "hard_hist": 5, "soft": 8, "soft_idx_hist": 9, "sample_hist": 5, "backward": 12,
+                  "backward_rate": 12}
 
 
 def parse_args():
@@ -54,10 +55,15 @@ def parse_args():
     ap.add_argument("--conv-form", action="store_true",
                     help="resnet18_b256: run the layers that cdl_qconv_* supports in convolution form")
     ap.add_argument("--no-implicit", action="store_true", help="skip the extra measurement of the layer in convolution form")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="default line without its sweep / gemm / network blocks (e.g. for a profiler capture)")
+    ap.add_argument("--no-network", action="store_true", help="default line without the whole-network block")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step one by one instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
-    ap.add_argument("--sweep-max-log2n", type=int, default=28)
+    ap.add_argument("--sweep-max-log2n", type=int, default=30)
+    ap.add_argument("--sweep-dist", default="mixture", choices=["normal", "laplace", "mixture"],
+                    help="with --sweep: N(0,1), Laplace(0,1) or their element-wise 50/50 mixture")
     ap.add_argument("--sweep-point", type=float, nargs=3, metavar=("L", "ALPHA", "LOG2N"),
                     help="with --sweep: only this point of the grid (any L <= 127, any alpha), e.g. for a profiler capture")
     ap.add_argument("--gemm", type=int, nargs=3, metavar=("M", "K", "N"), action="append",
@@ -71,6 +77,64 @@ def peaks():
         p = json.loads(f.read_text())
         return p, "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def int8_yardstick(torch, reps=10):
+    """A library int8 matrix product timed the way the bf16 peak was measured (8192^3, best of `reps`, CUDA
+    events): the int8 throughput cuBLASLt reaches on this device, in TOPS; None if the routine is unavailable."""
+    try:
+        n = 8192
+        a = torch.randint(-8, 8, (n, n), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (n, n), dtype=torch.int8, device="cuda")
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        best = float("inf")
+        stream = torch.cuda.current_stream()
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            torch._int_mm(a, b)
+            e1.record(stream)
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    except Exception:
+        return None
+
+
+def tensor_peaks(pk, pk_kind, yardstick, region_seconds):
+    """int8 tensor peaks the fractions are quoted against.  `used`: 2 x the measured bf16 figure (nominal int8 : bf16
+    ratio) - the burst one when the kernels were timed in a region shorter than a second or alone, the sustained
+    one inside a long step.  `library_int8_8192`: the library int8 product measured in this run."""
+    burst = region_seconds < BURST_REGION_SECONDS
+    bf16 = float(pk["bf16_tflops"] if burst else pk.get("bf16_tflops_sustained", pk["bf16_tflops"]))
+    return {"used": bf16 * INT8_OVER_BF16,
+            "used_source": f"{pk_kind} {'burst' if burst else 'sustained'} bf16 x {INT8_OVER_BF16:g} (nominal int8:bf16)",
+            "burst_x2": float(pk["bf16_tflops"]) * INT8_OVER_BF16,
+            "sustained_x2": float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])) * INT8_OVER_BF16,
+            "library_int8_8192": yardstick,
+            "library_int8_note": "torch._int_mm 8192^3, best of 10, CUDA events (this run)" if yardstick else "unavailable"}
+
+
+def git_blob_sha1(path: Path) -> str:
+    data = path.read_bytes()
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+
+
+def traffic_from_profiles(workload, call):
+    """DRAM bytes per launch of `call` from the committed ncu summaries: a line
+    `bench-traffic: workload=W call=C bytes=B source=<file> sha1=<git blob hash of that file when captured>`.
+    Returns (bytes, note); bytes is None when there is no such line or the kernel's source has changed since."""
+    pat = re.compile(r"bench-traffic:\s+workload=(\S+)\s+call=(\S+)\s+bytes=(\d+)\s+source=(\S+)\s+sha1=([0-9a-f]{40})")
+    for f in sorted((ROOT / "profiles").glob("*.md")):
+        for m in pat.finditer(f.read_text()):
+            if m.group(1) == workload and m.group(2) == call:
+                src = ROOT / m.group(4)
+                if src.exists() and git_blob_sha1(src) == m.group(5):
+                    return int(m.group(3)), f"ncu capture summarised in profiles/{f.name}, kernel source unchanged since"
+                return None, f"profiles/{f.name} holds counters for an older version of {m.group(4)}"
+    return None, "no ncu capture of this call committed"
 
 
 def make_case(name, seed_offset=0):
@@ -88,7 +152,6 @@ def make_case(name, seed_offset=0):
 def host_inputs(case, w, x, hist_x):
     """Remaining inputs of a step: im2col index matrix (drawn from the activations' own level histogram),
     gradient arriving at the output, gradient arriving at the quantized activations."""
-    import numpy as np
     from paper_2501_09849_b200 import inputs
     A = inputs.indices_from_histogram((case.M, case.K), hist_x, case.aq.lo, seed=case.seed, stream=3)
     dY = inputs.normal((case.M, case.N), G_STD, seed=case.seed, stream=4)
@@ -125,7 +188,55 @@ def conv_call_model(case, n_x):
     return m
 
 
-def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, peaks_hbm, int8_tops):
+def queue_ahead(torch, ms=8.0):
+    """Keeps the device busy for about `ms` so that the host can enqueue the launches that follow before the device
+    reaches them: the intervals between their events then hold device time only, not the host's launch path."""
+    sleep = getattr(torch.cuda, "_sleep", None)
+    if sleep is not None:
+        sleep(int(ms * 1e-3 * 1.9e9))
+
+
+def per_call_times(torch, step, calls, k_steps, stream, **run_kw):
+    """Mean device time of each call of a step: k_steps steps launched call by call with one CUDA event between
+    calls, the host kept ahead of the device (queue_ahead) in chunks that fit the launch queue."""
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(k_steps)]
+    chunk = 32
+    for it0 in range(0, k_steps, chunk):
+        torch.cuda.synchronize()
+        queue_ahead(torch)
+        for it in range(it0, min(k_steps, it0 + chunk)):
+            ev = iter(events[it])
+            step.run(mark=lambda name: next(ev).record(stream), **run_kw)
+    torch.cuda.synchronize()
+    return {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(k_steps)) / k_steps
+            for i, name in enumerate(calls)}
+
+
+def kernel_table(calls, model, per_call_ms, hbm, tp):
+    """Per call: time, algorithmic GB/s, and for the products int8 TOPS and the fraction of min(tensor, HBM) roofline
+    (tensor peak: tp['used']; the fraction of the library int8 product is given beside it)."""
+    kernels = {}
+    for name in calls:
+        m, ms = model[name], per_call_ms[name]
+        k = {"ms": round(ms, 5), "GBps": round(m["bytes"] / (ms * 1e-3) / 1e9, 1)}
+        if m["elems"]:
+            k["Gelem_per_s"] = round(m["elems"] / (ms * 1e-3) / 1e9, 2)
+            k["hbm_frac_measured"] = round(k["GBps"] / hbm, 4)
+            k["hbm_frac_8TBps"] = round(k["GBps"] / 8000.0, 4)
+        if "ops" in m:
+            tops = m["ops"] / (ms * 1e-3) / 1e12
+            k["int8_TOPS"] = round(tops, 1)
+            t_tensor, t_hbm = m["ops"] / (tp["used"] * 1e12), m["bytes"] / (hbm * 1e9)
+            k["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
+            k["roofline_frac"] = round(max(t_tensor, t_hbm) / (ms * 1e-3), 4)
+            k["int8_frac_of_peak"] = round(tops / tp["used"], 4)
+            if tp.get("library_int8_8192"):
+                k["int8_frac_of_library_int8"] = round(tops / tp["library_int8_8192"], 4)
+        kernels[name] = k
+    return kernels
+
+
+def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, peaks_hbm, tp):
     """The same layer as a convolution computed straight from the NHWC index tensor (cdl_qconv_*): same w, x and
     dL/dY, the data gradient feeds the activation quantizer's backward pass directly.  Returns a dict of times."""
     n_img, H, W, C = case.a_shape
@@ -151,25 +262,10 @@ def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, p
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    k_steps = min(steps, 200)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(k_steps)]
-    for it in range(k_steps):
-        ev = iter(events[it])
-        cs.run(mark=lambda name: next(ev).record(stream))
-    torch.cuda.synchronize()
-    per = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(k_steps)) / k_steps
-           for i, name in enumerate(CALLS)}
+    k_steps = max(50, min(steps, 200))
+    per = per_call_times(torch, cs, CALLS, k_steps, stream)
     model = conv_call_model(case, step.n_x)
-    kern = {}
-    for name in CALLS:
-        m, t = model[name], per[name]
-        k = {"ms": round(t, 5), "GBps": round(m["bytes"] / (t * 1e-3) / 1e9, 1)}
-        if "ops" in m:
-            k["int8_TOPS"] = round(m["ops"] / (t * 1e-3) / 1e12, 1)
-            t_tensor, t_hbm = m["ops"] / (int8_tops * 1e12), m["bytes"] / (peaks_hbm * 1e9)
-            k["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
-            k["roofline_frac"] = round(max(t_tensor, t_hbm) / (t * 1e-3), 4)
-        kern[name] = k
+    kern = kernel_table(CALLS, model, per, peaks_hbm, tp)
     quant_elems = sum(m["elems"] for m in model.values())
     # end to end: this form's inputs (w, x, dL/dY) from pinned host memory every step, scalars and dL/dw back
     pinned = {k: t.cpu().pin_memory() for k, t in cs.input_tensors().items()}
@@ -194,7 +290,7 @@ def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, p
             "note": "same layer through cdl_qconv_fwd/bwd: no stored patch matrix, dX in the layout of x"}
 
 
-def e2e_pipelined(torch, steps2, graphs2, pinned, out_host, e_steps, after_step=None):
+def e2e_pipelined(torch, steps2, graphs2, pinned, out_host, e_steps, run_kw=None):
     """End-to-end steps from host buffers: every step copies its inputs from pinned host memory, runs, and reads
     the scalars and dL/dw back.  Two sets of device buffers alternate, so the copy of step i+1 (on a copy stream)
     overlaps the kernels of step i; the host-to-device copies themselves are the critical path.
@@ -220,9 +316,7 @@ def e2e_pipelined(torch, steps2, graphs2, pinned, out_host, e_steps, after_step=
         if graphs2[b] is not None:
             graphs2[b].replay()
         else:
-            st.run()
-        if after_step is not None:
-            after_step(st)
+            st.run(**(run_kw or {}))
         out_host["scalars"].copy_(st.scalars, non_blocking=True)
         out_host["dw"].copy_(st.dw, non_blocking=True)
         done[b].record(stream)
@@ -334,6 +428,31 @@ def oracle_step_sample(case, host, frac=1.0):
     return t_total, desc, oracle.threads(), time.perf_counter() - t_wall0
 
 
+def cpu_baseline_block(case, host, quant_elems):
+    """The oracle, as it stands, on the host cores: at all threads and at one thread, each on a bounded sample."""
+    import oracle
+    oracle.build()
+    all_threads = oracle.threads()
+
+    def leg(seconds):
+        cal = oracle_step_sample(case, host, 1.0 / 256)[3]
+        frac = min(1.0, seconds / max(256.0 * cal, 1e-9))
+        return oracle_step_sample(case, host, frac)
+
+    t_cpu, desc, thr, _ = leg(CPU_BASELINE_SECONDS)
+    out = {"value": quant_elems / t_cpu / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc,
+           "ms_per_step_estimate": t_cpu * 1e3,
+           "timing": "time.perf_counter around each oracle call, one run per part, parts scaled to a full step"}
+    try:
+        oracle.set_threads(1)
+        t1, desc1, thr1, _ = leg(CPU_BASELINE_SECONDS_1T)
+        out.update(value_1thread=quant_elems / t1 / 1e9, ms_per_step_estimate_1thread=t1 * 1e3, sample_1thread=desc1,
+                   cores_1thread=thr1)
+    finally:
+        oracle.set_threads(all_threads)
+    return out
+
+
 def run_reference(args, rank):
     """Reference arm: the CPU oracle on a bounded sample of the same workload (rank 0 only)."""
     if rank != 0:
@@ -367,10 +486,169 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------- quantizer sweep
+def draw(torch, gen, n, dist, scale=1.0):
+    """n float32 values on the device: N(0,1), Laplace(0,1) (by inversion) or their element-wise 50/50 mixture."""
+    if dist == "normal":
+        x = torch.randn(n, device="cuda", generator=gen)
+    else:
+        u = torch.rand(n, device="cuda", generator=gen) - 0.5
+        x = -torch.sign(u) * torch.log1p(-2.0 * u.abs().clamp_(max=0.49999997))      # (u = -0.5 would give an infinity)
+        del u
+        if dist == "mixture":
+            pick = torch.rand(n, device="cuda", generator=gen) < 0.5
+            x = torch.where(pick, torch.randn(n, device="cuda", generator=gen), x)
+            del pick
+    if scale != 1.0:
+        x *= scale
+    return x.contiguous()
+
+
+class SweepBuffers:
+    """Device buffers of the quantizer-only timings and the timing loop itself."""
+
+    def __init__(self, torch, cdl, nmax, reps):
+        self.torch, self.cdl, self.nmax, self.reps = torch, cdl, nmax, reps
+        self.gen = torch.Generator(device="cuda").manual_seed(5)
+        self.x = None
+        self.g = torch.randn(nmax, device="cuda", generator=self.gen)
+        self.y = torch.empty(nmax, dtype=torch.float32, device="cuda")
+        self.idx = torch.empty(nmax, dtype=torch.int8, device="cuda")
+        self.s = torch.zeros(2, dtype=torch.float64, device="cuda")
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        self.stream = torch.cuda.current_stream()
+
+    def set_data(self, dist, scale=1.0):
+        self.x = None
+        self.x = draw(self.torch, self.gen, self.nmax, dist, scale)
+
+    def timed(self, make_fn, n):
+        """Median time of one launch.  Launches are issued back to back on distinct slices of the big buffers
+        (so that none finds its input in L2 and the CPU-side launch cost is hidden), one event pair around all."""
+        torch = self.torch
+        k = max(1, min(16, self.nmax // n))
+        fns = [make_fn(i * n) for i in range(k)]
+        for f in fns[:2]:
+            f()
+        ts = []
+        for _ in range(self.reps):
+            if k * n * 12 < (512 << 20):
+                self.flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for f in fns:
+                f()
+            e1.record(self.stream)
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1) / k)
+        return statistics.median(ts)
+
+    def passes(self, n, P, Pr, hist, which=None):
+        """{pass name: maker(offset) -> launcher} for n elements under quantizer P (Pr: the same with level
+        probabilities, for the rate term)."""
+        cdl, x, g, y, s = self.cdl, self.x, self.g, self.y, self.s
+        ix_t = self.idx if P.lo < 0 else self.idx.view(self.torch.uint8)
+
+        def mk(kind, PP=P):
+            def make(o):
+                xs, gs, ys, ix = x[o:o + n], g[o:o + n], y[o:o + n], ix_t[o:o + n]
+                if kind == "hard":
+                    return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, None)
+                if kind == "hard_hist":
+                    return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, hist)
+                if kind == "soft":
+                    return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, None, None)
+                if kind == "soft_idx_hist":
+                    return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, ix, hist)
+                if kind == "sample_hist":
+                    return lambda: cdl.cdl_quantize_sample(xs, n, PP, 7, o, ix, None, hist)
+                return lambda: cdl.cdl_quantize_backward(xs, gs, n, PP, ys, s[0:1], s[1:2])
+            return make
+        out = {"hard": mk("hard"), "hard_hist": mk("hard_hist"), "soft": mk("soft"), "soft_idx_hist": mk("soft_idx_hist"),
+               "sample_hist": mk("sample_hist"), "backward": mk("backward"), "backward_rate": mk("backward", Pr)}
+        return out if which is None else {k: out[k] for k in which}
+
+    def row(self, n, name, ms, hbm, **extra):
+        gbs = n * BYTES_PER_ELEM[name] / (ms * 1e-3) / 1e9
+        r = {"n": n, "pass": name, "ms": round(ms, 4), "Gelem_per_s": round(n / (ms * 1e-3) / 1e9, 2), "GBps": round(gbs, 1),
+             "hbm_frac_measured": round(gbs / hbm, 4), "hbm_frac_8TBps": round(gbs / 8000.0, 4)}
+        r.update(extra)
+        return r
+
+
+def entropy_pass_ms(torch, cdl, nlev, reps=200):
+    """cdl_index_entropy on its own: mean device time of back-to-back launches (a latency, not a bandwidth)."""
+    hist = torch.randint(1, 1 << 20, (nlev,), dtype=torch.int64, device="cuda")
+    H = torch.zeros(1, dtype=torch.float64, device="cuda")
+    lp = torch.zeros(nlev, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        cdl.cdl_index_entropy(hist, nlev, H, lp)
+    torch.cuda.synchronize()
+    queue_ahead(torch, 2.0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        cdl.cdl_index_entropy(hist, nlev, H, lp)
+    e1.record(stream)
+    e1.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def sweep_compact(torch, cdl, hbm, reps, layer_n):
+    """The part of the quantizer sweep the default line carries: hard / hard+hist / soft+idx+hist / backward / backward
+    with rate term at L = 7, alpha = 100 (step 4/L) on 2^28 elements of N(0,1), Laplace(0,1) and their mixture and on
+    2^30 elements of the mixture; the paper's own operating point (6 bits, alpha = 500, step from the mean magnitude,
+    weight-like data) on 2^25 elements; the same passes at the bench layer's tensor size, launched back to back on
+    distinct slices; the entropy pass on its own."""
+    rows = []
+    names = ("hard", "hard_hist", "soft_idx_hist", "backward", "backward_rate")
+
+    def point(B, n, L, alpha, q, lo, hi, tag, which=names, window=0):
+        nlev = hi - lo + 1
+        hist = torch.zeros(nlev, dtype=torch.int64, device="cuda")
+        lp = torch.full((nlev,), 1.0 / nlev, dtype=torch.float32, device="cuda")
+        lp[nlev // 2] *= 1.5
+        P = cdl.QuantParams(q, lo, hi, alpha, 0.01, None, window)
+        Pr = cdl.QuantParams(q, lo, hi, alpha, 0.01, lp, window)
+        for name, make in B.passes(n, P, Pr, hist, which).items():
+            rows.append(B.row(n, name, B.timed(make, n), hbm, L=L, alpha=alpha, data=tag, levels=nlev, window=window))
+
+    n28 = 1 << 28
+    B = SweepBuffers(torch, cdl, n28, reps)
+    for dist in ("normal", "laplace", "mixture"):
+        B.set_data(dist)
+        point(B, n28, 7, 100.0, 4.0 / 7, -7, 7, dist)
+    # bench layer size (12.85 M elements), mixture data still loaded: 16 distinct slices back to back
+    point(B, layer_n, 7, 100.0, 4.0 / 7, -7, 7, "mixture, layer-size tensors back to back")
+    # the layer's own activation quantizer (16 unsigned levels, window of five) on half-normal data of that size
+    B.x.abs_()
+    q_act = float(2.0 * B.x[:layer_n].mean() / 8.0 ** 0.5)
+    point(B, layer_n, None, 100.0, q_act, 0, 15, "half-normal, layer-size tensors back to back", window=5,
+          which=("soft_idx_hist", "backward_rate"))
+    # the paper's operating point: b = 6, alpha = 500, step 2 mean|w| / sqrt(2^(b-1)) on He-normal-like weights
+    n25 = 1 << 25
+    B.set_data("normal", scale=(2.0 / 2304.0) ** 0.5)
+    q6 = float(2.0 * B.x[:n25].abs().mean() / 32.0 ** 0.5)
+    point(B, n25, None, 500.0, q6, -32, 31, "He-normal weights, 6-bit paper point (Sec. VI-B.3)", which=("soft_idx_hist", "backward"))
+    del B
+    torch.cuda.empty_cache()
+    n30 = 1 << 30
+    B = SweepBuffers(torch, cdl, n30, max(3, reps // 2))
+    B.set_data("mixture")
+    point(B, n30, 7, 100.0, 4.0 / 7, -7, 7, "mixture", which=("hard", "soft_idx_hist", "backward"))
+    del B
+    torch.cuda.empty_cache()
+    ent = {f"nlev_{k}": round(entropy_pass_ms(torch, cdl, k) * 1e3, 2) for k in (15, 16, 255)}
+    return {"rows": rows, "entropy_pass_us": ent,
+            "timing": "median over repetitions of back-to-back launches on distinct slices (one CUDA event pair around "
+                      "up to 16 launches), inputs never L2-resident"}
+
+
 def run_sweep(args):
-    """Quantizer-only bandwidth sweep: fp32 tensors of 2^20 .. 2^max elements (50/50 N(0,1) / Laplace(0,1) mixture
-    drawn on the device), L in {1,3,7,15,127}, alpha in {1,100,1e4}, step 4/L; hard, hard+hist, soft, soft+idx+hist,
-    sampled index+hist, backward and backward+rate timed separately with CUDA events."""
+    """Quantizer-only bandwidth sweep: fp32 tensors of 2^20 .. 2^max elements (N(0,1), Laplace(0,1) or their 50/50
+    mixture, drawn on the device), L in {1,3,7,15,127}, alpha in {1,100,1e4}, step 4/L; hard, hard+hist, soft,
+    soft+idx+hist, sampled index+hist, backward and backward+rate timed separately with CUDA events."""
     import torch
 
     import paper_2501_09849_b200 as cdl
@@ -380,47 +658,14 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     pk, pk_kind = peaks()
     hbm = float(pk["hbm_gbs"])
-    gen = torch.Generator(device="cuda").manual_seed(5)
     grid_n = list(range(20, args.sweep_max_log2n + 1, 2))
     grid_L, grid_alpha = (1, 3, 7, 15, 127), (1.0, 100.0, 1e4)
     if args.sweep_point:
         grid_L, grid_alpha, grid_n = (int(args.sweep_point[0]),), (float(args.sweep_point[1]),), [int(args.sweep_point[2])]
         args.sweep_max_log2n = grid_n[0]
     nmax = 1 << args.sweep_max_log2n
-    pick = torch.rand(nmax, device="cuda", generator=gen) < 0.5
-    xn = torch.randn(nmax, device="cuda", generator=gen)
-    u = torch.rand(nmax, device="cuda", generator=gen) - 0.5
-    xl = -torch.sign(u) * torch.log1p(-2.0 * u.abs())           # Laplace(0,1) by inversion
-    x = torch.where(pick, xn, xl).contiguous()
-    del pick, xn, xl, u
-    g = torch.randn(nmax, device="cuda", generator=gen)
-    y = torch.empty(nmax, dtype=torch.float32, device="cuda")
-    idx = torch.empty(nmax, dtype=torch.int8, device="cuda")
-    s = torch.zeros(2, dtype=torch.float64, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    stream = torch.cuda.current_stream()
-    reps = max(3, args.steps // 4)
-
-    def timed(make_fn, n):
-        """Median time of one launch.  Launches are issued back to back on distinct slices of the big buffers
-        (so that none finds its input in L2 and the CPU-side launch cost is hidden), one event pair around all."""
-        k = max(1, min(16, nmax // n))
-        fns = [make_fn(i * n) for i in range(k)]
-        for f in fns[:2]:
-            f()
-        ts = []
-        for _ in range(reps):
-            if k * n * 12 < (512 << 20):
-                flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for f in fns:
-                f()
-            e1.record(stream)
-            e1.synchronize()
-            ts.append(e0.elapsed_time(e1) / k)
-        return statistics.median(ts)
-
+    B = SweepBuffers(torch, cdl, nmax, max(3, args.steps // 4))
+    B.set_data(args.sweep_dist)
     rows = []
     for log2n in grid_n:
         n = 1 << log2n
@@ -431,58 +676,30 @@ def run_sweep(args):
             for alpha in grid_alpha:
                 P = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01)
                 Pr = cdl.QuantParams(4.0 / L, -L, L, alpha, 0.01, lp)
-
-                def mk(kind, PP=P):
-                    def make(o):
-                        xs, gs, ys, ix = x[o:o + n], g[o:o + n], y[o:o + n], idx[o:o + n]
-                        if kind == "hard":
-                            return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, None)
-                        if kind == "hard_hist":
-                            return lambda: cdl.cdl_quantize_hard(xs, n, PP, ix, hist)
-                        if kind == "soft":
-                            return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, None, None)
-                        if kind == "soft_idx_hist":
-                            return lambda: cdl.cdl_quantize_soft(xs, n, PP, ys, ix, hist)
-                        if kind == "sample_hist":
-                            return lambda: cdl.cdl_quantize_sample(xs, n, PP, 7, o, ix, None, hist)
-                        return lambda: cdl.cdl_quantize_backward(xs, gs, n, PP, ys, s[0:1], s[1:2])
-                    return make
-                passes = {"hard": (5, mk("hard")), "hard_hist": (5, mk("hard_hist")), "soft": (8, mk("soft")),
-                          "soft_idx_hist": (9, mk("soft_idx_hist")), "sample_hist": (5, mk("sample_hist")),
-                          "backward": (12, mk("backward")),
-                          "backward_rate": (12, mk("backward", Pr))}
+                passes = B.passes(n, P, Pr, hist)
                 if alpha != grid_alpha[0]:
                     passes.pop("hard"), passes.pop("hard_hist")      # the hard passes do not depend on alpha
-                for name, (bpe, make) in passes.items():
-                    ms = timed(make, n)
-                    gbs = n * bpe / (ms * 1e-3) / 1e9
-                    rows.append({"log2n": log2n, "L": L, "alpha": alpha, "pass": name, "ms": round(ms, 4),
-                                 "Gelem_per_s": round(n / (ms * 1e-3) / 1e9, 2), "GBps": round(gbs, 1),
-                                 "hbm_frac_measured": round(gbs / hbm, 4), "hbm_frac_8TBps": round(gbs / 8000.0, 4)})
-    print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "peak_hbm_gbs": hbm, "peak_source": pk_kind,
-                      "data": "synthetic", "config": {"workload": "quantizer_sweep", "max_log2n": args.sweep_max_log2n}}),
-          flush=True)
+                for name, make in passes.items():
+                    r = B.row(n, name, B.timed(make, n), hbm, L=L, alpha=alpha)
+                    r["log2n"] = log2n
+                    rows.append(r)
+    ent = {f"nlev_{k}": round(entropy_pass_ms(torch, cdl, k) * 1e3, 2) for k in (3, 7, 15, 31, 255)}
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "entropy_pass_us": ent, "peak_hbm_gbs": hbm,
+                      "peak_source": pk_kind, "data": "synthetic",
+                      "config": {"workload": "quantizer_sweep", "max_log2n": args.sweep_max_log2n,
+                                 "distribution": args.sweep_dist}}), flush=True)
 
 
-def run_gemm(args):
-    """Index GEMMs alone: forward, dX and dW for each requested (M, K, N), 4-bit activation / weight indices and
-    8-bit gradient indices drawn uniformly on the device, float outputs; operands are rotated over several
-    buffer sets when one set would fit in L2."""
-    import torch
-
-    import paper_2501_09849_b200 as cdl
-    from paper_2501_09849_b200 import build as cdl_build
-    cdl_build.build()
-    cdl.load_library()
-    torch.cuda.set_device(0)
-    pk, pk_kind = peaks()
-    hbm = float(pk["hbm_gbs"])
-    int8_tops = float(pk["bf16_tflops"]) * INT8_OVER_BF16          # kernels timed alone: burst figure
+# ----------------------------------------------------------------------------------------------- index GEMMs alone
+def gemm_rows(torch, cdl, shapes, steps, hbm, tp):
+    """Index GEMMs alone: forward, dX and dW for each (M, K, N), 4-bit activation / weight indices and 8-bit gradient
+    indices drawn uniformly on the device, float outputs; operands are rotated over several buffer sets when one set
+    would fit in L2; each product's pass over the buffer sets is replayed from a CUDA graph."""
     stream = torch.cuda.current_stream()
     gen = torch.Generator(device="cuda").manual_seed(7)
     a, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
     out = []
-    for M, K, N in args.gemm:
+    for M, K, N in shapes:
         set_bytes = M * K + K * N + M * N + 4 * (M * N + M * K + K * N)
         nset = max(1, min(4, (400 << 20) // set_bytes + 1))
         sets = []
@@ -505,8 +722,6 @@ def run_gemm(args):
         for name, fn in calls.items():
             for t in sets:
                 fn(t)
-            # one pass over the buffer sets recorded as a graph: calls of a few microseconds would otherwise be
-            # timed by the host's launch path, not by the device
             torch.cuda.synchronize()
             side = torch.cuda.Stream()
             graph = torch.cuda.CUDAGraph()
@@ -514,7 +729,7 @@ def run_gemm(args):
                 with torch.cuda.graph(graph, stream=side):
                     for t in sets:
                         fn(t)
-            rounds = max(2, min(40, args.steps) // nset)
+            rounds = max(2, min(40, steps) // nset)
             graph.replay()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -525,44 +740,57 @@ def run_gemm(args):
             e1.synchronize()
             ms = e0.elapsed_time(e1) / (rounds * nset)
             ops = 2.0 * M * K * N
-            t_tensor, t_hbm = ops / (int8_tops * 1e12), bytes_[name] / (hbm * 1e9)
-            row[name] = {"ms": round(ms, 5), "int8_TOPS": round(ops / (ms * 1e-3) / 1e12, 1),
-                         "int8_frac_of_peak": round(ops / (ms * 1e-3) / 1e12 / int8_tops, 4),
+            tops = ops / (ms * 1e-3) / 1e12
+            t_tensor, t_hbm = ops / (tp["burst_x2"] * 1e12), bytes_[name] / (hbm * 1e9)
+            row[name] = {"ms": round(ms, 5), "int8_TOPS": round(tops, 1),
+                         "int8_frac_of_peak": round(tops / tp["burst_x2"], 4),
                          "GBps": round(bytes_[name] / (ms * 1e-3) / 1e9, 1), "bound": "tensor" if t_tensor >= t_hbm else "hbm",
                          "roofline_frac": round(max(t_tensor, t_hbm) / (ms * 1e-3), 4)}
+            if tp.get("library_int8_8192"):
+                row[name]["int8_frac_of_library_int8"] = round(tops / tp["library_int8_8192"], 4)
         row["status"] = cdl.cdl_workspace_status(ws, check=False)
         out.append(row)
         del sets
-    print(json.dumps({"metric": METRIC, "unit": "int8 TOPS", "gemm": out, "int8_peak_tops": int8_tops,
-                      "peak_source": f"{pk_kind} burst bf16 x {INT8_OVER_BF16:g} (nominal int8:bf16)", "peak_hbm_gbs": hbm,
-                      "data": "synthetic", "config": {"workload": "index_gemm"}}), flush=True)
+    return out
 
 
-def run_network(args):
-    """Whole ResNet-18 (224x224) as a sequence of CDL layer steps: every conv and the FC layer with its true im2col
-    GEMM shape, 3-bit weights (step = std(w) / 3), 4-bit activations (step from the mean magnitude), window of 5.
-    Inputs are drawn on the device (seeded); each layer owns its buffers, so a step touches ~40 GB at batch 256."""
+def run_gemm(args):
     import torch
 
     import paper_2501_09849_b200 as cdl
     from paper_2501_09849_b200 import build as cdl_build
-    from paper_2501_09849_b200 import inputs
-    from paper_2501_09849_b200.layer import CALLS, CdlLayerStep
     cdl_build.build()
     cdl.load_library()
     torch.cuda.set_device(0)
+    pk, pk_kind = peaks()
+    hbm = float(pk["hbm_gbs"])
+    tp = tensor_peaks(pk, pk_kind, int8_yardstick(torch), 0.0)       # kernels timed alone: burst figure
+    rows = gemm_rows(torch, cdl, args.gemm, args.steps, hbm, tp)
+    print(json.dumps({"metric": METRIC, "unit": "int8 TOPS", "gemm": rows, "int8_peak_tops": tp["burst_x2"],
+                      "tensor_peaks": tp, "peak_hbm_gbs": hbm, "data": "synthetic",
+                      "config": {"workload": "index_gemm"}}), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- whole network
+def network_step(torch, cdl, batch, conv_form, steps, warm, use_graph=True):
+    """Whole ResNet-18 (224x224) as a sequence of CDL layer steps: every conv and the FC layer with its true im2col
+    GEMM shape, 3-bit weights (step = std(w) / 3), 4-bit activations (step from the mean magnitude), window of 5.
+    Inputs are drawn on the device (seeded); each layer owns its buffers, so a step touches ~40 GB at batch 256.
+    Returns the fields of the network line."""
+    from paper_2501_09849_b200 import inputs
+    from paper_2501_09849_b200.layer import CALLS, CdlLayerStep
     gen = torch.Generator(device="cuda").manual_seed(4)
     stream = torch.cuda.current_stream()
     q_g = 4.0 * G_STD / 127.0
     layers = []
-    for name, M, K, N, n_x in inputs.resnet18_layers(args.batch):
+    for name, M, K, N, n_x in inputs.resnet18_layers(batch):
         Np = (N + 15) // 16 * 16                  # index matrices need 16-byte row pitches: fc's 1000 columns -> 1008
         w = torch.randn(K * Np, device="cuda", generator=gen) * (2.0 / K) ** 0.5
         x = torch.randn(n_x, device="cuda", generator=gen).abs_()
         wq = inputs.Quantizer(float(w.std()) / 3.0, -3, 3, 100.0, 0.01, 0)
         xq = inputs.Quantizer(float(2.0 * x.mean() / 8.0 ** 0.5), 0, 15, 100.0, 0.01, 5)
-        geo = inputs.resnet18_conv_geometry(name) if args.conv_form else None
-        shape = cdl.ConvShape(args.batch, geo[0], geo[1], geo[2], geo[3], geo[4]) if geo else None
+        geo = inputs.resnet18_conv_geometry(name) if conv_form else None
+        shape = cdl.ConvShape(batch, *geo) if geo else None
         st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g, need_dx=(name != "conv1"), conv=shape)   # the image needs no gradient
         st.w.copy_(w)
         st.x.copy_(x)
@@ -586,14 +814,12 @@ def run_network(args):
         for li, (_, _, _, _, _, st) in enumerate(layers):
             st.run(mark=(lambda nm, li=li: mark(li, nm)) if mark else None)
 
-    warm = max(3, min(args.warmup, 5))
-    steps = max(3, min(args.steps, 20))
     for _ in range(warm):
         run_all()
     torch.cuda.synchronize()
     # the whole network step as one CUDA graph (each layer recorded on three streams), replayed `steps` times
     graph = None
-    if not args.no_graph:
+    if use_graph:
         graph = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
         side.wait_stream(stream)
@@ -611,15 +837,18 @@ def run_network(args):
         g1.record(stream)
         torch.cuda.synchronize()
         graph_ms = g0.elapsed_time(g1) / steps
-    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in layers] for _ in range(steps)]
+    c_steps = min(steps, 5)
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in layers] for _ in range(c_steps)]
     cnt = {}
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(0)
     sampler.start()
     time.sleep(0.3)
     wall0 = time.time()
+    torch.cuda.synchronize()
+    queue_ahead(torch)
     t0.record(stream)
-    for it in range(steps):
+    for it in range(c_steps):
         cnt.clear()
 
         def mark(li, nm, it=it):
@@ -630,20 +859,19 @@ def run_network(args):
     t1.record(stream)
     torch.cuda.synchronize()
     clocks = sampler.stop(wall0, time.time())
-    ms_step = t0.elapsed_time(t1) / steps
+    ms_step = t0.elapsed_time(t1) / c_steps
     call_by_call_ms = ms_step
     if graph is not None:
         ms_step = graph_ms
-    pk, pk_kind = peaks()
-    hbm = float(pk["hbm_gbs"])
     table, tot_ops, tot_q, gemm_ms, quant_ms = [], 0.0, 0, 0.0, 0.0
     for li, (name, M, K, N, n_x, st) in enumerate(layers):
-        per = {c: sum(ev[it][li][i].elapsed_time(ev[it][li][i + 1]) for it in range(steps)) / steps for i, c in enumerate(CALLS)}
+        per = {c: sum(ev[it][li][i].elapsed_time(ev[it][li][i + 1]) for it in range(c_steps)) / c_steps for i, c in enumerate(CALLS)}
         g_ms = per["qlinear_fwd"] + per["qlinear_bwd_dx"] + per["qlinear_bwd_dw"]
         q_ms = sum(v for c, v in per.items() if c.startswith("quantize"))
         ops = (6.0 if st.need_dx else 4.0) * M * K * N
         q_el = 2 * (n_x + K * N) + M * N
-        table.append({"layer": name, "M": M, "K": K, "N": N, "ms": round(sum(per.values()), 4), "gemm_ms": round(g_ms, 4),
+        table.append({"layer": name, "M": M, "K": K, "N": N, "form": "convolution" if st.conv is not None else "stored patch matrix",
+                      "ms": round(sum(per.values()), 4), "gemm_ms": round(g_ms, 4),
                       "gemm_int8_TOPS": round(ops / (g_ms * 1e-3) / 1e12, 1), "quantizer_ms": round(q_ms, 4),
                       "quantizer_Gelem_per_s": round(q_el / (q_ms * 1e-3) / 1e9, 1),
                       "calls_us": {c: round(v * 1e3, 1) for c, v in per.items()},
@@ -652,22 +880,38 @@ def run_network(args):
         tot_q += q_el
         gemm_ms += g_ms
         quant_ms += q_ms
-    print(json.dumps({
-        "metric": METRIC, "value": tot_q / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32+s8",
-        "data": "synthetic",
-        "config": {"workload": "resnet18_b256", "batch": args.batch, "layers": len(layers),
-                   "form": ("convolution form for the %d stride-1 3x3 layers, stored patch matrices "
-                            "for the rest" % sum(1 for *_, st in layers if st.conv is not None)) if args.conv_form
+    n_conv = sum(1 for *_, st in layers if st.conv is not None)
+    return {
+        "value": tot_q / (ms_step * 1e-3) / 1e9, "unit": UNIT, "steps": steps, "warmup": warm, "ms_per_step": ms_step,
+        "config": {"workload": "resnet18_b256", "batch": batch, "layers": len(layers),
+                   "form": ("convolution form for %d layers, stored patch matrices for the rest" % n_conv) if conv_form
                    else "stored patch matrices (im2col GEMMs)",
                    "launch": "stream launches" if graph is None else "CUDA graph replay of the network step",
                    "call_by_call_ms": call_by_call_ms, "weight_levels": 7,
                    "activation_levels": 16, "window_x": 5, "l2": "every layer's tensors exceed the 126 MB L2"},
         "network_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": tot_ops / (gemm_ms * 1e-3) / 1e12,
         "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": tot_q / (quant_ms * 1e-3) / 1e9,
-        "layers": table, "clocks": clocks, "peak_hbm_gbs": hbm, "peak_source": pk_kind,
-        "e2e": None, "e2e_note": "not measured for this workload (a step's inputs are ~11 GB); see the default workload",
-        "gpu_launches": steps * sum(st.kernels_per_step() for *_, st in layers)}), flush=True)
+        "layers": table, "clocks": clocks,
+        "gpu_launches": steps * sum(st.kernels_per_step() for *_, st in layers)}
+
+
+def run_network(args):
+    import torch
+
+    import paper_2501_09849_b200 as cdl
+    from paper_2501_09849_b200 import build as cdl_build
+    cdl_build.build()
+    cdl.load_library()
+    torch.cuda.set_device(0)
+    pk, pk_kind = peaks()
+    warm = max(3, min(args.warmup, 5))
+    steps = max(3, min(args.steps, 20))
+    net = network_step(torch, cdl, args.batch, args.conv_form, steps, warm, use_graph=not args.no_graph)
+    line = {"metric": METRIC, "n_gpus": 1, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32+s8", "data": "synthetic", "peak_hbm_gbs": float(pk["hbm_gbs"]), "peak_source": pk_kind,
+            "e2e": None, "e2e_note": "not measured for this workload (a step's inputs are ~11 GB); see the default workload"}
+    line.update(net)
+    print(json.dumps(line), flush=True)
 
 
 def main():
@@ -708,8 +952,10 @@ def main():
         dist.barrier()
     cdl.load_library()
 
-    # ---- inputs: seeded, host-generated, one independent batch per rank (weak scaling)
+    # ---- inputs: seeded, host-generated, one independent batch per rank (weak scaling); the weights are replicated
     case, w, x = make_case(args.workload, seed_offset=100 * rank)
+    if rank > 0:
+        w = make_case(args.workload, seed_offset=0)[1]
     M, K, N, n_x = case.M, case.K, case.N, x.size
     q_g = float(np.float32(4.0 * G_STD / 127.0))
     step = CdlLayerStep(torch, M, K, N, n_x, case.wq, case.aq, q_g)
@@ -717,6 +963,7 @@ def main():
     hist = torch.zeros(case.aq.nlev, dtype=torch.int64, device="cuda")
     cdl.cdl_quantize_hard(xd, n_x, cdl.QuantParams(case.aq.q, case.aq.lo, case.aq.hi), None, hist)
     host = host_inputs(case, w, x, hist.cpu().numpy().view(np.uint64))
+    del xd
     pinned = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in host.items()}
     dev_in = step.input_tensors()
     for k, t in dev_in.items():
@@ -724,21 +971,20 @@ def main():
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
 
-    def exchange():
-        # data-parallel exchange of a step: the weight-side results are sums over the global batch
-        sharding.exchange(dist, world, step.dW, step.hist_x, step.scalars)
+    # data-parallel ranks: the step runs with its exchange points (activation histogram before the entropy, integer
+    # dW accumulators before the conversion, the activation quantizer's two scalars at the end), launched call by call
+    run_kw = {"exchange": sharding.StepExchange(dist, world), "rows_global": M * world} if world > 1 else {}
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     for _ in range(max(args.warmup, 3)):
-        step.run()
-        exchange()
+        step.run(**run_kw)
     torch.cuda.synchronize()
 
     # ---- timed region: device-resident inputs, the step replayed from a CUDA graph (launch gaps between the ten
     # short kernels of a step are a tenth of its time when they are launched one by one)
-    graph = step.capture() if not args.no_graph else None
+    graph = step.capture() if (not args.no_graph and world == 1) else None
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -750,8 +996,7 @@ def main():
         if graph is not None:
             graph.replay()
         else:
-            step.run()
-        exchange()
+            step.run(**run_kw)
     t_end.record(stream)
     torch.cuda.synchronize()
     wall1 = time.time()
@@ -761,15 +1006,8 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
 
     # ---- per-call times: a second pass over the same steps, launched call by call with an event between calls
-    k_steps = min(args.steps, 500)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(k_steps)]
-    for it in range(k_steps):
-        ev = iter(events[it])
-        step.run(mark=lambda name: next(ev).record(stream))
-        exchange()
-    torch.cuda.synchronize()
-    per_call_ms = {name: sum(events[it][i].elapsed_time(events[it][i + 1]) for it in range(k_steps)) / k_steps
-                   for i, name in enumerate(CALLS)}
+    k_steps = max(50, min(args.steps, 500))
+    per_call_ms = per_call_times(torch, step, CALLS, k_steps, stream, **run_kw)
     status = cdl.cdl_workspace_status(step.ws, check=False)
 
     # ---- end to end: host buffers in, results out, every step
@@ -781,12 +1019,11 @@ def main():
     step_b = CdlLayerStep(torch, M, K, N, n_x, case.wq, case.aq, q_g)       # second set of device buffers
     for k, t in step_b.input_tensors().items():
         t.copy_(pinned[k].view(t.shape), non_blocking=True)
-    step_b.run()
+    step_b.run(**run_kw)
     graph_b = step_b.capture() if graph is not None else None
     if world > 1:
         dist.barrier()
-    e2e_ms = e2e_pipelined(torch, (step, step_b), (graph, graph_b), pinned, out_host, e_steps,
-                           after_step=(lambda st: sharding.exchange(dist, world, st.dW, st.hist_x, st.scalars)) if world > 1 else None)
+    e2e_ms = e2e_pipelined(torch, (step, step_b), (graph, graph_b), pinned, out_host, e_steps, run_kw=run_kw)
     del step_b, graph_b
 
     ms_step = total_ms / args.steps
@@ -802,31 +1039,20 @@ def main():
         value = world * quant_elems / (ms_step * 1e-3) / 1e9
         e2e_value = world * quant_elems / (e2e_ms * 1e-3) / 1e9
         hbm = float(pk["hbm_gbs"])
-        int8_tops = float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])) * INT8_OVER_BF16
-        kernels = {}
-        for name in CALLS:
-            m, ms = model[name], per_call_ms[name]
-            k = {"ms": round(ms, 5), "GBps": round(m["bytes"] / (ms * 1e-3) / 1e9, 1)}
-            if m["elems"]:
-                k["Gelem_per_s"] = round(m["elems"] / (ms * 1e-3) / 1e9, 2)
-                k["hbm_frac_measured"] = round(k["GBps"] / hbm, 4)
-                k["hbm_frac_8TBps"] = round(k["GBps"] / 8000.0, 4)
-            if "ops" in m:
-                k["int8_TOPS"] = round(m["ops"] / (ms * 1e-3) / 1e12, 1)
-                t_tensor, t_hbm = m["ops"] / (int8_tops * 1e12), m["bytes"] / (hbm * 1e9)
-                k["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
-                k["roofline_frac"] = round(max(t_tensor, t_hbm) / (ms * 1e-3), 4)
-            kernels[name] = k
+        yard = int8_yardstick(torch) if world == 1 else None
+        # the per-call times come from call-by-call launches in a region of k_steps steps
+        tp = tensor_peaks(pk, pk_kind, yard, k_steps * ms_step * 1e-3)
+        kernels = kernel_table(CALLS, model, per_call_ms, hbm, tp)
         dom = max(CALLS, key=lambda c: per_call_ms[c])
         dm, dms = model[dom], per_call_ms[dom]
-        if "ops" in dm and dm["ops"] / (int8_tops * 1e12) >= dm["bytes"] / (hbm * 1e9):
-            roof = {"kernel": dom, "bound": "tensor", "achieved": dm["ops"] / (dms * 1e-3) / 1e12, "peak": int8_tops,
-                    "unit": "TFLOP/s", "peak_source": f"{pk_kind} sustained bf16 x {INT8_OVER_BF16:g} (nominal int8:bf16)"}
+        if "ops" in dm and dm["ops"] / (tp["used"] * 1e12) >= dm["bytes"] / (hbm * 1e9):
+            roof = {"kernel": dom, "bound": "tensor", "achieved": dm["ops"] / (dms * 1e-3) / 1e12, "peak": tp["used"],
+                    "unit": "TFLOP/s", "peak_source": tp["used_source"]}
         else:
             roof = {"kernel": dom, "bound": "hbm", "achieved": dm["bytes"] / (dms * 1e-3) / 1e9, "peak": hbm,
                     "unit": "GB/s", "peak_source": f"{pk_kind} copy bandwidth"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.workload, dom))
+        roof["traffic"], roof["traffic_note"] = traffic_from_profiles(args.workload, dom)
         gemm_ms = sum(per_call_ms[c] for c in ("qlinear_fwd", "qlinear_bwd_dx", "qlinear_bwd_dw"))
         quant_ms = sum(per_call_ms[c] for c in CALLS if model[c]["elems"])
         step_bytes = sum(model[c]["bytes"] for c in CALLS)
@@ -840,26 +1066,40 @@ def main():
                        "l2": ("per-step working set is several times the 126 MB L2 (inputs larger than L2)"
                               if step_bytes > 2 * 126e6 else
                               "a step moves %.0f MB in all, of the order of the 126 MB L2: a parity-size workload, not a bandwidth figure" % (step_bytes / 1e6)),
-                       "parallelism": f"replicas x{world}, all-reduce of dW / histogram / scalars" if world > 1 else "single GPU"},
+                       "parallelism": (f"batch rows split over {world} ranks; all-reduce of the activation histogram (before "
+                                       "the entropy), the int32 dW accumulators (before the conversion) and two scalars")
+                       if world > 1 else "single GPU"},
             "layer_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": 6.0 * M * K * N / (gemm_ms * 1e-3) / 1e12,
             "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": quant_elems / (quant_ms * 1e-3) / 1e9,
             "quantizer_hbm_frac_measured": sum(model[c]["bytes"] for c in CALLS if model[c]["elems"]) / (quant_ms * 1e-3) / 1e9 / hbm,
-            "kernels": kernels, "roofline": roof, "clocks": clocks,
+            "kernels": kernels, "roofline": roof, "tensor_peaks": tp, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e_steps,
                     "overlap": "two sets of device buffers: the copy of step i+1 overlaps the kernels of step i"},
-            "gpu_launches": args.steps * step.kernels_per_step(), "device_status": status,
+            "gpu_launches": args.steps * (step.kernels_per_step() + (1 if world > 1 else 0)), "device_status": status,
             "launch": "stream launches" if graph is None else "CUDA graph replay of one step",
-            "kernel_timing": f"second pass of {k_steps} steps launched call by call, one CUDA event between calls",
+            "kernel_timing": (f"second pass of {k_steps} steps launched call by call, one CUDA event between calls, the "
+                              "host kept ahead of the device"),
         }
         if world == 1 and args.workload == "resnet18_layer3_conv" and not args.no_implicit:
-            line["implicit_conv"] = run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, args.steps, hbm, int8_tops)
+            line["implicit_conv"] = run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, args.steps, hbm, tp)
+        extras = world == 1 and args.workload == "resnet18_layer3_conv" and not args.no_extras
+        if extras:
+            del step, graph
+            torch.cuda.empty_cache()
+            tp_alone = tensor_peaks(pk, pk_kind, yard, 0.0)
+            line["gemm"] = {"rows": gemm_rows(torch, cdl, [(12544, 4608, 512), (8192, 8192, 8192)], min(args.steps, 40), hbm, tp_alone),
+                            "int8_peak_tops": tp_alone["burst_x2"], "peak_source": tp_alone["used_source"],
+                            "note": "index GEMMs alone (ResNet-18 layer4 3x3 and a square 8192^3), graph replay over rotated buffer sets"}
+            line["sweep"] = sweep_compact(torch, cdl, hbm, max(3, min(args.steps, 40) // 4), n_x)
+            if not args.no_network:
+                torch.cuda.empty_cache()
+                net = network_step(torch, cdl, 256, True, 5, 3)
+                net.pop("clocks", None)
+                line["network"] = net
+                torch.cuda.empty_cache()
         if world == 1 and not args.no_cpu_baseline:
-            import oracle
-            oracle.build()
-            t_cpu, desc, thr, _ = oracle_step_sample(case, host, frac=min(1.0, CPU_BASELINE_SECONDS / max(256.0 * oracle_step_sample(case, host, 1.0 / 256)[3], 1e-9)))
-            line["cpu_baseline"] = {"value": quant_elems / t_cpu / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle",
-                                    "sample": desc, "ms_per_step_estimate": t_cpu * 1e3}
+            line["cpu_baseline"] = cpu_baseline_block(case, host, quant_elems)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

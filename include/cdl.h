@@ -243,6 +243,18 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g,
                     void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * The rescale of the products' epilogue on its own (Sec. V-A: the integer sums times the two step sizes), for
+ * accumulators that were summed outside a product call - data-parallel ranks all-reduce the int32 dWacc of
+ * cdl_qlinear_bwd / cdl_qconv_bwd (integers: the sum does not depend on the number of ranks or their order) and
+ * convert once afterwards:   out[i] = (float)acc[i] * (q_x * q_y),   the two step sizes of the product's operands
+ * multiplied once in binary32, the conversion and the multiply each rounded to binary32 - the bits a single product
+ * over the whole batch gives.
+ *   acc [dev] n integers of acc_bits (32 or 64; 64 when the sum over all ranks could leave int32), naturally aligned;
+ *   out [dev] n floats.  n = 0 is valid.
+ */
+int cdl_rescale_acc(const void *acc, int32_t acc_bits, int64_t n, float q_x, float q_y, float *out, void *stream);
+
+/*
  * Backward layer products for a real-valued incoming gradient (Algorithm 1's backward pass as printed: dL/dY is
  * not quantized there; cdl_qlinear_bwd is the int8-gradient reading).  The gradient is expanded in two int8 digits,
  *   g ~ q1 i1 + q2 i2,  q1 = g_absmax / 127,  q2 = q1 / 254,
@@ -283,7 +295,7 @@ size_t cdl_qlinear_bwd_fp_workspace_bytes(int32_t M, int32_t N, int32_t K);
  * Limits: K * N <= CDL_NOALLOC_MAX_DW_ELEMS, otherwise CDL_ERR_TOO_LARGE; and M * max|a| * max|g| < 2^31 for the
  * declared index ranges (the sum over M must fit the int32 accumulators: there is no room here for the per-part
  * slabs with which cdl_qlinear_bwd sums longer reductions in int64), otherwise CDL_ERR_OVERFLOW_RISK - for
- * indices 0..15 against -127..127 that is M <= 1,127,287 rows.  In both cases nothing is launched.  Within the
+ * indices 0..15 against -127..127 that is M <= 1,127,288 rows.  In both cases nothing is launched.  Within the
  * limits the values are those of cdl_qlinear_bwd, bit for bit.
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  * Set-up: the first call on each device (with that device current) looks up the array's device address;

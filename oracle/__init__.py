@@ -43,6 +43,8 @@ def _load():
         c = ctypes
         P = c.c_void_p
         lib.cdl_oracle_threads.restype = c.c_int
+        lib.cdl_oracle_set_threads.restype = c.c_int
+        lib.cdl_oracle_set_threads.argtypes = [c.c_int]
         lib.cdl_oracle_cpmf.argtypes = [c.c_double, c.c_double, c.c_int, c.c_int, c.c_double, c.c_int, P]
         lib.cdl_oracle_soft.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, P]
         lib.cdl_oracle_partials.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int,
@@ -91,6 +93,11 @@ def _check_levels(lo, hi):
 def threads() -> int:
     """Host threads the oracle's parallel loops use."""
     return int(_load().cdl_oracle_threads())
+
+
+def set_threads(n: int) -> int:
+    """Sets the number of host threads of the oracle's parallel loops; returns the count in effect."""
+    return int(_load().cdl_oracle_set_threads(int(n)))
 
 
 def cpmf(theta, q, lo, hi, alpha, window=0):

@@ -54,6 +54,19 @@ int cdl_oracle_threads(void)
 #endif
 }
 
+/* Number of host threads the parallel loops use from now on (timing at one thread and at all cores); changes
+ * no arithmetic.  Returns the count in effect. */
+int cdl_oracle_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+    return omp_get_max_threads();
+#else
+    (void)n;
+    return 1;
+#endif
+}
+
 /* ---------------------------------------------------------------------------
  * CPMF of Sec. IV-A, Eq. (4) and its softmax form Eq. (6) (per layer: Eqs. (12), (13)):
  *  P[i-lo] = softmax_i( -alpha (theta - i q)^2 ).

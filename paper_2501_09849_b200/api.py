@@ -13,7 +13,7 @@ __all__ = [
     "CdlError", "QuantParams", "IndexDesc", "library_path", "load_library",
     "cdl_version", "cdl_strerror", "cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample",
     "cdl_index_entropy", "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_noalloc_status",
-    "cdl_workspace_bytes", "cdl_workspace_status", "CDL_NOALLOC_MAX_DW_ELEMS",
+    "cdl_workspace_bytes", "cdl_workspace_status", "cdl_rescale_acc", "CDL_NOALLOC_MAX_DW_ELEMS",
     "cdl_huffman_lengths", "cdl_qconv_bwd_fp", "cdl_qconv_bwd_fp_workspace_bytes", "cdl_qlinear_bwd_fp", "cdl_qlinear_bwd_fp_workspace_bytes", "cdl_qlinear_fwd_next", "cdl_qconv_fwd_next", "ConvShape", "cdl_qconv_fwd", "cdl_qconv_bwd", "cdl_qconv_workspace_bytes",
     "CDL_HIST_ACCUMULATE", "CDL_OP_QLINEAR_FWD", "CDL_OP_QLINEAR_BWD", "CDL_MAX_LEVELS",
 ]
@@ -118,6 +118,8 @@ def load_library():
     lib.cdl_workspace_bytes.restype = C.c_size_t
     lib.cdl_workspace_status.argtypes = [P, P]
     lib.cdl_noalloc_status.argtypes = [P]
+    lib.cdl_rescale_acc.argtypes = [P, I32, I64, C.c_float, C.c_float, P, P]
+    lib.cdl_rescale_acc.restype = C.c_int
     lib.cdl_noalloc_status.restype = C.c_int
     for name in ("cdl_quantize_hard", "cdl_quantize_soft", "cdl_quantize_backward", "cdl_quantize_sample", "cdl_index_entropy",
                  "cdl_qlinear_fwd", "cdl_qlinear_bwd", "cdl_qlinear_bwd_dw_noalloc", "cdl_workspace_status",
@@ -332,3 +334,8 @@ def cdl_noalloc_status(stream=None, check=True):
     current device (the record lives in the library's built-in scratch); allocates nothing."""
     rc = load_library().cdl_noalloc_status(_stream(stream))
     return _check(rc, "cdl_noalloc_status", check)
+
+
+def cdl_rescale_acc(acc, acc_bits, n, q_x, q_y, out, stream=None, check=True):
+    rc = load_library().cdl_rescale_acc(_ptr(acc), acc_bits, n, float(q_x), float(q_y), _ptr(out), _stream(stream))
+    return _check(rc, "cdl_rescale_acc", check)

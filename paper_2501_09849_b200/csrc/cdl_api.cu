@@ -142,6 +142,17 @@ inline bool overflow_risk(int64_t terms, const IndexRange &x, const IndexRange &
 
 constexpr size_t kStatusBytes = 256;
 
+// float output of accumulators that were summed outside a product call (across ranks): one conversion, one multiply
+template <typename T>
+__global__ void __launch_bounds__(256) rescale_acc_kernel(const T *__restrict__ acc, long long n, float scale, float *__restrict__ out)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const float v = sizeof(T) == 8 ? __ll2float_rn((long long)acc[i]) : (float)(int)acc[i];
+        out[i] = __fmul_rn(v, scale);
+    }
+}
+
 }  // namespace
 }  // namespace cdl
 
@@ -543,6 +554,25 @@ int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx,
         if (rc != CDL_OK) return rc;
     }
     return CDL_OK;
+}
+
+int cdl_rescale_acc(const void *acc, int32_t acc_bits, int64_t n, float q_x, float q_y, float *out, void *stream)
+{
+    const float scale = q_x * q_y;      // formed once in binary32, as in the products' epilogue
+    if (n < 0 || (n > 0 && (acc == nullptr || out == nullptr))) return CDL_ERR_ARG;
+    if (acc_bits != 32 && acc_bits != 64) return CDL_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(acc) & (uintptr_t)(acc_bits / 8 - 1)) || bad_f32_ptr(out)) return CDL_ERR_ALIGN;
+    if (!(q_x > 0.0f) || !(q_y > 0.0f) || !isfinite(scale)) return CDL_ERR_RANGE;
+    int rc = check_device();
+    if (rc != CDL_OK) return rc;
+    if (n == 0) return CDL_OK;
+    const int sms = sm_count();
+    long long blocks = (n + 255) / 256;
+    if (blocks > (long long)sms * 8) blocks = (long long)sms * 8;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (acc_bits == 64) rescale_acc_kernel<long long><<<(unsigned int)blocks, 256, 0, st>>>(static_cast<const long long *>(acc), n, scale, out);
+    else rescale_acc_kernel<int><<<(unsigned int)blocks, 256, 0, st>>>(static_cast<const int *>(acc), n, scale, out);
+    return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
 }
 
 namespace {

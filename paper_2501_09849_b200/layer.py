@@ -15,6 +15,11 @@ Step (names follow the paper: w weights, x activations, q / s step sizes, alpha 
 The im2col gather / scatter between the activation tensor and the GEMM operand is outside the library:
 A_idx and the gradient arriving at the quantized activations are inputs of the step.
 
+Data-parallel ranks pass run(exchange=StepExchange): the activation histogram is then summed over the ranks before
+step 4, the weight-gradient product of step 7 delivers its int32 accumulators, which are summed over the ranks and
+converted to float once (cdl_rescale_acc), and the two scalar gradients of the activation quantizer are summed at
+the end; everything that depends on the weights alone is identical on every rank and is not exchanged.
+
 With conv=ConvShape(...) the layer is a stride-1 convolution computed straight from the NHWC index tensor
 (cdl_qconv_fwd / cdl_qconv_bwd): steps 5 and 7 read X_idx itself, dA becomes dL/dQ(x) in the layout of x, and step 8
 takes it as its incoming gradient, so the only inputs of a step are w, x and dL/dY.
@@ -191,18 +196,36 @@ class CdlLayerStep:
             cdl.cdl_qconv_bwd(self.G_idx, self.dg, None, None, self.W_idx, N, self.dw_desc, self.conv, N,
                               None, self.dA, None, None, self.ws, self.ws_bytes, stream)
 
-    def _bwd_dw(self, stream):
+    def _bwd_dw(self, stream, acc=None):
+        """dW as floats, or (acc given) as int32 accumulators for a later sum over ranks."""
         M, K, N = self.M, self.K, self.N
+        dWf = self.dW if acc is None else None
         if self.conv is None:
             cdl.cdl_qlinear_bwd(self.G_idx, N, self.dg, self.A_idx, self.lda, self.da, None, N, None,
-                                M, N, K, None, None, None, self.dW, self.ws, self.ws_bytes, stream)
+                                M, N, K, None, None, acc, dWf, self.ws, self.ws_bytes, stream)
         else:
             cdl.cdl_qconv_bwd(self.G_idx, self.dg, self.X_idx, self.da, None, N, None, self.conv, N,
-                              None, None, None, self.dW, self.ws, self.ws_bytes, stream)
+                              None, None, acc, dWf, self.ws, self.ws_bytes, stream)
 
-    def run(self, stream=None, mark=None):
+    def _bwd_dw_exchanged(self, stream, exchange, rows_global):
+        """Weight gradient of the global batch: local integer accumulators, summed over the ranks as integers,
+        one conversion to float afterwards - the bits of a single product over all rows."""
+        from . import sharding
+        t = self.torch
+        if not hasattr(self, "dWacc"):
+            self.dWacc = t.empty((self.K, self.N), dtype=t.int32, device=self.dW.device)
+        self._bwd_dw(stream, acc=self.dWacc)
+        amax = max(abs(self.xq.lo), abs(self.xq.hi))
+        bits = sharding.acc_bits_for(rows_global, amax, 127)
+        acc = self.dWacc if bits == 32 else self.dWacc.to(t.int64)
+        exchange.accumulators(acc)
+        cdl.cdl_rescale_acc(acc, bits, self.K * self.N, self.q_g, self.xq.q, self.dW, stream)
+
+    def run(self, stream=None, mark=None, exchange=None, rows_global=None):
         """Enqueue one step.  mark(name), if given, is called before each ABI call and once at the end
-        (used to drop CUDA events between the calls)."""
+        (used to drop CUDA events between the calls).  exchange: a sharding.StepExchange when this rank holds a block
+        of the batch rows (rows_global = rows of all ranks together); the collectives run on the current stream,
+        which must then be the stream the calls are enqueued on."""
         s = self.scalars
         M, K, N = self.M, self.K, self.N
         nlw, nlx = self.Pw.nlev, self.Px.nlev
@@ -210,12 +233,20 @@ class CdlLayerStep:
         m(CALLS[0]); cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, stream)
         m(CALLS[1]); cdl.cdl_index_entropy(self.hist_w, nlw, s[0:1], self.prob_w, None, stream)
         m(CALLS[2]); cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, stream)
+        if exchange is not None:
+            exchange.histogram(self.hist_x)          # level counts of the whole batch, before H(x) and prob_x
         m(CALLS[3]); cdl.cdl_index_entropy(self.hist_x, nlx, s[1:2], self.prob_x, None, stream)
         m(CALLS[4]); self._fwd(stream)
         m(CALLS[5]); cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, stream)
         # the two backward products are issued as two calls so that each can be timed on its own
         m(CALLS[6]); self._bwd_dx(stream)
-        m(CALLS[7]); self._bwd_dw(stream)
+        m(CALLS[7])
+        if exchange is None:
+            self._bwd_dw(stream)
+        else:
+            self._bwd_dw_exchanged(stream, exchange, rows_global if rows_global is not None else M * exchange.world)
         m(CALLS[8]); cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, s[4:5], s[5:6], stream)
         m(CALLS[9]); cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, s[2:3], s[3:4], stream)
+        if exchange is not None:
+            exchange.batch_scalars(s[4:6])           # dL/ds, dL/dbeta: sums over the batch; the rest is replicated
         m("end")

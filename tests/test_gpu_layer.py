@@ -287,6 +287,78 @@ def test_step_replayed_from_a_cuda_graph_equals_the_step_launched_call_by_call(t
     assert cdl.cdl_workspace_status(step.ws, check=False) == 0
 
 
+class _LoopbackCollective:
+    """Stands in for torch.distributed on one GPU: two ranks run one after the other.  In the recording pass every
+    tensor a rank hands to all_reduce is stored; in the second pass all_reduce returns the sum over both ranks."""
+
+    class ReduceOp:
+        SUM = "sum"
+
+    def __init__(self):
+        self.recorded, self.total, self.slot = {}, None, 0
+
+    def all_reduce(self, t, op=None):
+        key = self.slot
+        self.slot += 1
+        if self.total is None:
+            self.recorded.setdefault(key, []).append(t.clone())
+        else:
+            t.copy_(self.total[key])
+
+
+def test_two_row_blocks_with_the_exchange_equal_the_whole_batch(torch):
+    # the data-parallel step on one GPU: the batch rows are split in two blocks, each block runs the real kernels
+    # through CdlLayerStep.run(exchange=...), and what the exchange hands over is the sum of both blocks.  Histogram,
+    # entropy, level probabilities, dW, dL/dw and every row of dL/dx must be the bits of the whole-batch step.
+    from paper_2501_09849_b200 import sharding
+    from paper_2501_09849_b200.layer import CdlLayerStep
+    case, wt, at = inputs.tiny_layer(seed=6)
+    M, K, N = case.M, case.K, case.N
+    case.aq.window = 5
+    ai = oracle.hard(at, f32(case.aq.q), case.aq.lo, case.aq.hi)[0].astype(np.uint8).reshape(M, K)
+    dY = inputs.normal((M, N), 3e-2, seed=6, stream=7)
+    gx = inputs.normal((M, K), 1e-2, seed=6, stream=8)
+
+    def make(r0, r1):
+        st = CdlLayerStep(torch, r1 - r0, K, N, (r1 - r0) * K, case.wq, case.aq, q_g=1e-3)
+        st.w.copy_(dev(torch, wt).reshape(-1))
+        st.x.copy_(dev(torch, at[r0:r1]).reshape(-1))
+        st.A_idx[:, :K].copy_(dev(torch, ai[r0:r1]))
+        st.dY.copy_(dev(torch, dY[r0:r1]))
+        st.gx_in.copy_(dev(torch, gx[r0:r1]).reshape(-1))
+        return st
+
+    whole = make(0, M)
+    whole.run()
+    blocks = [sharding.row_range(M, r, 2) for r in range(2)]
+    parts = [make(r0, r1) for r0, r1 in blocks]
+    link = _LoopbackCollective()
+    for st in parts:                      # recording pass: what each rank would send
+        link.slot = 0
+        st.run(exchange=sharding.StepExchange(link, 2), rows_global=M)
+    torch.cuda.synchronize()
+    # the last recorded tensor (the two batch scalars) depends on the exchanged probabilities: take it from pass two
+    link.total = {k: v[0] + v[1] for k, v in link.recorded.items()}
+    scal = []
+    for st in parts:
+        link.slot = 0
+        ex = sharding.StepExchange(link, 2)
+        st.scalars.zero_()
+        orig = ex.batch_scalars
+        ex.batch_scalars = lambda t, orig=orig: scal.append(t.clone())      # summed by hand below
+        st.run(exchange=ex, rows_global=M)
+        assert [c[0] for c in ex.calls] == ["histogram", "accumulators"] and [c[1] for c in ex.calls] == ["int64", "int32"]
+    torch.cuda.synchronize()
+    for st in parts:
+        for k in ("hist_x", "prob_x", "dW", "dw", "hist_w", "prob_w", "W_idx"):
+            assert torch.equal(getattr(st, k), getattr(whole, k)), k
+        assert torch.equal(st.scalars[:4], whole.scalars[:4]) or torch.allclose(st.scalars[2:4], whole.scalars[2:4], rtol=1e-12)
+        assert torch.equal(st.scalars[:2], whole.scalars[:2])            # H(w) and H(x) of the whole batch, never a sum
+    assert torch.equal(torch.cat([st.dx for st in parts]), whole.dx)
+    assert torch.equal(torch.cat([st.Y for st in parts]), whole.Y)
+    assert torch.allclose(scal[0] + scal[1], whole.scalars[4:6], rtol=1e-11, atol=1e-14)
+
+
 def test_convolution_form_step_graph_equals_call_by_call(torch):
     # the three-stream recording of the step in convolution form has its own dependencies (the forward product waits
     # for X_idx, the activation backward pass for the data gradient): it must write what the serial step writes
