@@ -45,6 +45,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kBatch = 2;            // float4 loads in flight per thread
+constexpr int kHistCluster = 8;      // CTAs per cluster in launches that fill a histogram (portable cluster size)
 // streaming accesses: every element is touched once, so loads and stores bypass the usual cache retention
 #define CDL_LD(p) __ldcs(p)
 #define CDL_ST(p, v) __stcs(p, v)
@@ -107,7 +108,9 @@ __device__ __forceinline__ float philox_uniform(unsigned long long seed, unsigne
 // independent of the order in which elements arrive.
 __device__ __forceinline__ void mp_add(unsigned long long *mp_s, int bin, int lane, float P)
 {
-    atomicAdd(&mp_s[bin * 32 + lane], (unsigned long long)__float2uint_rn(P * 4294967296.0f));
+    // a reduction on a 32-bit shared-window address (no result, no generic-address arithmetic)
+    const unsigned int a = (unsigned int)__cvta_generic_to_shared(mp_s) + (unsigned int)(((bin << 5) + lane) << 3);
+    asm volatile("red.shared.add.u64 [%0], %1;" ::"r"(a), "l"((unsigned long long)__float2uint_rn(P * 4294967296.0f)) : "memory");
 }
 
 struct ElemOut {
@@ -607,9 +610,43 @@ __device__ __forceinline__ void quant_quad_lattice(const QuantDev &P, const floa
     o[1] = lattice_finish<MODE>(P, s1, make_float2(gs[2], gs[3]));
 }
 
-__device__ __forceinline__ void hist_add(unsigned int *hist_s, int bin, int lane)
+// ---- thread-block cluster helpers (a launch without a cluster attribute is a cluster of one CTA)
+__device__ __forceinline__ unsigned int cluster_ctarank()
 {
-    atomicAdd(&hist_s[bin * 32 + lane], 1u);
+    unsigned int r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ unsigned int cluster_nctarank()
+{
+    unsigned int r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the 64-bit word at the same shared-memory offset as `p` in CTA `rank` of the cluster
+__device__ __forceinline__ unsigned long long ld_cluster_u64(const unsigned long long *p, unsigned int rank)
+{
+    unsigned long long v;
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
+        "ld.shared::cluster.u64 %0, [ra];\n\t}"
+        : "=l"(v)
+        : "r"((unsigned int)__cvta_generic_to_shared(p)), "r"(rank)
+        : "memory");
+    return v;
+}
+
+// One more element at level k.  hist_a is the 32-bit shared-window address of this lane's counter of level 0 (the
+// counters of one level are 32 consecutive words, one per lane, so a warp never meets a bank conflict): one address
+// computation and one reduction per element.
+__device__ __forceinline__ void hist_inc(unsigned int hist_a, int k)
+{
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(hist_a + ((unsigned int)k << 7)), "r"(1u) : "memory");
 }
 
 // Vector region: elements [head, head + 4 n4); the remaining head + tail elements are done one by one.
@@ -666,7 +703,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         for (int k = threadIdx.x; k < P.nlev * 32; k += kThreads) hist_s[k] = 0u;
     if (RATE || do_hist || PATH == PATH_LATTICE) __syncthreads();
 
-    unsigned int *const hist_l = hist_s + (lane - P.lo * 32);    // this lane's column, indexed by level: hist_l[k * 32]
+    // this lane's column of the index histogram, addressed by level: level k sits at hist_a + 128 k
+    const unsigned int hist_a = (unsigned int)__cvta_generic_to_shared(hist_s) + (unsigned int)((lane - P.lo * 32) * 4);
     double acc_q = 0.0, acc_a = 0.0;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
     const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -751,8 +789,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                         packed = h == 0 ? __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040)
                                         : __byte_perm(packed, __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040), 0x5410);
                         if (MODE != MODE_BWD && do_hist) {
-                            atomicAdd(hist_l + o.k0[0] * 32, 1u);
-                            atomicAdd(hist_l + o.k0[1] * 32, 1u);
+                            hist_inc(hist_a, o.k0[0]);
+                            hist_inc(hist_a, o.k0[1]);
                         }
                     }
                 }
@@ -764,8 +802,8 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                         packed = h == 0 ? __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040)
                                         : __byte_perm(packed, __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040), 0x5410);
                         if (do_hist) {
-                            atomicAdd(hist_l + k0 * 32, 1u);
-                            atomicAdd(hist_l + k1 * 32, 1u);
+                            hist_inc(hist_a, k0);
+                            hist_inc(hist_a, k1);
                         }
                     }
                 }
@@ -778,7 +816,7 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
                     part_q += o.tq;
                     part_a += o.ta;
                     packed |= ((unsigned int)o.k0 & 0xffu) << (8 * c);
-                    if (MODE != MODE_BWD && do_hist) hist_add(hist_s, o.k0 - P.lo, lane);
+                    if (MODE != MODE_BWD && do_hist) hist_inc(hist_a, o.k0);
                 }
                 if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) CDL_ST(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
                 if (MODE == MODE_BWD && gx != nullptr) CDL_ST(gx4 + i, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
@@ -806,27 +844,51 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
             acc_a += (double)o.ta;
         } else {
             if (idx != nullptr) idx[i] = (unsigned char)((unsigned int)o.k0 & 0xffu);
-            if (do_hist) hist_add(hist_s, o.k0 - P.lo, lane);
+            if (do_hist) hist_inc(hist_a, o.k0);
         }
     }
 
-    if (MODE == MODE_SOFT && RATE) {   // RATE doubles as "soft histogram requested" in the soft pass
+    // Histograms leave the CTA in two steps.  Each CTA adds up its 32 lane-private columns; then the CTAs of a
+    // thread-block cluster (kHistCluster of them when a histogram is asked for) read one another's totals through
+    // distributed shared memory, every CTA taking the bins congruent to its rank, and only these cluster sums go to
+    // global memory.  All blocks hit the same few addresses there, and those reductions are served one at a time:
+    // with one reduction per bin per CTA they cost as much as a quarter of a launch on a 13 M-element tensor.
+    const bool do_mp = MODE == MODE_SOFT && RATE;   // RATE doubles as "soft histogram requested" in the soft pass
+    if (MODE != MODE_BWD && (do_hist || do_mp)) {
+        unsigned long long *tot_c = reinterpret_cast<unsigned long long *>(
+            smem_raw + CDL_MAX_LEVELS * sizeof(float) + (do_hist ? (size_t)P.nlev * 32 * sizeof(unsigned int) : 0) +
+            (do_mp ? (size_t)P.nlev * 32 * sizeof(unsigned long long) : 0));
+        unsigned long long *tot_m = tot_c + P.nlev;
         __syncthreads();
         const int warp = threadIdx.x >> 5;
         for (int b = warp; b < P.nlev; b += kThreads / 32) {
-            unsigned long long c = mp_s[b * 32 + lane];
+            if (do_hist) {
+                const unsigned int c = __reduce_add_sync(0xffffffffu, hist_s[b * 32 + lane]);
+                if (lane == 0) tot_c[b] = c;
+            }
+            if (do_mp) {
+                unsigned long long c = mp_s[b * 32 + lane];
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) c += __shfl_down_sync(0xffffffffu, c, off);
-            if (lane == 0 && c != 0ull) atomicAdd(&mp[b], c);
+                for (int off = 16; off > 0; off >>= 1) c += __shfl_down_sync(0xffffffffu, c, off);
+                if (lane == 0) tot_m[b] = c;
+            }
         }
-    }
-    if (MODE != MODE_BWD && do_hist) {
-        __syncthreads();
-        const int warp = threadIdx.x >> 5;
-        for (int b = warp; b < P.nlev; b += kThreads / 32) {
-            const unsigned int c = __reduce_add_sync(0xffffffffu, hist_s[b * 32 + lane]);
-            if (lane == 0 && c != 0u) atomicAdd(&hist[b], (unsigned long long)c);
+        cluster_sync_all();                        // every CTA's totals are in place (also orders them within the CTA)
+        const unsigned int csize = cluster_nctarank(), crank = cluster_ctarank();
+        for (int b = threadIdx.x; b < P.nlev; b += kThreads) {
+            if ((unsigned int)b % csize != crank) continue;
+            if (do_hist) {
+                unsigned long long sum = 0ull;
+                for (unsigned int r = 0; r < csize; ++r) sum += ld_cluster_u64(&tot_c[b], r);
+                if (sum != 0ull) atomicAdd(&hist[b], sum);
+            }
+            if (do_mp) {
+                unsigned long long sum = 0ull;
+                for (unsigned int r = 0; r < csize; ++r) sum += ld_cluster_u64(&tot_m[b], r);
+                if (sum != 0ull) atomicAdd(&mp[b], sum);
+            }
         }
+        cluster_sync_all();                        // no CTA leaves while another may still read its totals
     }
     if (MODE == MODE_BWD && (gq != nullptr || ga != nullptr)) {
         __shared__ double red[2][kThreads / 32];
@@ -858,8 +920,10 @@ int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int6
              float *y, unsigned char *idx, unsigned long long *hist, float *gx, double *gq, double *ga,
              unsigned long long *mp, cudaStream_t stream)
 {
+    const bool histo = MODE != MODE_BWD && (hist != nullptr || mp != nullptr);
     const size_t smem = CDL_MAX_LEVELS * sizeof(float) + (hist ? (size_t)qd.nlev * 32 * sizeof(unsigned int) : 0) +
-                        (mp ? (size_t)qd.nlev * 32 * sizeof(unsigned long long) : 0);
+                        (mp ? (size_t)qd.nlev * 32 * sizeof(unsigned long long) : 0) +
+                        (histo ? 2 * (size_t)qd.nlev * sizeof(unsigned long long) : 0);     // per-CTA totals of both histograms
     auto kern = quantize_kernel<MODE, PATH, RATE>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -879,8 +943,36 @@ int launch_t(const QuantDev &qd, const float *x, const float *g, int64_t n, int6
     const int64_t cap = (int64_t)sms * per_sm;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    kern<<<(unsigned int)blocks, kThreads, smem, stream>>>(qd, x, g, n, head, n4, y, idx, hist, gx, gq, ga, mp);
-    return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
+    if (!histo) {
+        kern<<<(unsigned int)blocks, kThreads, smem, stream>>>(qd, x, g, n, head, n4, y, idx, hist, gx, gq, ga, mp);
+        return cudaGetLastError() == cudaSuccess ? CDL_OK : CDL_ERR_LAUNCH;
+    }
+    // histogram launches: clusters of kHistCluster CTAs (CTAs without elements still take part in the reduction)
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kHistCluster;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3((unsigned int)(cap / kHistCluster * kHistCluster));
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
+        (void)cudaGetLastError();
+        max_clusters = (int)(cap / kHistCluster) > 0 ? (int)(cap / kHistCluster) : 1;
+    }
+    int64_t clusters = (blocks + kHistCluster - 1) / kHistCluster;
+    if (clusters > max_clusters) clusters = max_clusters;
+    cfg.gridDim = dim3((unsigned int)(clusters * kHistCluster));
+    if (cudaLaunchKernelEx(&cfg, kern, qd, x, g, n, head, n4, y, idx, hist, gx, gq, ga, mp) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CDL_ERR_LAUNCH;
+    }
+    return CDL_OK;
 }
 
 inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
