@@ -97,7 +97,55 @@ struct TcParams {
     int nq_fast, nq_vec;    // reciprocal product allowed; rows can be written 16 bytes at a time
     int slab_rows;          // 0: splits add into one I x J buffer.  > 0: split s stores its partial tile into rows
                             // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
+    int slots;              // work slots (CTA pairs, or CTAs) = the grid: slot p takes units p, p + slots, ...
 };
+
+// One piece of work of a slot: pipeline stages [rb0, rb1) of a tile (a unit of tiles * splits).
+struct WorkItem {
+    int valid;
+    int tile, split, rb0, rb1;
+};
+
+// The units of a slot, in order.  The threads that walk them are single lanes on the critical path of the pipeline
+// (TMA producers, MMA issuer), and a product with a short reduced dimension has thousands of units of two or three
+// stages each: stepping to the next unit is an addition, with divisions only when the reduced dimension is split
+// (then a slot has few units).
+struct SlotWork {
+    long long units, u;
+    int slots, rblocks, splits;
+};
+
+__device__ __forceinline__ SlotWork slot_work(const TcParams &P, int p)
+{
+    SlotWork s;
+    s.units = (long long)P.tiles_i * P.tiles_j * P.splits;
+    s.u = p;
+    s.slots = P.slots;
+    s.rblocks = P.rblocks;
+    s.splits = P.splits;
+    return s;
+}
+
+__device__ __forceinline__ WorkItem next_item(SlotWork &s)
+{
+    WorkItem w;
+    w.valid = s.u < s.units;
+    if (s.splits == 1) {
+        w.tile = (int)s.u;
+        w.split = 0;
+        w.rb0 = 0;
+        w.rb1 = s.rblocks;
+    } else {
+        const unsigned int u32 = (unsigned int)s.u, sp = (unsigned int)s.splits;      // units < 2^31 (checked by the launcher)
+        const unsigned int tile = u32 / sp, split = u32 - tile * sp;
+        w.tile = (int)tile;
+        w.split = (int)split;
+        w.rb0 = (int)(((long long)s.rblocks * split) / sp);
+        w.rb1 = (int)(((long long)s.rblocks * (split + 1u)) / sp);
+    }
+    s.u += s.slots;
+    return w;
+}
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
@@ -315,8 +363,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     static_assert(kStages * kStageBytes + kEpiWarps * kOutBlocks * kOutWarpBytes + 1024 <= kSmemBytes, "shared memory");
     constexpr int TMU = PAIR ? 2 * TM : TM;                   // rows of a work unit's tile
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // CTA 0 of a pair issues the MMAs
-    const int cta_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int cta_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int slot = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;     // this CTA's (pair's) work slot, of P.slots
 
     auto full_bar = [&](int s) { return smem_u32(&bars[s]); };
     auto empty_bar = [&](int s) { return smem_u32(&bars[kStagesMax + s]); };
@@ -352,7 +399,6 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    const int units = P.tiles_i * P.tiles_j * P.splits;
     const int b_blocks = PAIR ? 1 : (P.TN + 127) / 128;                   // 128-wide blocks of an MN-major B tile
     const uint32_t b_bytes = PAIR ? (uint32_t)(128 * BR)
                                   : (P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR));
@@ -366,12 +412,13 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const bool do_a = warp == 0, do_b = !kSplitProducer || warp != 0;
         if (lane == 0) {
             uint32_t it = 0;
-            for (int u = cta_first; u < units && !failed; u += cta_step) {
-                const int split = u % P.splits;
-                const int tile = u / P.splits;
+            SlotWork sw = slot_work(P, slot);
+            while (!failed) {
+                const WorkItem w = next_item(sw);
+                if (!w.valid) break;
+                const int tile = w.tile;
                 const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
-                const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
-                const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
+                const int rb0 = w.rb0, rb1 = w.rb1;
                 const int arow = ti * TMU + (int)rank * TM;
                 // Patch gather: pixel block, channel block and filter tap of the first stage of this unit, kept up
                 // to date with additions only inside the loop (this one thread feeds the whole pipeline).
@@ -465,10 +512,11 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // ------------------------------------------------------------ MMA issuer (one lane; CTA 0 in pair mode)
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, tcount = 0;
-            for (int u = cta_first; u < units && !failed; u += cta_step, ++tcount) {
-                const int split = u % P.splits;
-                const int rb0 = (int)(((long long)P.rblocks * split) / P.splits);
-                const int rb1 = (int)(((long long)P.rblocks * (split + 1)) / P.splits);
+            SlotWork sw = slot_work(P, slot);
+            for (; !failed; ++tcount) {
+                const WorkItem w = next_item(sw);
+                if (!w.valid) break;
+                const int rb0 = w.rb0, rb1 = w.rb1;
                 const int buf = tcount & 1;
                 const uint32_t tph = (tcount >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, P.wait_ns)) {
@@ -571,10 +619,13 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             __syncwarp();
         };
 
-        for (int u = cta_first; u < units; u += cta_step, ++tcount) {
-            const int tile = u / P.splits;
+        SlotWork sw = slot_work(P, slot);
+        for (;; ++tcount) {
+            const WorkItem w = next_item(sw);
+            if (!w.valid) break;
+            const int tile = w.tile;
             const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
-            const int slab_row0 = (u % P.splits) * P.slab_rows;     // 0 unless partial tiles go to per-split slabs
+            const int slab_row0 = w.split * P.slab_rows;             // 0 unless partial tiles go to per-split slabs
             const int buf = tcount & 1;
             const uint32_t tph = (tcount >> 1) & 1u;
             // the epilogue warps agree on the outcome, so that either all of them or none release the accumulator
@@ -909,7 +960,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const int sms = sm_count();
     if (sms <= 0) return CDL_ERR_LAUNCH;
     const long long tiles = (long long)P.tiles_i * P.tiles_j;
-    if (tiles > 0x3fffffff) return CDL_ERR_ARG;
+    if (tiles > 0x3fffffff || tiles * splits > 0x7fffffff) return CDL_ERR_ARG;
     P.splits = splits;
     P.a_mn_major = a_mn ? 1 : 0;
     P.b_mn_major = b_mn ? 1 : 0;
@@ -1023,18 +1074,19 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         attr_set[dev] = true;
     }
     const long long units = tiles * splits;
+    const int dev_slots = pair ? pair_slots[dev] : sms;
+    P.slots = (int)(units < dev_slots ? units : dev_slots);
     // bytes a CTA loads per work unit against the bytes it stores (4-byte outputs of a 128 x TN tile)
     const long long unit_load = (long long)((P.rblocks + splits - 1) / splits) * (kABytes + (pair ? 128 : TN) * BR);
     const bool store_heavy = unit_load <= 2ll * TM * TN * 4;
     if (pair) {
-        const int slots = pair_slots[dev];
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2;
         at[0].val.clusterDim.y = 1;
         at[0].val.clusterDim.z = 1;
-        cfg.gridDim = dim3(2u * (unsigned)(units < slots ? units : slots));
+        cfg.gridDim = dim3(2u * (unsigned)P.slots);
         cfg.blockDim = dim3(threads_tc(store_heavy));
         cfg.dynamicSmemBytes = kSmemBytes;
         cfg.stream = stream;
@@ -1047,9 +1099,8 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
             return CDL_ERR_LAUNCH;
         }
     } else {
-        const int grid = (int)(units < sms ? units : sms);
-        if (store_heavy) index_gemm_tc_kernel<false, true><<<grid, threads_tc(true), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
-        else index_gemm_tc_kernel<false, false><<<grid, threads_tc(false), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        if (store_heavy) index_gemm_tc_kernel<false, true><<<P.slots, threads_tc(true), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
+        else index_gemm_tc_kernel<false, false><<<P.slots, threads_tc(false), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (f_out != nullptr && (splits > 1 || slabs)) {

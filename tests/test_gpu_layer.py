@@ -243,6 +243,61 @@ def test_resnet18_conv1_and_fc_shapes(torch):
     check_all_products(torch, A, W, G, cdl.IndexDesc(0.25, 0, 15), w, g)
 
 
+def test_float_only_outputs_with_a_ragged_last_round_of_tiles(torch):
+    # 89 x 2 tiles of 256 x 256 on 74 CTA-pair slots: two whole rounds and 30 tiles left over, ragged in all three
+    # dimensions, float output only.  Every element of the float output must equal the int32 accumulators of a
+    # second run times the step product, bit for bit; the accumulators themselves are compared with the oracle on
+    # rows of the last round's tiles (the last 15 tile rows), of the earlier rounds and of both edges.  A bias goes
+    # through the same path; repeated calls on the same buffers give the same bits.
+    M, K, N = 89 * 256 - 100, 1584, 384
+    A = inputs.uniform_indices((M, K), 0, 15, seed=61)
+    W = inputs.uniform_indices((K, N), -7, 7, seed=62)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=63)
+    a, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    bias = inputs.normal((N,), 1.0, seed=64)
+    acc, _ = run_fwd(torch, A, W, a, w, want_y=False)
+    for rep in range(2):
+        _, y = run_fwd(torch, A, W, a, w, want_acc=False)
+        assert np.array_equal(y, scaled(acc.astype(np.int64), a.q, w.q)), rep
+    _, yb = run_fwd(torch, A, W, a, w, bias=bias, want_acc=False)
+    assert np.array_equal(yb, scaled(acc.astype(np.int64), a.q, w.q, bias))
+    rng = np.random.default_rng(2)
+    rows = np.unique(np.concatenate([np.arange(0, 3), np.arange(M - 3, M), np.arange(74 * 256 - 2, 74 * 256 + 2),
+                                     rng.integers(74 * 256, M, size=200), rng.integers(0, 74 * 256, size=100)]))
+    assert np.array_equal(acc[rows].astype(np.int64), oracle.gemm_fwd(A[rows], W))
+    # dX of the same shape family: (M, N) x (K, N)^T with K = 512 -> 89 x 2 tiles again, reduced dimension N = 1584
+    M2, N2, K2 = M, 1584, 512
+    G2 = inputs.uniform_indices((M2, N2), -127, 127, seed=65)
+    W2 = inputs.uniform_indices((K2, N2), -7, 7, seed=66)
+    full = run_bwd(torch, G2, None, W2, g, None, w, want=("dXacc",))["dXacc"]
+    only = run_bwd(torch, G2, None, W2, g, None, w, want=("dX",))["dX"]
+    assert np.array_equal(only, scaled(full.astype(np.int64), g.q, w.q))
+    assert np.array_equal(full[rows].astype(np.int64), oracle.gemm_dx(G2[rows], W2))
+
+
+@pytest.mark.parametrize("M,K,N", [(4096 + 5, 640, 512), (300, 2304, 256), (50176, 256, 272), (1031, 1152, 1000)])
+def test_float_only_outputs_with_fewer_tiles_than_slots(torch, M, K, N):
+    # Products with fewer 256 x 256 tiles than CTA-pair slots and float outputs only: the reduced dimension is split
+    # over the slots (the weight gradient reduces over M with a handful of tiles); all three products against the oracle.
+    A = inputs.uniform_indices((M, K), 0, 15, seed=M % 97)
+    W = inputs.uniform_indices((K, N), -7, 7, seed=K % 97)
+    G = inputs.uniform_indices((M, N), -127, 127, seed=N % 97)
+    a, w, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(0.02, -7, 7), cdl.IndexDesc(1e-3, -127, 127)
+    _, y = run_fwd(torch, A, W, a, w, want_acc=False)
+    out = run_bwd(torch, G, A, W, g, a, w, want=("dX", "dW"))
+    if M * K * N <= 3e9:
+        assert np.array_equal(y, scaled(oracle.gemm_fwd(A, W), a.q, w.q))
+        assert np.array_equal(out["dX"], scaled(oracle.gemm_dx(G, W), g.q, w.q))
+        assert np.array_equal(out["dW"], scaled(oracle.gemm_dw(A, G), g.q, a.q))
+    else:
+        rng = np.random.default_rng(3)
+        rows = np.unique(np.concatenate([np.arange(0, 2), np.arange(M - 2, M), rng.integers(0, M, size=200)]))
+        assert np.array_equal(y[rows], scaled(oracle.gemm_fwd(A[rows], W), a.q, w.q))
+        assert np.array_equal(out["dX"][rows], scaled(oracle.gemm_dx(G[rows], W), g.q, w.q))
+        ks = np.unique(np.concatenate([[0, 1, K - 1], rng.integers(0, K, size=12)]))
+        assert np.array_equal(out["dW"][ks], scaled(oracle.gemm_dw(np.ascontiguousarray(A[:, ks]), G), g.q, a.q))
+
+
 def test_step_replayed_from_a_cuda_graph_equals_the_step_launched_call_by_call(torch):
     # the recorded step must write exactly what the eager step writes (same kernels, same launch shapes); the
     # products themselves are checked against the oracle above
