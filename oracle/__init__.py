@@ -56,9 +56,9 @@ def _load():
         lib.cdl_oracle_gemm_fwd.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dx.argtypes = [P, c.c_int64, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
         lib.cdl_oracle_gemm_dw.argtypes = [P, c.c_int64, c.c_int, P, c.c_int64, c.c_int, c.c_int, c.c_int, P]
-        lib.cdl_oracle_conv_fwd.argtypes = [P, c.c_int, P, c.c_int64] + [c.c_int] * 9 + [P]
-        lib.cdl_oracle_conv_dx.argtypes = [P, P, c.c_int64] + [c.c_int] * 9 + [P]
-        lib.cdl_oracle_conv_dw.argtypes = [P, c.c_int, P] + [c.c_int] * 9 + [P]
+        lib.cdl_oracle_conv_fwd.argtypes = [P, c.c_int, P, c.c_int64] + [c.c_int] * 10 + [P]
+        lib.cdl_oracle_conv_dx.argtypes = [P, P, c.c_int64] + [c.c_int] * 10 + [P]
+        lib.cdl_oracle_conv_dw.argtypes = [P, c.c_int, P] + [c.c_int] * 10 + [P]
         for f in (lib.cdl_oracle_conv_fwd, lib.cdl_oracle_conv_dx, lib.cdl_oracle_conv_dw):
             f.restype = None
         lib.cdl_oracle_mpmf.argtypes = [P, c.c_int64, c.c_float, c.c_int, c.c_int, c.c_float, c.c_int, P]
@@ -219,40 +219,44 @@ def _conv_dims(X, Wt, R, S):
     return X, Wt, ldw, (N, H, W, C), Wt.shape[1]
 
 
-def conv_fwd(X, Wt, R, S, pad_h, pad_w):
-    """Stride-1 cross-correlation with zero padding on indices, int64: X [N,H,W,C] int8|uint8, Wt [(r*S+s)*C+c, CO]
+def conv_out_dims(H, W, R, S, pad_h, pad_w, stride=1):
+    return (H + 2 * pad_h - R) // stride + 1, (W + 2 * pad_w - S) // stride + 1
+
+
+def conv_fwd(X, Wt, R, S, pad_h, pad_w, stride=1):
+    """Strided cross-correlation with zero padding on indices, int64: X [N,H,W,C] int8|uint8, Wt [(r*S+s)*C+c, CO]
     int8 -> [N,P,Q,CO]."""
     X, Wt, ldw, (N, H, W, C), CO = _conv_dims(X, Wt, R, S)
-    P, Q = H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1
+    P, Q = conv_out_dims(H, W, R, S, pad_h, pad_w, stride)
     acc = np.empty((N, P, Q, CO), dtype=np.int64)
     _load().cdl_oracle_conv_fwd(_ptr(X), int(X.dtype == np.uint8), _ptr(Wt), ldw, N, H, W, C, R, S, pad_h, pad_w, CO,
-                                _ptr(acc))
+                                stride, _ptr(acc))
     return acc
 
 
-def conv_dx(G, Wt, x_shape, R, S, pad_h, pad_w):
+def conv_dx(G, Wt, x_shape, R, S, pad_h, pad_w, stride=1):
     """Adjoint of conv_fwd in X: G [N,P,Q,CO] int8, Wt as in conv_fwd -> [N,H,W,C] int64."""
     N, H, W, C = x_shape
     G = np.ascontiguousarray(G)
     Wt, ldw, wu = _idx_bytes(Wt)
     CO = Wt.shape[1]
     assert G.dtype == np.int8 and not wu and Wt.shape[0] == R * S * C
-    assert G.shape == (N, H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1, CO)
+    assert G.shape == (N,) + conv_out_dims(H, W, R, S, pad_h, pad_w, stride) + (CO,)
     acc = np.empty((N, H, W, C), dtype=np.int64)
-    _load().cdl_oracle_conv_dx(_ptr(G), _ptr(Wt), ldw, N, H, W, C, R, S, pad_h, pad_w, CO, _ptr(acc))
+    _load().cdl_oracle_conv_dx(_ptr(G), _ptr(Wt), ldw, N, H, W, C, R, S, pad_h, pad_w, CO, stride, _ptr(acc))
     return acc
 
 
-def conv_dw(X, G, R, S, pad_h, pad_w):
+def conv_dw(X, G, R, S, pad_h, pad_w, stride=1):
     """Adjoint of conv_fwd in Wt: X [N,H,W,C] int8|uint8, G [N,P,Q,CO] int8 -> [(r*S+s)*C+c, CO] int64."""
     X = np.ascontiguousarray(X)
     G = np.ascontiguousarray(G)
     N, H, W, C = X.shape
     CO = G.shape[3]
     assert X.dtype in (np.int8, np.uint8) and G.dtype == np.int8
-    assert G.shape == (N, H + 2 * pad_h - R + 1, W + 2 * pad_w - S + 1, CO)
+    assert G.shape == (N,) + conv_out_dims(H, W, R, S, pad_h, pad_w, stride) + (CO,)
     acc = np.empty((R * S * C, CO), dtype=np.int64)
-    _load().cdl_oracle_conv_dw(_ptr(X), int(X.dtype == np.uint8), _ptr(G), N, H, W, C, R, S, pad_h, pad_w, CO,
+    _load().cdl_oracle_conv_dw(_ptr(X), int(X.dtype == np.uint8), _ptr(G), N, H, W, C, R, S, pad_h, pad_w, CO, stride,
                                _ptr(acc))
     return acc
 

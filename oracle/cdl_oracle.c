@@ -425,21 +425,23 @@ void cdl_oracle_gemm_dw(const void *A, int64_t lda, int a_unsigned,
 }
 
 /* -------------------------------------------------------------------------
- * Convolutional layer products on index tensors.  The paper's networks are CNNs (Sec. VI-C, VI-D: ResNets) whose
- * layers apply the quantized weights to the quantized activations (Algorithm 1, forward and backward over the
- * quantized tensors); the convolution itself is the textbook cross-correlation with zero padding, stride 1:
+ * Convolutional layer products on index tensors.  The paper's networks are CNNs (Sec. VI-C, VI-D: ResNets, whose
+ * stages begin with stride-2 layers) whose layers apply the quantized weights to the quantized activations
+ * (Algorithm 1, forward and backward over the quantized tensors); the convolution itself is the textbook strided
+ * cross-correlation with zero padding:
  *   X [N,H,W,C] (index bytes), Wt [(r*S+s)*C + c, co] (int8, row pitch ldw), G [N,P,Q,CO] (int8),
- *   P = H + 2 pad_h - R + 1,  Q = W + 2 pad_w - S + 1
- *   fwd : Y [n,p,q,co]        = sum_{r,s,c}  X[n, p-pad_h+r, q-pad_w+s, c] * Wt[(r*S+s)*C+c, co]
- *   dX  : dX[n,h,w,c]         = sum_{r,s,co} G[n, h+pad_h-r, w+pad_w-s, co] * Wt[(r*S+s)*C+c, co]
- *   dW  : dW[(r*S+s)*C+c, co] = sum_{n,p,q}  X[n, p-pad_h+r, q-pad_w+s, c] * G[n,p,q,co]
+ *   P = (H + 2 pad_h - R) / stride + 1,  Q = (W + 2 pad_w - S) / stride + 1   (integer division)
+ *   fwd : Y [n,p,q,co]        = sum_{r,s,c}  X[n, p*stride-pad_h+r, q*stride-pad_w+s, c] * Wt[(r*S+s)*C+c, co]
+ *   dX  : dX[n,h,w,c]         = sum over (r,s,co) and the (p,q) with p*stride-pad_h+r = h, q*stride-pad_w+s = w
+ *                               of G[n,p,q,co] * Wt[(r*S+s)*C+c, co]
+ *   dW  : dW[(r*S+s)*C+c, co] = sum_{n,p,q}  X[n, p*stride-pad_h+r, q*stride-pad_w+s, c] * G[n,p,q,co]
  * (a term whose spatial position falls outside the tensor is zero).  dX and dW are the adjoints of fwd in X and
  * in Wt.  Sums are int64.
  * ------------------------------------------------------------------------- */
 void cdl_oracle_conv_fwd(const void *X, int x_unsigned, const int8_t *Wt, int64_t ldw, int N, int H, int W, int C,
-                         int R, int S, int pad_h, int pad_w, int CO, int64_t *acc)
+                         int R, int S, int pad_h, int pad_w, int CO, int stride, int64_t *acc)
 {
-    const int P = H + 2 * pad_h - R + 1, Q = W + 2 * pad_w - S + 1;
+    const int P = (H + 2 * pad_h - R) / stride + 1, Q = (W + 2 * pad_w - S) / stride + 1;
 #pragma omp parallel for schedule(static) collapse(2)
     for (int n = 0; n < N; ++n)
         for (int p = 0; p < P; ++p)
@@ -447,10 +449,10 @@ void cdl_oracle_conv_fwd(const void *X, int x_unsigned, const int8_t *Wt, int64_
                 for (int co = 0; co < CO; ++co) {
                     int64_t sum = 0;
                     for (int r = 0; r < R; ++r) {
-                        const int h = p - pad_h + r;
+                        const int h = p * stride - pad_h + r;
                         if (h < 0 || h >= H) continue;
                         for (int s = 0; s < S; ++s) {
-                            const int w = q - pad_w + s;
+                            const int w = q * stride - pad_w + s;
                             if (w < 0 || w >= W) continue;
                             for (int c = 0; c < C; ++c)
                                 sum += ld_idx(X, (((int64_t)n * H + h) * W + w) * C + c, x_unsigned) *
@@ -462,9 +464,9 @@ void cdl_oracle_conv_fwd(const void *X, int x_unsigned, const int8_t *Wt, int64_
 }
 
 void cdl_oracle_conv_dx(const int8_t *G, const int8_t *Wt, int64_t ldw, int N, int H, int W, int C,
-                        int R, int S, int pad_h, int pad_w, int CO, int64_t *acc)
+                        int R, int S, int pad_h, int pad_w, int CO, int stride, int64_t *acc)
 {
-    const int P = H + 2 * pad_h - R + 1, Q = W + 2 * pad_w - S + 1;
+    const int P = (H + 2 * pad_h - R) / stride + 1, Q = (W + 2 * pad_w - S) / stride + 1;
 #pragma omp parallel for schedule(static) collapse(2)
     for (int n = 0; n < N; ++n)
         for (int h = 0; h < H; ++h)
@@ -472,11 +474,13 @@ void cdl_oracle_conv_dx(const int8_t *G, const int8_t *Wt, int64_t ldw, int N, i
                 for (int c = 0; c < C; ++c) {
                     int64_t sum = 0;
                     for (int r = 0; r < R; ++r) {
-                        const int p = h + pad_h - r;
-                        if (p < 0 || p >= P) continue;
+                        const int ph = h + pad_h - r;            /* = p * stride for the output row that reads h at tap r */
+                        if (ph < 0 || ph % stride != 0 || ph / stride >= P) continue;
+                        const int p = ph / stride;
                         for (int s = 0; s < S; ++s) {
-                            const int q = w + pad_w - s;
-                            if (q < 0 || q >= Q) continue;
+                            const int qw = w + pad_w - s;
+                            if (qw < 0 || qw % stride != 0 || qw / stride >= Q) continue;
+                            const int q = qw / stride;
                             for (int co = 0; co < CO; ++co)
                                 sum += (int64_t)G[(((int64_t)n * P + p) * Q + q) * CO + co] *
                                        (int64_t)Wt[((int64_t)(r * S + s) * C + c) * ldw + co];
@@ -487,9 +491,9 @@ void cdl_oracle_conv_dx(const int8_t *G, const int8_t *Wt, int64_t ldw, int N, i
 }
 
 void cdl_oracle_conv_dw(const void *X, int x_unsigned, const int8_t *G, int N, int H, int W, int C,
-                        int R, int S, int pad_h, int pad_w, int CO, int64_t *acc)
+                        int R, int S, int pad_h, int pad_w, int CO, int stride, int64_t *acc)
 {
-    const int P = H + 2 * pad_h - R + 1, Q = W + 2 * pad_w - S + 1;
+    const int P = (H + 2 * pad_h - R) / stride + 1, Q = (W + 2 * pad_w - S) / stride + 1;
 #pragma omp parallel for schedule(static) collapse(2)
     for (int r = 0; r < R; ++r)
         for (int s = 0; s < S; ++s)
@@ -498,10 +502,10 @@ void cdl_oracle_conv_dw(const void *X, int x_unsigned, const int8_t *G, int N, i
                     int64_t sum = 0;
                     for (int n = 0; n < N; ++n)
                         for (int p = 0; p < P; ++p) {
-                            const int h = p - pad_h + r;
+                            const int h = p * stride - pad_h + r;
                             if (h < 0 || h >= H) continue;
                             for (int q = 0; q < Q; ++q) {
-                                const int w = q - pad_w + s;
+                                const int w = q * stride - pad_w + s;
                                 if (w < 0 || w >= W) continue;
                                 sum += ld_idx(X, (((int64_t)n * H + h) * W + w) * C + c, x_unsigned) *
                                        (int64_t)G[(((int64_t)n * P + p) * Q + q) * CO + co];
