@@ -790,7 +790,7 @@ def network_step(torch, cdl, batch, conv_form, steps, warm, use_graph=True):
         wq = inputs.Quantizer(float(w.std()) / 3.0, -3, 3, 100.0, 0.01, 0)
         xq = inputs.Quantizer(float(2.0 * x.mean() / 8.0 ** 0.5), 0, 15, 100.0, 0.01, 5)
         geo = inputs.resnet18_conv_geometry(name) if conv_form else None
-        shape = cdl.ConvShape(batch, *geo) if geo else None
+        shape = cdl.ConvShape(batch, geo[0], geo[1], geo[2], geo[3], geo[4], geo[5], geo[6], geo[6]) if geo else None
         st = CdlLayerStep(torch, M, K, Np, n_x, wq, xq, q_g, need_dx=(name != "conv1"), conv=shape)   # the image needs no gradient
         st.w.copy_(w)
         st.x.copy_(x)

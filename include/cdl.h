@@ -317,28 +317,33 @@ int cdl_noalloc_status(void *stream);
 
 /*
  * The same three layer products for a convolutional layer (the layers of the paper's networks, Sec. VI-C and
- * VI-D, are convolutions; Algorithm 1, forward and backward pass), computed straight from the NHWC index
- * tensors: the patch matrix whose rows cdl_qlinear_* takes as A_idx is never written to memory, its tiles are
- * gathered by the loads of the kernel, with zero (= index 0 = level 0) outside the image.
- * Stride 1, filter R x S with R and S odd, padding (R-1)/2 and (S-1)/2: the output has the spatial size of the
- * input (3 x 3 and 1 x 1 layers of a ResNet).  C and C_out multiples of 64 (else CDL_ERR_ARG: form the patch
- * matrix and call cdl_qlinear_*).
- *   X_idx [dev] N x H x W x C index bytes (signedness from x);  G_idx [dev] N x H x W x C_out int8;
+ * VI-D, are convolutions, the first of every ResNet stage with stride 2; Algorithm 1, forward and backward pass),
+ * computed straight from the NHWC index tensors: the patch matrix whose rows cdl_qlinear_* takes as A_idx is never
+ * written to memory, its tiles are gathered by the loads of the kernel, with zero (= index 0 = level 0) outside the
+ * image.
+ * Cross-correlation with filter R x S (1 <= R, S <= 7), stride 1..4 (the same in both directions) and zero padding
+ * pad_h < R, pad_w < S; output P x Q per image, P = (H + 2 pad_h - R) / stride + 1, Q likewise (integer division).
+ * C and C_out multiples of 64 (else CDL_ERR_ARG: form the patch matrix and call cdl_qlinear_*).
+ *   X_idx [dev] N x H x W x C index bytes (signedness from x);  G_idx [dev] N x P x Q x C_out int8;
  *   W_idx [dev] (R*S*C) x C_out int8, row (r*S + s)*C + c, leading dimension ldw (multiple of 16);
  *   all three 16-byte aligned.
- *   forward   ACC[n,p,q,co] = sum_{r,s,c} X_idx[n, p-(R-1)/2+r, q-(S-1)/2+s, c] * W_idx[(r*S+s)*C+c, co]
- *             Y = (float)ACC * (x->q * w->q) + bias[co]            acc_out, y_out: N x H x W x C_out, nullable
- *   backward  dXACC[n,h,w,c] = sum_{r,s,co} G_idx[n, h+(R-1)/2-r, w+(S-1)/2-s, co] * W_idx[(r*S+s)*C+c, co]
+ *   forward   ACC[n,p,q,co] = sum_{r,s,c} X_idx[n, p*stride-pad_h+r, q*stride-pad_w+s, c] * W_idx[(r*S+s)*C+c, co]
+ *             Y = (float)ACC * (x->q * w->q) + bias[co]            acc_out, y_out: N x P x Q x C_out, nullable
+ *   backward  dXACC[n,h,w,c] = sum of G_idx[n,p,q,co] * W_idx[(r*S+s)*C+c, co] over co and the (r,s,p,q) with
+ *             p*stride-pad_h+r = h, q*stride-pad_w+s = w (the adjoint of the forward map in X)
  *             dX = (float)dXACC * (g->q * w->q)                     dXacc, dX: N x H x W x C, nullable
- *             dWACC[(r*S+s)*C+c, co] = sum_{n,p,q} X_idx[n, p-(R-1)/2+r, q-(S-1)/2+s, c] * G_idx[n,p,q,co]
+ *             dWACC[(r*S+s)*C+c, co] = sum_{n,p,q} X_idx[n, p*stride-pad_h+r, q*stride-pad_w+s, c] * G_idx[n,p,q,co]
  *             dW = (float)dWACC * (g->q * x->q)                     dWacc, dW: (R*S*C) x C_out (ld C_out), nullable
  *   X_idx may be NULL when no dW output is wanted, W_idx when no dX output is.
  *   ws [dev]: cdl_qconv_workspace_bytes(shape, C_out) bytes, 256-byte aligned.
- * Overflow rule and the int64 summation of long reductions as for cdl_qlinear_*.
+ * Overflow rule and the int64 summation of long reductions as for cdl_qlinear_* (with a stride above 1 the data
+ * gradient is one product per residue class of pixels and has no such long-reduction path: CDL_ERR_OVERFLOW_RISK).
  */
 typedef struct {
     int32_t N, H, W, C;   /* the layer's input tensor */
     int32_t R, S;         /* filter height and width */
+    int32_t stride;       /* 1..4; 0 means 1 */
+    int32_t pad_h, pad_w; /* zero padding on each side; a negative value means (R-1)/2 resp. (S-1)/2 */
 } cdl_conv_shape;
 
 int cdl_qconv_fwd(const void *X_idx, const cdl_index_desc *x, const void *W_idx, int64_t ldw, const cdl_index_desc *w,

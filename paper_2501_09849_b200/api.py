@@ -282,17 +282,31 @@ def cdl_qlinear_bwd(G_idx, ldg, g: IndexDesc, A_idx, lda, a, W_idx, ldw, w, M, N
 
 
 class _ConvShapeC(C.Structure):
-    _fields_ = [("N", C.c_int32), ("H", C.c_int32), ("W", C.c_int32), ("C", C.c_int32), ("R", C.c_int32), ("S", C.c_int32)]
+    _fields_ = [("N", C.c_int32), ("H", C.c_int32), ("W", C.c_int32), ("C", C.c_int32), ("R", C.c_int32), ("S", C.c_int32),
+                ("stride", C.c_int32), ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
 
 
 class ConvShape:
-    """cdl_conv_shape: input tensor N x H x W x C, filter R x S (stride 1, padding (R-1)/2, (S-1)/2)."""
+    """cdl_conv_shape: input tensor N x H x W x C, filter R x S, stride, zero padding (default (R-1)/2, (S-1)/2)."""
 
-    def __init__(self, N, H, W, C, R, S):
+    def __init__(self, N, H, W, C, R, S, stride=1, pad_h=None, pad_w=None):
         self.N, self.H, self.W, self.C, self.R, self.S = int(N), int(H), int(W), int(C), int(R), int(S)
+        self.stride = int(stride)
+        self.pad_h = (self.R - 1) // 2 if pad_h is None else int(pad_h)
+        self.pad_w = (self.S - 1) // 2 if pad_w is None else int(pad_w)
+
+    @property
+    def P(self):
+        """output rows per image"""
+        return (self.H + 2 * self.pad_h - self.R) // self.stride + 1
+
+    @property
+    def Q(self):
+        """output columns per image"""
+        return (self.W + 2 * self.pad_w - self.S) // self.stride + 1
 
     def _c(self):
-        return _ConvShapeC(self.N, self.H, self.W, self.C, self.R, self.S)
+        return _ConvShapeC(self.N, self.H, self.W, self.C, self.R, self.S, self.stride, self.pad_h, self.pad_w)
 
 
 def cdl_qconv_workspace_bytes(shape: ConvShape, C_out):

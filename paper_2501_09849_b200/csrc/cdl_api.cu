@@ -414,29 +414,125 @@ int cdl_qlinear_bwd(const void *G_idx, int64_t ldg, const cdl_index_desc *g, con
 }
 
 namespace {
-// pixels, taps and patch length of a supported convolution shape; false when the shape is not supported
-bool conv_dims(const cdl_conv_shape *s, int32_t C_out, int64_t *M, int *taps)
+// Geometry of a supported convolution shape: output grid, pixel counts, taps.
+struct ConvGeo {
+    int stride, pad_h, pad_w;
+    int P, Q;               // output pixels per image column / row
+    int64_t M_out, M_in;    // N * P * Q, N * H * W
+    int taps;
+};
+
+// false when the shape is not supported
+bool conv_geo(const cdl_conv_shape *s, int32_t C_out, ConvGeo *g)
 {
     if (s == nullptr || s->N <= 0 || s->H <= 0 || s->W <= 0 || s->C <= 0 || C_out <= 0) return false;
-    if (s->R <= 0 || s->S <= 0 || (s->R & 1) == 0 || (s->S & 1) == 0 || s->R > 127 || s->S > 127) return false;
+    if (s->R <= 0 || s->S <= 0 || s->R > 7 || s->S > 7) return false;
     if ((s->C % 64) != 0 || (C_out % 64) != 0) return false;
-    *M = (int64_t)s->N * s->H * s->W;
-    *taps = s->R * s->S;
-    if (*M > 0x7fffff00ll || (int64_t)*taps * (s->C + 64) > 0x7fffff00ll || (int64_t)*taps * (C_out + 64) > 0x7fffff00ll) return false;
+    g->stride = s->stride == 0 ? 1 : s->stride;                   // 0 and a negative padding: the defaults
+    g->pad_h = s->pad_h < 0 ? (s->R - 1) / 2 : s->pad_h;
+    g->pad_w = s->pad_w < 0 ? (s->S - 1) / 2 : s->pad_w;
+    if (g->stride < 1 || g->stride > 4 || g->pad_h >= s->R || g->pad_w >= s->S) return false;
+    if (s->H + 2 * g->pad_h < s->R || s->W + 2 * g->pad_w < s->S) return false;
+    g->P = (s->H + 2 * g->pad_h - s->R) / g->stride + 1;
+    g->Q = (s->W + 2 * g->pad_w - s->S) / g->stride + 1;
+    g->M_out = (int64_t)s->N * g->P * g->Q;
+    g->M_in = (int64_t)s->N * s->H * s->W;
+    g->taps = s->R * s->S;
+    if (g->M_out > 0x7fffff00ll || g->M_in > 0x7fffff00ll || (int64_t)g->taps * (s->C + 64) > 0x7fffff00ll ||
+        (int64_t)g->taps * (C_out + 64) > 0x7fffff00ll)
+        return false;
     return true;
+}
+
+// the patch matrix of the layer's input: rows = output pixels, taps in filter order
+cdl::ConvGather input_gather(const cdl_conv_shape *s, const ConvGeo &g, int transposed)
+{
+    cdl::ConvGather cg;
+    memset(&cg, 0, sizeof cg);
+    cg.N = s->N;
+    cg.H = s->H;
+    cg.W = s->W;
+    cg.C = s->C;
+    cg.P = g.P;
+    cg.Q = g.Q;
+    cg.lower_h = -g.pad_h;
+    cg.lower_w = -g.pad_w;
+    cg.stride = g.stride;
+    cg.taps = g.taps;
+    for (int t = 0; t < g.taps; ++t) {
+        cg.oh[t] = (signed char)(t / s->S);
+        cg.ow[t] = (signed char)(t % s->S);
+    }
+    cg.transposed = transposed;
+    return cg;
+}
+
+// The patch matrix of the gradient tensor [N,P,Q,C_out] for the data gradient of the input pixels h = st i + a,
+// w = st j + b (st = the layer's stride; st = 1: all pixels, a = b = 0): only the filter taps r = a + pad_h (mod st),
+// s = b + pad_w (mod st) reach such a pixel, tap r from gradient row i + (a + pad_h - r) / st.  Returns the number of
+// taps (0: these pixels receive nothing).
+int gradient_gather(const cdl_conv_shape *s, const ConvGeo &g, int32_t C_out, int a, int b, cdl::ConvGather *out)
+{
+    cdl::ConvGather cg;
+    memset(&cg, 0, sizeof cg);
+    const int st = g.stride;
+    int rs[8], dr[8], nr = 0, ss[8], ds[8], ns = 0;
+    for (int r = 0; r < s->R; ++r)
+        if ((a + g.pad_h - r) % st == 0) {
+            rs[nr] = r;
+            dr[nr++] = (a + g.pad_h - r) / st;
+        }
+    for (int c = 0; c < s->S; ++c)
+        if ((b + g.pad_w - c) % st == 0) {
+            ss[ns] = c;
+            ds[ns++] = (b + g.pad_w - c) / st;
+        }
+    if (nr == 0 || ns == 0) return 0;
+    int dmin_h = dr[0], dmin_w = ds[0];
+    for (int i = 1; i < nr; ++i) dmin_h = dr[i] < dmin_h ? dr[i] : dmin_h;
+    for (int i = 1; i < ns; ++i) dmin_w = ds[i] < dmin_w ? ds[i] : dmin_w;
+    cg.N = s->N;
+    cg.H = g.P;
+    cg.W = g.Q;
+    cg.C = C_out;
+    cg.P = (s->H - a + st - 1) / st;          // pixels h = st i + a < H
+    cg.Q = (s->W - b + st - 1) / st;
+    cg.lower_h = dmin_h;
+    cg.lower_w = dmin_w;
+    cg.stride = 1;
+    cg.taps = nr * ns;
+    for (int i = 0; i < nr; ++i)
+        for (int j = 0; j < ns; ++j) {
+            const int t = i * ns + j;
+            cg.oh[t] = (signed char)(dr[i] - dmin_h);
+            cg.ow[t] = (signed char)(ds[j] - dmin_w);
+            cg.ytap[t] = (unsigned char)(rs[i] * s->S + ss[j]);
+        }
+    cg.transposed = 0;
+    cg.y_tap_rows = s->C;
+    cg.y_rows = g.taps * s->C;
+    if (st > 1) {
+        cg.sc_on = 1;
+        cg.sc_H = s->H;
+        cg.sc_W = s->W;
+        cg.sc_s = st;
+        cg.sc_a = a;
+        cg.sc_b = b;
+    }
+    *out = cg;
+    return cg.taps;
 }
 }  // namespace
 
 size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
 {
-    int64_t M;
-    int taps;
-    if (!conv_dims(shape, C_out, &M, &taps)) return 0;
+    ConvGeo g;
+    if (!conv_geo(shape, C_out, &g)) return 0;
     // the tiling pads every tap to whole 128-channel blocks
     const int cp = (shape->C + 127) / 128 * 128, cop = (C_out + 127) / 128 * 128;
-    const size_t f = tc_gemm_scratch_bytes((int)M, C_out, taps * cp);
-    const size_t dx = tc_gemm_scratch_bytes((int)M, shape->C, taps * cop);
-    const size_t dw = tc_gemm_scratch_bytes(taps * cp, C_out, (int)M);
+    const size_t f = tc_gemm_scratch_bytes((int)g.M_out, C_out, g.taps * cp);
+    const size_t dx = g.stride == 1 ? tc_gemm_scratch_bytes((int)g.M_in, shape->C, g.taps * cop) : 0;   // (strided: no split)
+    const size_t dw = tc_gemm_scratch_bytes(g.taps * cp, C_out, (int)g.M_out);
     size_t m = f > dx ? f : dx;
     if (dw > m) m = dw;
     return kStatusBytes + m;
@@ -447,9 +543,8 @@ int cdl_qconv_fwd_next(const void *X_idx, const cdl_index_desc *x, const void *W
                        const float *bias, const cdl_index_desc *next, void *idx_next, void *ws, size_t ws_bytes,
                        void *stream)
 {
-    int64_t M;
-    int taps;
-    if (X_idx == nullptr || W_idx == nullptr || !conv_dims(shape, C_out, &M, &taps)) return CDL_ERR_ARG;
+    ConvGeo geo;
+    if (X_idx == nullptr || W_idx == nullptr || !conv_geo(shape, C_out, &geo)) return CDL_ERR_ARG;
     if (acc_out == nullptr && y_out == nullptr && idx_next == nullptr) return CDL_ERR_ARG;
     NextQuant nq;
     {
@@ -466,14 +561,14 @@ int cdl_qconv_fwd_next(const void *X_idx, const cdl_index_desc *x, const void *W
     if (bad_f32_ptr(acc_out) || bad_f32_ptr(y_out) || bad_f32_ptr(bias)) return CDL_ERR_ALIGN;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_workspace_bytes(shape, C_out))
         return CDL_ERR_WORKSPACE;
-    const int K = taps * shape->C;
+    const int K = geo.taps * shape->C;
     if (acc_out != nullptr && overflow_risk(K, rx, rw)) return CDL_ERR_OVERFLOW_RISK;
     if ((rc = check_device()) != CDL_OK) return rc;
     // Y[pixel, co] = sum_{tap, c} patch(pixel; tap, c) * W[tap * C + c, co]
-    ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 0, 0};
+    const ConvGather cg = input_gather(shape, geo, 0);
     GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
     GemmOperand Y{W_idx, 1, ldw, false, (int)rw.absmax};
-    return launch_index_gemm_tc(X, Y, (int)M, C_out, K, acc_out, y_out, (x->q * w->q), bias,
+    return launch_index_gemm_tc(X, Y, (int)geo.M_out, C_out, K, acc_out, y_out, (x->q * w->q), bias,
                                 static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws),
                                 static_cast<cudaStream_t>(stream), &cg, &nq);
 }
@@ -491,13 +586,13 @@ namespace {
 // entry point returns before anything is enqueued.
 int check_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx, const cdl_index_desc *x,
                     const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
-                    const int32_t *dXacc, const float *dX, const int32_t *dWacc, const float *dW, int64_t *M_out,
-                    int *taps_out, cdl::IndexRange *rg, cdl::IndexRange *rx, cdl::IndexRange *rw)
+                    const int32_t *dXacc, const float *dX, const int32_t *dWacc, const float *dW, ConvGeo *geo,
+                    cdl::IndexRange *rg, cdl::IndexRange *rx, cdl::IndexRange *rw)
 {
     using namespace cdl;
     const bool want_dx = dXacc != nullptr || dX != nullptr;
     const bool want_dw = dWacc != nullptr || dW != nullptr;
-    if (G_idx == nullptr || !conv_dims(shape, C_out, M_out, taps_out)) return CDL_ERR_ARG;
+    if (G_idx == nullptr || !conv_geo(shape, C_out, geo)) return CDL_ERR_ARG;
     if (!want_dx && !want_dw) return CDL_ERR_ARG;
     if ((want_dx && W_idx == nullptr) || (want_dw && X_idx == nullptr)) return CDL_ERR_ARG;
     if (want_dx && ldw < C_out) return CDL_ERR_ARG;
@@ -513,8 +608,69 @@ int check_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_id
     if (want_dw && (reinterpret_cast<uintptr_t>(X_idx) & 15u)) return CDL_ERR_ALIGN;
     if (want_dx && ((ldw & 15) || (reinterpret_cast<uintptr_t>(W_idx) & 15u))) return CDL_ERR_ALIGN;
     if (bad_f32_ptr(dXacc) || bad_f32_ptr(dX) || bad_f32_ptr(dWacc) || bad_f32_ptr(dW)) return CDL_ERR_ALIGN;
-    if (dXacc != nullptr && overflow_risk((int64_t)*taps_out * C_out, *rg, *rw)) return CDL_ERR_OVERFLOW_RISK;
-    if (dWacc != nullptr && overflow_risk(*M_out, *rx, *rg)) return CDL_ERR_OVERFLOW_RISK;
+    if (dXacc != nullptr && overflow_risk((int64_t)geo->taps * C_out, *rg, *rw)) return CDL_ERR_OVERFLOW_RISK;
+    if (dWacc != nullptr && overflow_risk(geo->M_out, *rx, *rg)) return CDL_ERR_OVERFLOW_RISK;
+    return CDL_OK;
+}
+
+// The two backward products of a convolutional layer for one gradient index tensor (already validated arguments).
+// accumulate: the float outputs are added to (second digit plane of a real-valued gradient).
+int run_qconv_bwd(const void *G_idx, float q_g, const cdl::IndexRange &rg, const void *X_idx, const cdl_index_desc *x,
+                  const cdl::IndexRange &rx, const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl::IndexRange &rw,
+                  const cdl_conv_shape *shape, const ConvGeo &geo, int32_t C_out, int32_t *dXacc, float *dX, int32_t *dWacc,
+                  float *dW, bool accumulate, void *ws, cudaStream_t st)
+{
+    using namespace cdl;
+    char *scratch = static_cast<char *>(ws) + kStatusBytes;
+    int *status = static_cast<int *>(ws);
+    int rc;
+    if (dXacc != nullptr || dX != nullptr) {
+        // dX[pixel, c] = sum over the filter taps that reach the pixel and over co of G[..] * W[tap * C + c, co]: the
+        // patches of the gradient tensor against the filter taps.  With a stride st > 1 the input pixels fall into
+        // st x st residue classes (h mod st, w mod st), each reached by its own subset of taps: one product per class,
+        // its rows written to the pixels of the class; a class no tap reaches receives zeros.
+        GemmOperand X{G_idx, 0, 0, false, (int)rg.absmax};
+        GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
+        const int st_ = geo.stride;
+        bool cleared = false;
+        for (int a = 0; a < st_; ++a)
+            for (int b = 0; b < st_; ++b) {
+                ConvGather cg;
+                const int ntaps = gradient_gather(shape, geo, C_out, a, b, &cg);
+                if (ntaps == 0) {
+                    if (!cleared && !accumulate) {       // (cleared before any class is written: the stream keeps the order)
+                        const size_t n = (size_t)geo.M_in * shape->C;
+                        if ((dX != nullptr && cudaMemsetAsync(dX, 0, n * sizeof(float), st) != cudaSuccess) ||
+                            (dXacc != nullptr && cudaMemsetAsync(dXacc, 0, n * sizeof(int32_t), st) != cudaSuccess)) {
+                            (void)cudaGetLastError();
+                            return CDL_ERR_LAUNCH;
+                        }
+                        cleared = true;
+                    }
+                    continue;
+                }
+                (void)ntaps;
+            }
+        for (int a = 0; a < st_; ++a)
+            for (int b = 0; b < st_; ++b) {
+                ConvGather cg;
+                const int ntaps = gradient_gather(shape, geo, C_out, a, b, &cg);
+                if (ntaps == 0 || cg.P <= 0 || cg.Q <= 0) continue;
+                const long long rows = (long long)shape->N * cg.P * cg.Q;
+                rc = launch_index_gemm_tc(X, Y, (int)rows, shape->C, ntaps * C_out, dXacc, dX, (q_g * w->q), nullptr, scratch,
+                                          status, st, &cg, nullptr, accumulate);
+                if (rc != CDL_OK) return rc;
+            }
+    }
+    if (dWacc != nullptr || dW != nullptr) {
+        // dW[tap * C + c, co] = sum_pixel patch(pixel; tap, c) * G[pixel, co]
+        const ConvGather cg = input_gather(shape, geo, 1);
+        GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
+        GemmOperand Y{G_idx, 1, C_out, false, (int)rg.absmax};
+        rc = launch_index_gemm_tc(X, Y, geo.taps * shape->C, C_out, (int)geo.M_out, dWacc, dW, (q_g * x->q), nullptr, scratch,
+                                  status, st, &cg, nullptr, accumulate);
+        if (rc != CDL_OK) return rc;
+    }
     return CDL_OK;
 }
 }  // namespace
@@ -523,37 +679,15 @@ int cdl_qconv_bwd(const void *G_idx, const cdl_index_desc *g, const void *X_idx,
                   const void *W_idx, int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out,
                   int32_t *dXacc, float *dX, int32_t *dWacc, float *dW, void *ws, size_t ws_bytes, void *stream)
 {
-    const bool want_dx = dXacc != nullptr || dX != nullptr;
-    const bool want_dw = dWacc != nullptr || dW != nullptr;
-    int64_t M;
-    int taps;
+    ConvGeo geo;
     IndexRange rg, rx{false, 0}, rw{false, 0};
-    int rc = check_qconv_bwd(G_idx, g, X_idx, x, W_idx, ldw, w, shape, C_out, dXacc, dX, dWacc, dW, &M, &taps, &rg, &rx, &rw);
+    int rc = check_qconv_bwd(G_idx, g, X_idx, x, W_idx, ldw, w, shape, C_out, dXacc, dX, dWacc, dW, &geo, &rg, &rx, &rw);
     if (rc != CDL_OK) return rc;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_workspace_bytes(shape, C_out))
         return CDL_ERR_WORKSPACE;
     if ((rc = check_device()) != CDL_OK) return rc;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (want_dx) {
-        // dX[pixel, c] = sum_{tap', co} patchG(pixel; tap', co) * W[(taps-1-tap') * C + c, co]: the patches of the
-        // gradient tensor (same padding) against the filter taps in mirrored order
-        ConvGather cg{shape->N, shape->H, shape->W, C_out, shape->R, shape->S, 0, shape->C};
-        GemmOperand X{G_idx, 0, 0, false, (int)rg.absmax};
-        GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
-        rc = launch_index_gemm_tc(X, Y, (int)M, shape->C, taps * C_out, dXacc, dX, (g->q * w->q), nullptr,
-                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg);
-        if (rc != CDL_OK) return rc;
-    }
-    if (want_dw) {
-        // dW[tap * C + c, co] = sum_pixel patch(pixel; tap, c) * G[pixel, co]
-        ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 1, 0};
-        GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
-        GemmOperand Y{G_idx, 1, C_out, false, (int)rg.absmax};
-        rc = launch_index_gemm_tc(X, Y, taps * shape->C, C_out, (int)M, dWacc, dW, (g->q * x->q), nullptr,
-                                  static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg);
-        if (rc != CDL_OK) return rc;
-    }
-    return CDL_OK;
+    return run_qconv_bwd(G_idx, g->q, rg, X_idx, x, rx, W_idx, ldw, w, rw, shape, geo, C_out, dXacc, dX, dWacc, dW, false, ws,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int cdl_rescale_acc(const void *acc, int32_t acc_bits, int64_t n, float q_x, float q_y, float *out, void *stream)
@@ -653,70 +787,40 @@ int cdl_qlinear_bwd_fp(const float *G, float g_absmax, const void *A_idx, int64_
 size_t cdl_qconv_bwd_fp_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
 {
     const size_t base = cdl_qconv_workspace_bytes(shape, C_out);
-    if (base == 0) return 0;
-    const size_t pixels = (size_t)shape->N * shape->H * shape->W;
-    return align256(base) + 2 * align256(pixels * (size_t)C_out);
+    ConvGeo geo;
+    if (base == 0 || !conv_geo(shape, C_out, &geo)) return 0;
+    return align256(base) + 2 * align256((size_t)geo.M_out * (size_t)C_out);
 }
 
 int cdl_qconv_bwd_fp(const float *G, float g_absmax, const void *X_idx, const cdl_index_desc *x, const void *W_idx,
                      int64_t ldw, const cdl_index_desc *w, const cdl_conv_shape *shape, int32_t C_out, float *dX, float *dW,
                      void *ws, size_t ws_bytes, void *stream)
 {
-    int64_t M;
-    int taps;
-    if (G == nullptr || !conv_dims(shape, C_out, &M, &taps) || (dX == nullptr && dW == nullptr)) return CDL_ERR_ARG;
+    ConvGeo geo;
+    if (G == nullptr || !conv_geo(shape, C_out, &geo) || (dX == nullptr && dW == nullptr)) return CDL_ERR_ARG;
     if (!(g_absmax > 0.0f) || !(g_absmax < 1e30f)) return CDL_ERR_RANGE;
     if (bad_f32_ptr(G)) return CDL_ERR_ALIGN;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < cdl_qconv_bwd_fp_workspace_bytes(shape, C_out))
         return CDL_ERR_WORKSPACE;
     const float q1 = g_absmax / 127.0f, q2 = q1 / 254.0f;
+    if (!(q1 > 0.0f) || !(q2 > 0.0f)) return CDL_ERR_RANGE;
     const size_t base = align256(cdl_qconv_workspace_bytes(shape, C_out));
-    const size_t plane = align256((size_t)M * (size_t)C_out);
+    const size_t plane = align256((size_t)geo.M_out * (size_t)C_out);
     char *d1 = static_cast<char *>(ws) + base, *d2 = d1 + plane;
     // every argument is checked before the first operation is enqueued (the digit planes stand in for G_idx)
-    int rc;
-    {
-        const cdl_index_desc gd{q1, -127, 127};
-        IndexRange cg_, cx_{false, 0}, cw_{false, 0};
-        int64_t M2;
-        int taps2;
-        if (!(q1 > 0.0f) || !(q2 > 0.0f)) return CDL_ERR_RANGE;
-        rc = check_qconv_bwd(d1, &gd, X_idx, x, W_idx, ldw, w, shape, C_out, nullptr, dX, nullptr, dW, &M2, &taps2, &cg_, &cx_, &cw_);
-        if (rc != CDL_OK) return rc;
-    }
+    const cdl_index_desc gd{q1, -127, 127};
+    IndexRange rg, rx{false, 0}, rw{false, 0};
+    int rc = check_qconv_bwd(d1, &gd, X_idx, x, W_idx, ldw, w, shape, C_out, nullptr, dX, nullptr, dW, &geo, &rg, &rx, &rw);
+    if (rc != CDL_OK) return rc;
     if ((rc = check_device()) != CDL_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((rc = launch_gradient_digits(G, M, C_out, C_out, q1, q2, d1, d2, st)) != CDL_OK) return rc;
+    if ((rc = launch_gradient_digits(G, geo.M_out, C_out, C_out, q1, q2, d1, d2, st)) != CDL_OK) return rc;
     // each digit plane is a gradient index tensor of its own step: the first pass stores, the second adds.  The
-    // products share the front of the workspace (status word, split slabs); calls on one stream run in order.
+    // products share the front of the workspace (status block, split slabs); calls on one stream run in order.
     for (int pass = 0; pass < 2; ++pass) {
-        const cdl_index_desc gd{pass == 0 ? q1 : q2, -127, 127};
-        const char *dig = pass == 0 ? d1 : d2;
-        if (pass == 0) {
-            rc = cdl_qconv_bwd(dig, &gd, X_idx, x, W_idx, ldw, w, shape, C_out, nullptr, dX, nullptr, dW, ws, base, stream);
-            if (rc != CDL_OK) return rc;
-            continue;
-        }
-        // second digit: same validation already passed; accumulate into the outputs of the first
-        IndexRange rg{false, 127}, rx{false, 0}, rw{false, 0};
-        if (dW != nullptr && (rc = index_range(x, &rx)) != CDL_OK) return rc;
-        if (dX != nullptr && (rc = index_range(w, &rw)) != CDL_OK) return rc;
-        if (dX != nullptr) {
-            ConvGather cg{shape->N, shape->H, shape->W, C_out, shape->R, shape->S, 0, shape->C};
-            GemmOperand X{dig, 0, 0, false, (int)rg.absmax};
-            GemmOperand Y{W_idx, ldw, 1, false, (int)rw.absmax};
-            rc = launch_index_gemm_tc(X, Y, (int)M, shape->C, taps * C_out, nullptr, dX, (gd.q * w->q), nullptr,
-                                      static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg, nullptr, true);
-            if (rc != CDL_OK) return rc;
-        }
-        if (dW != nullptr) {
-            ConvGather cg{shape->N, shape->H, shape->W, shape->C, shape->R, shape->S, 1, 0};
-            GemmOperand X{X_idx, 0, 0, rx.is_unsigned, (int)rx.absmax};
-            GemmOperand Y{dig, 1, C_out, false, (int)rg.absmax};
-            rc = launch_index_gemm_tc(X, Y, taps * shape->C, C_out, (int)M, nullptr, dW, (gd.q * x->q), nullptr,
-                                      static_cast<char *>(ws) + kStatusBytes, static_cast<int *>(ws), st, &cg, nullptr, true);
-            if (rc != CDL_OK) return rc;
-        }
+        rc = run_qconv_bwd(pass == 0 ? d1 : d2, pass == 0 ? q1 : q2, rg, X_idx, x, rx, W_idx, ldw, w, rw, shape, geo, C_out,
+                           nullptr, dX, nullptr, dW, pass == 1, ws, st);
+        if (rc != CDL_OK) return rc;
     }
     return CDL_OK;
 }

@@ -33,6 +33,7 @@
 #include <cuda.h>
 
 #include <atomic>
+#include <string.h>
 
 #include "cdl_internal.h"
 #include "cdl_wait.cuh"
@@ -62,6 +63,7 @@ constexpr int kOutWarpBytes = 32 * 128;  // epilogue staging block of one warp: 
 // The whole 227 KB opt-in window is requested (stages need 193 KB): operand descriptors then address
 // allocated shared memory for any stride a 128 x 256 x 128 tile can produce.
 constexpr int kSmemBytes = 232448 - 1024;
+constexpr int kMaxTaps = kConvMaxTaps;   // filter taps of a gathered patch matrix (7 x 7 fits)
 constexpr int kPlanSMs = 148;           // B200: splits are planned for this count so that workspace sizes are fixed
 constexpr unsigned long long kWaitNs = 2000000000ull;  // limit of every device-side wait: 2 s
 
@@ -85,12 +87,20 @@ struct TcParams {
     // Implicit patch matrix (convolution): the X operand is gathered by TMA im2col loads from an [N,H,W,C] index
     // tensor instead of being read from a stored matrix.
     int conv;               // 0: stored matrix; 1: X(i = pixel, r = tap * C + c); 2: X(i = tap * C + c, r = pixel)
-    int cH, cW, cC, cS;     // image height and width, channels, filter width
+    int cH, cW, cC;         // base pixels per image column and row (the gather's output grid), channels
     int cblocks;            // 128-channel blocks per tap (C rounded up to 128: channels past C read as zero)
     int cpad;               // 128 * cblocks
-    int pad_h, pad_w;
-    int taps;               // R * S
-    int y_tap_rows;         // > 0: the Y block of tap t starts at row (taps - 1 - t) * y_tap_rows of the stored matrix
+    int pad_h, pad_w;       // the base pixel of grid position (p, q) sits at (p * c_stride - pad_h, q * c_stride - pad_w)
+    int c_stride;
+    int taps;
+    int y_tap_rows;         // > 0: the Y block of tap t starts at row tap_y[t] * y_tap_rows of the stored matrix
+    signed char tap_oh[kMaxTaps], tap_ow[kMaxTaps];   // offset of each tap from the base pixel
+    unsigned char tap_y[kMaxTaps];
+    // Scattered output rows (data gradient of a strided convolution, one residue class of pixels per launch): row i
+    // of the product is position (n, p, q) of an sc_P x sc_Q grid per image and is stored as pixel
+    // (n, sc_s p + sc_a, sc_s q + sc_b) of an sc_H x sc_W image.
+    int sc_on, sc_P, sc_Q, sc_H, sc_W, sc_s, sc_a, sc_b;
+    int copy_vec;           // outputs copied out by the warps may be written 16 bytes at a time (J % 4 == 0, aligned bases)
     // next layer's hard index from the float output (forward products, single split)
     unsigned char *nq_out;  // nullptr: not requested
     float nq_q, nq_rq, nq_flo, nq_fhi;
@@ -434,8 +444,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const int rem = pix - g_n * (P.cH * P.cW);
                     g_h = rem / P.cW;
                     g_w = rem % P.cW;
-                    g_oh = g_tap / P.cS;
-                    g_ow = g_tap % P.cS;
+                    g_oh = P.tap_oh[g_tap];
+                    g_ow = P.tap_ow[g_tap];
                 }
                 const int pix_dh = BR / (P.cW > 0 ? P.cW : 1), pix_dw = BR % (P.cW > 0 ? P.cW : 1);   // 128 pixels further on
                 for (int rb = rb0; rb < rb1; ++rb, ++it) {
@@ -448,19 +458,17 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
                     const uint32_t sb = sa + kABytes;
                     int b_row = tj * P.TN + brow;
-                    if (P.y_tap_rows > 0) b_row += (P.taps - 1 - g_tap) * P.y_tap_rows;
+                    if (P.y_tap_rows > 0) b_row += (int)P.tap_y[g_tap] * P.y_tap_rows;
                     // Y coordinate along r: the stored matrix has C (not the padded count) rows per tap
                     const int b_red = P.y_tap_rows > 0 ? g_cb * BR : (P.conv == 1 ? g_tap * P.cC + g_cb * BR : rb * BR);
                     const int g_c = P.conv == 1 ? g_cb * BR : g_c0;
-                    const int c_w = g_w - P.pad_w, c_h = g_h - P.pad_h, c_n = g_n, c_ow = g_ow, c_oh = g_oh;
+                    const int c_w = g_w * P.c_stride - P.pad_w, c_h = g_h * P.c_stride - P.pad_h, c_n = g_n, c_ow = g_ow, c_oh = g_oh;
                     if (P.conv == 1) {            // next stage: next channel block, then next tap
                         if (++g_cb == P.cblocks) {
                             g_cb = 0;
-                            ++g_tap;
-                            if (++g_ow == P.cS) {
-                                g_ow = 0;
-                                ++g_oh;
-                            }
+                            g_tap = g_tap + 1 < P.taps ? g_tap + 1 : g_tap;      // (past the last tap nothing more is loaded)
+                            g_oh = P.tap_oh[g_tap];
+                            g_ow = P.tap_ow[g_tap];
                         }
                     } else if (P.conv == 2) {     // next stage: 128 pixels further on
                         g_w += pix_dw;
@@ -599,13 +607,33 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         };
         // Same staging, then the warp copies its 32 rows out itself, one row (up to 128 contiguous bytes) per
         // instruction: for outputs TMA cannot take (row pitch or base not a multiple of 16 bytes, 16-column tiles).
+        int my_orow = 0;            // scattered output: where this thread's row of the current tile goes
         auto stage_and_copy = [&](const uint32_t (&w)[32], int32_t *out, bool reduce, long long row_off, int row0,
                                   int col0, int ncol, bool as_float = false) {
             const uint32_t blk = stage(w);
             __syncwarp();
+            if (!reduce && ncol == 32 && P.copy_vec) {
+                // whole 32-column chunk, 16-byte aligned rows: eight lanes write the 128 bytes of one row, four rows
+                // per instruction
+                const int c4 = lane & 7;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int rr = it * 4 + (lane >> 3);
+                    int grow = row0 + rr;
+                    const bool live = grow < P.I_out;
+                    if (P.sc_on) grow = __shfl_sync(0xffffffffu, my_orow, rr);
+                    uint4 val;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                 : "r"(blk + (uint32_t)rr * 128u + (uint32_t)((c4 ^ (rr & 7)) << 4)));
+                    if (live) *reinterpret_cast<uint4 *>(out + (row_off + grow) * P.J + col0 + 4 * c4) = val;
+                }
+                __syncwarp();
+                return;
+            }
             for (int rr = 0; rr < 32; ++rr) {
-                const int grow = row0 + rr;
+                int grow = row0 + rr;
                 if (grow >= P.I_out) break;                                // uniform over the warp
+                if (P.sc_on) grow = __shfl_sync(0xffffffffu, my_orow, rr);
                 uint32_t val;
                 asm volatile("ld.shared.b32 %0, [%1];" : "=r"(val)
                              : "r"(blk + (uint32_t)rr * 128u + (uint32_t)(((lane >> 2) ^ (rr & 7)) << 4) + (uint32_t)((lane & 3) << 2)));
@@ -640,6 +668,11 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             if (P.conv == 2 && P.cpad != P.cC) {
                 const int tap = wrow0 / P.cpad, c = wrow0 - tap * P.cpad;
                 wrow0 = c < P.cC ? tap * P.cC + c : 0x7fffff00;
+            }
+            if (P.sc_on) {
+                const int grow = wrow0 + lane, per = P.sc_P * P.sc_Q;
+                const int n = grow / per, rem = grow - n * per, pi = rem / P.sc_Q, qj = rem - pi * P.sc_Q;
+                my_orow = (n * P.sc_H + P.sc_s * pi + P.sc_a) * P.sc_W + P.sc_s * qj + P.sc_b;
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
             const int tile_cols = min(P.TN, P.J - tj * P.TN);
@@ -830,8 +863,9 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
                                    const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                    CUtensorMapFloatOOBfill);
 
-// [N,H,W,C] byte tensor read in im2col mode: one load fetches 128 consecutive base pixels x 128 channel bytes,
-// the base pixels running over the input shifted by the padding, the filter tap given per load as an offset.
+// [N,H,W,C] byte tensor read in im2col mode: one load fetches 128 consecutive base pixels x 128 channel bytes, the
+// base pixels running over the gather's grid (first at the lower corner, `stride` apart), the filter tap given per
+// load as an offset.
 bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g)
 {
     static EncodeIm2colFn fn = nullptr;
@@ -845,12 +879,12 @@ bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g)
         }
         fn = reinterpret_cast<EncodeIm2colFn>(p);
     }
-    const int pad_h = (g.R - 1) / 2, pad_w = (g.S - 1) / 2;
     const cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
     const cuuint64_t strides[3] = {(cuuint64_t)g.C, (cuuint64_t)g.C * g.W, (cuuint64_t)g.C * g.W * g.H};
-    const int lower[2] = {-pad_w, -pad_h};                          // {w, h}: first base pixel
-    const int upper[2] = {pad_w - (g.S - 1), pad_h - (g.R - 1)};    // last base pixel relative to the far corner
-    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    const int lower[2] = {g.lower_w, g.lower_h};                    // {w, h}: first base pixel
+    // last base pixel, relative to the far corner of the tensor
+    const int upper[2] = {g.lower_w + (g.Q - 1) * g.stride - (g.W - 1), g.lower_h + (g.P - 1) * g.stride - (g.H - 1)};
+    const cuuint32_t estr[4] = {1u, (cuuint32_t)g.stride, (cuuint32_t)g.stride, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, 128u, 128u,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -930,8 +964,8 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     int It = I, Rt = R;
     if (conv != nullptr) {
         const int cpad = (conv->C + BR - 1) / BR * BR;
-        if (conv->transposed) It = conv->R * conv->S * cpad;
-        else Rt = conv->R * conv->S * cpad;
+        if (conv->transposed) It = conv->taps * cpad;
+        else Rt = conv->taps * cpad;
     }
     TcParams P;
     P.I = It;
@@ -946,7 +980,10 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1);
     const bool want_next = next != nullptr && next->idx_out != nullptr;
     if (want_next && wide) return CDL_ERR_OVERFLOW_RISK;     // the index is taken from one finished accumulator
-    const int TN = pl.TN, splits = want_next ? 1 : pl.splits;
+    const int TN = pl.TN;
+    const bool scatter = conv != nullptr && conv->sc_on != 0;
+    if (scatter && wide) return CDL_ERR_OVERFLOW_RISK;       // scattered rows are written by the product's own epilogue
+    const int splits = (want_next || scatter) ? 1 : pl.splits;
     const bool pair = pl.pair != 0;
     P.TN = TN;
     P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
@@ -979,20 +1016,41 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         P.nq_vec = ((J & 15) == 0 && (reinterpret_cast<uintptr_t>(next->idx_out) & 15u) == 0) ? 1 : 0;
     }
     P.conv = 0;
-    P.cH = P.cW = P.cC = P.cS = P.cblocks = P.cpad = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
+    P.cH = P.cW = P.cC = P.cblocks = P.cpad = P.pad_h = P.pad_w = P.taps = P.y_tap_rows = 0;
+    P.c_stride = 1;
+    P.sc_on = P.sc_P = P.sc_Q = P.sc_H = P.sc_W = P.sc_s = P.sc_a = P.sc_b = 0;
+    memset(P.tap_oh, 0, sizeof P.tap_oh);
+    memset(P.tap_ow, 0, sizeof P.tap_ow);
+    memset(P.tap_y, 0, sizeof P.tap_y);
     if (conv != nullptr) {
-        if (conv->C % 64 != 0 || (conv->R & 1) == 0 || (conv->S & 1) == 0) return CDL_ERR_ARG;
+        if (conv->C % 64 != 0 || conv->taps < 1 || conv->taps > kMaxTaps || conv->stride < 1) return CDL_ERR_ARG;
         P.conv = conv->transposed ? 2 : 1;
-        P.cH = conv->H;
-        P.cW = conv->W;
+        P.cH = conv->P;
+        P.cW = conv->Q;
         P.cC = conv->C;
-        P.cS = conv->S;
         P.cblocks = (conv->C + BR - 1) / BR;
         P.cpad = P.cblocks * BR;
-        P.pad_h = (conv->R - 1) / 2;
-        P.pad_w = (conv->S - 1) / 2;
-        P.taps = conv->R * conv->S;
+        P.pad_h = -conv->lower_h;
+        P.pad_w = -conv->lower_w;
+        P.c_stride = conv->stride;
+        P.taps = conv->taps;
         P.y_tap_rows = conv->y_tap_rows;
+        for (int t = 0; t < conv->taps; ++t) {
+            if (conv->oh[t] < 0 || conv->ow[t] < 0) return CDL_ERR_ARG;
+            P.tap_oh[t] = conv->oh[t];
+            P.tap_ow[t] = conv->ow[t];
+            P.tap_y[t] = conv->ytap[t];
+        }
+        if (scatter) {
+            P.sc_on = 1;
+            P.sc_P = conv->P;
+            P.sc_Q = conv->Q;
+            P.sc_H = conv->sc_H;
+            P.sc_W = conv->sc_W;
+            P.sc_s = conv->sc_s;
+            P.sc_a = conv->sc_a;
+            P.sc_b = conv->sc_b;
+        }
     }
     P.scale = scale;
     P.f_acc = accumulate_f ? 1 : 0;
@@ -1022,14 +1080,15 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
     else if (conv != nullptr && conv->y_tap_rows > 0)   // all taps' row blocks of the stored matrix, conv->C reduced columns each
-        ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->R * conv->S * conv->y_tap_rows,
+        ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->y_rows,
                               (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
     else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
     // outputs through shared memory + TMA when their pitch and base allow it and the tile is at least one box wide
     CUtensorMap map_f = map_a, map_acc = map_a;      // placeholders when unused
-    const bool out_ok = TN >= 32 && (J & 3) == 0;
+    const bool out_ok = TN >= 32 && (J & 3) == 0 && !scatter;      // scattered rows are copied out by the warps
     P.tma_f = 0;
     P.tma_acc = 0;
+    P.copy_vec = ((J & 3) == 0 && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0 && (reinterpret_cast<uintptr_t>(P.acc_out) & 15u) == 0) ? 1 : 0;
     if (out_ok && splits == 1 && !slabs && f_out != nullptr && (reinterpret_cast<uintptr_t>(f_out) & 15u) == 0) {
         ok = ok && encode_out_map(&map_f, f_out, (uint64_t)J, (uint64_t)I, true);
         P.tma_f = 1;

@@ -77,15 +77,24 @@ int launch_gradient_digits(const float *g, long long rows, int cols, int ld, flo
 int launch_huffman(const unsigned long long *hist, int nlev, unsigned char *lengths, unsigned long long *total_bits,
                    double *avg_bits, cudaStream_t stream);
 
-// The X operand as an implicit patch matrix of a convolution (stride 1, zero padding, output the size of the
-// input): X.ptr then is an [N,H,W,C] tensor of index bytes, C a multiple of 128, and the rows / columns of the
-// patch matrix are gathered by TMA im2col loads, never stored.
+// The X operand as an implicit patch matrix of a convolution: X.ptr then is an [N,H,W,C] tensor of index bytes and
+// the rows / columns of the patch matrix are gathered by TMA im2col loads, never stored.  The gather is described by
+// a grid of P x Q base pixels per image - base pixel (p, q) sits at (lower_h + p * stride, lower_w + q * stride), which
+// may lie outside the tensor (padding reads as zero) - and by `taps` filter taps, tap t reading the pixel at offset
+// (oh[t], ow[t]) >= 0 from the base pixel.
+constexpr int kConvMaxTaps = 64;
 struct ConvGather {
     int N, H, W, C;         // the gathered tensor
-    int R, S;               // filter height and width (odd); padding is (R-1)/2, (S-1)/2
+    int P, Q;               // base pixels per image (rows of the patch matrix = N * P * Q)
+    int lower_h, lower_w, stride;
+    int taps;
+    signed char oh[kConvMaxTaps], ow[kConvMaxTaps];
     int transposed;         // 0: X(i = pixel, r = tap * C + c);  1: X(i = tap * C + c, r = pixel)
-    int y_tap_rows;         // > 0: Y is stored as [taps * y_tap_rows][C] (r contiguous) and the block of tap t is the
-                            //      one of the mirrored tap, rows (taps - 1 - t) * y_tap_rows ..  (backward-data product)
+    int y_tap_rows;         // > 0: Y is stored as [.. * y_tap_rows][C] (r contiguous) and the block of tap t starts at row
+    unsigned char ytap[kConvMaxTaps];   //  ytap[t] * y_tap_rows  (backward-data products: the filter's own tap of gather tap t)
+    int y_rows;             //  ... and y_rows rows in all
+    // output rows scattered over a larger image (see TcParams): row (n, p, q) -> pixel (n, sc_s p + sc_a, sc_s q + sc_b)
+    int sc_on, sc_H, sc_W, sc_s, sc_a, sc_b;
 };
 
 // Hard index of the next layer's quantizer, computed in the forward product's epilogue from the float output:

@@ -159,11 +159,18 @@ def resnet18_layers(batch: int = 256):
 
 
 def resnet18_conv_geometry(name: str):
-    """(H, W, C, R, S) of the ResNet-18 layers that are stride-1 3x3 convolutions with as many output as input
-    channels (the layers the convolution form of the products covers), else None."""
+    """(H, W, C, R, S, stride, padding) of a ResNet-18 layer as a convolution on its NHWC input tensor, for the layers
+    the convolution form of the products covers: every 3 x 3 layer (the first of stages 2-4 with stride 2) and the
+    1 x 1 stride-2 shortcuts.  None for conv1 (3 input channels) and the fully connected layer."""
     side = {"layer1": (56, 64), "layer2": (28, 128), "layer3": (14, 256), "layer4": (7, 512)}
     stage, _, idx = name.partition(".")
-    if stage in side and (idx in ("1", "2", "3") or (stage == "layer1" and idx == "0")):
-        hw, c = side[stage]
-        return hw, hw, c, 3, 3
+    if stage not in side:
+        return None
+    hw, c = side[stage]
+    if idx in ("1", "2", "3") or (stage == "layer1" and idx == "0"):
+        return hw, hw, c, 3, 3, 1, 1
+    if idx == "0":                      # opens the stage: input of the previous stage's size, stride 2
+        return 2 * hw, 2 * hw, c // 2, 3, 3, 2, 1
+    if idx == "ds":
+        return 2 * hw, 2 * hw, c // 2, 1, 1, 2, 0
     return None

@@ -20,7 +20,7 @@ step 4, the weight-gradient product of step 7 delivers its int32 accumulators, w
 converted to float once (cdl_rescale_acc), and the two scalar gradients of the activation quantizer are summed at
 the end; everything that depends on the weights alone is identical on every rank and is not exchanged.
 
-With conv=ConvShape(...) the layer is a stride-1 convolution computed straight from the NHWC index tensor
+With conv=ConvShape(...) the layer is a convolution (any stride and padding cdl_qconv_* takes) computed straight from the NHWC index tensor
 (cdl_qconv_fwd / cdl_qconv_bwd): steps 5 and 7 read X_idx itself, dA becomes dL/dQ(x) in the layout of x, and step 8
 takes it as its incoming gradient, so the only inputs of a step are w, x and dL/dY.
 """
@@ -36,11 +36,12 @@ class CdlLayerStep:
     def __init__(self, torch, M, K, N, n_x, wq, xq, q_g, device="cuda", lda=None, need_dx=True, conv=None):
         """wq / xq: objects with q, lo, hi, alpha, rate_weight, window (weights / activations); n_x: number of
         activation elements quantized per step (the layer's input tensor, before im2col); conv: a ConvShape for
-        the convolution form (then M = N*H*W pixels, K = R*S*C, n_x = M*C)."""
+        the convolution form (then M = N*P*Q output pixels, K = R*S*C, n_x = N*H*W*C input elements)."""
         self.torch = torch
         self.conv = conv
         if conv is not None:
-            assert M == conv.N * conv.H * conv.W and K == conv.R * conv.S * conv.C and n_x == M * conv.C
+            assert M == conv.N * conv.P * conv.Q and K == conv.R * conv.S * conv.C
+            assert n_x == conv.N * conv.H * conv.W * conv.C
         self.M, self.K, self.N, self.n_x, self.n_w = M, K, N, n_x, K * N
         self.need_dx = need_dx      # False for the first layer of a network: its input needs no gradient
         self.lda = lda if lda is not None else (K + 15) // 16 * 16     # row pitch of A_idx (multiple of 16 bytes)
