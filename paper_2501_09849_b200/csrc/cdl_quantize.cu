@@ -715,117 +715,146 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
     float4 *gx4 = reinterpret_cast<float4 *>(gx + head);
     unsigned int *idx4 = reinterpret_cast<unsigned int *>(idx + head);
 
-    for (int64_t base = tid; base < n4; base += stride * kBatch) {
-        float4 xv[kBatch], gv[kBatch];
+    // One 128-bit group (four elements): quantize, store, count.  The running sums of the scalar gradients are kept
+    // across the groups of a batch and flushed to double precision after it.
+    float part_q = 0.0f, part_a = 0.0f;
+    float2 part_q2 = make_float2(0.0f, 0.0f), part_a2 = make_float2(0.0f, 0.0f);    // pair path: two running sums each
+    auto group = [&](const float4 xq, const float4 gq, const int64_t i, float4 *yp, float4 *gxp, unsigned int *ip) {
+        const float xs[4] = {xq.x, xq.y, xq.z, xq.w};
+        float gs[4] = {0.f, 0.f, 0.f, 0.f};
+        if (MODE == MODE_BWD) {
+            gs[0] = gq.x;
+            gs[1] = gq.y;
+            gs[2] = gq.z;
+            gs[3] = gq.w;
+        }
+        if (MODE == MODE_SAMPLE) {
+            // the uniform numbers of elements e0 .. e0+3: one Philox block when e0 is a multiple of 4
+            const unsigned long long e0 = P.first_index + (unsigned long long)(head + 4 * i);
+            if ((e0 & 3ull) == 0ull) {
+                const uint4 r = philox4x32_10(e0 >> 2, P.seed);
+                gs[0] = u01(r.x);
+                gs[1] = u01(r.y);
+                gs[2] = u01(r.z);
+                gs[3] = u01(r.w);
+            } else {
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int64_t i = base + b * stride;
-            if (i < n4) {
-                xv[b] = CDL_LD(x4 + i);
-                if (MODE == MODE_BWD) gv[b] = CDL_LD(g4 + i);
+                for (int c = 0; c < 4; ++c) gs[c] = philox_uniform(P.seed, e0 + c);
             }
         }
-        float part_q = 0.0f, part_a = 0.0f;
-        float2 part_q2 = make_float2(0.0f, 0.0f), part_a2 = make_float2(0.0f, 0.0f);    // pair path: two running sums each
+        float ys[4], gxs[4];
+        unsigned int packed = 0u;
+        constexpr bool kPairs = (PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE))) ||
+                                (PATH == PATH_LATTICE && !RATE && (MODE == MODE_BWD || MODE == MODE_SOFT));
+        // LATTICE: the table form serves a warp all of whose elements have jmax levels on either side of
+        // their nearest one; a warp with an element near the edge of the index set (or outside it) takes
+        // the level loop, which visits exactly each element's levels
+        bool use_pairs = kPairs;
+        PairOut quad[2];
+        if (PATH == PATH_LATTICE && kPairs) {
+            LatPair s0, s1;
+            lattice_index(P, make_float2(xs[0], xs[1]), s0);
+            lattice_index(P, make_float2(xs[2], xs[3]), s1);
+            const int klo = P.lo + P.jmax, khi = P.hi - P.jmax;
+            const bool inner = min(min(s0.k0, s0.k1), min(s1.k0, s1.k1)) >= klo &&
+                               max(max(s0.k0, s0.k1), max(s1.k0, s1.k1)) <= khi;
+            use_pairs = __all_sync(__activemask(), inner);
+            if (use_pairs) quant_quad_lattice<MODE>(P, Gtab, Htab, xs, gs, s0, s1, quad);
+        }
+        if (kPairs && use_pairs) {
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int64_t i = base + b * stride;
-            if (i < n4) {
-                const float xs[4] = {xv[b].x, xv[b].y, xv[b].z, xv[b].w};
-                float gs[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int h = 0; h < 2; ++h) {
+                const float2 xp = make_float2(xs[2 * h], xs[2 * h + 1]), gp = make_float2(gs[2 * h], gs[2 * h + 1]);
+                const PairOut o = PATH == PATH_LATTICE ? quad[h] : quant_pair_near3<MODE, RATE>(P, Dtab, xp, gp);
+                ys[2 * h] = o.y.x;
+                ys[2 * h + 1] = o.y.y;
+                gxs[2 * h] = o.gx.x;
+                gxs[2 * h + 1] = o.gx.y;
                 if (MODE == MODE_BWD) {
-                    gs[0] = gv[b].x;
-                    gs[1] = gv[b].y;
-                    gs[2] = gv[b].z;
-                    gs[3] = gv[b].w;
+                    const float2 gg = make_float2(gs[2 * h], gs[2 * h + 1]);
+                    part_q2 = __ffma2_rn(gg, o.tq, part_q2);
+                    part_a2 = __ffma2_rn(gg, o.ta, part_a2);
                 }
-                if (MODE == MODE_SAMPLE) {
-                    // the uniform numbers of elements e0 .. e0+3: one Philox block when e0 is a multiple of 4
-                    const unsigned long long e0 = P.first_index + (unsigned long long)(head + 4 * i);
-                    if ((e0 & 3ull) == 0ull) {
-                        const uint4 r = philox4x32_10(e0 >> 2, P.seed);
-                        gs[0] = u01(r.x);
-                        gs[1] = u01(r.y);
-                        gs[2] = u01(r.z);
-                        gs[3] = u01(r.w);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) gs[c] = philox_uniform(P.seed, e0 + c);
-                    }
+                packed = h == 0 ? __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040)
+                                : __byte_perm(packed, __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040), 0x5410);
+                if (MODE != MODE_BWD && do_hist) {
+                    hist_inc(hist_a, o.k0[0]);
+                    hist_inc(hist_a, o.k0[1]);
                 }
-                float ys[4], gxs[4];
-                unsigned int packed = 0u;
-                constexpr bool kPairs = (PATH == PATH_NEAR3 && (MODE == MODE_BWD || MODE == MODE_SAMPLE || (MODE == MODE_SOFT && !RATE))) ||
-                                        (PATH == PATH_LATTICE && !RATE && (MODE == MODE_BWD || MODE == MODE_SOFT));
-                // LATTICE: the table form serves a warp all of whose elements have jmax levels on either side of
-                // their nearest one; a warp with an element near the edge of the index set (or outside it) takes
-                // the level loop, which visits exactly each element's levels
-                bool use_pairs = kPairs;
-                PairOut quad[2];
-                if (PATH == PATH_LATTICE && kPairs) {
-                    LatPair s0, s1;
-                    lattice_index(P, make_float2(xs[0], xs[1]), s0);
-                    lattice_index(P, make_float2(xs[2], xs[3]), s1);
-                    const int klo = P.lo + P.jmax, khi = P.hi - P.jmax;
-                    const bool inner = min(min(s0.k0, s0.k1), min(s1.k0, s1.k1)) >= klo &&
-                                       max(max(s0.k0, s0.k1), max(s1.k0, s1.k1)) <= khi;
-                    use_pairs = __all_sync(__activemask(), inner);
-                    if (use_pairs) quant_quad_lattice<MODE>(P, Gtab, Htab, xs, gs, s0, s1, quad);
-                }
-                if (kPairs && use_pairs) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const float2 xp = make_float2(xs[2 * h], xs[2 * h + 1]), gp = make_float2(gs[2 * h], gs[2 * h + 1]);
-                        const PairOut o = PATH == PATH_LATTICE ? quad[h] : quant_pair_near3<MODE, RATE>(P, Dtab, xp, gp);
-                        ys[2 * h] = o.y.x;
-                        ys[2 * h + 1] = o.y.y;
-                        gxs[2 * h] = o.gx.x;
-                        gxs[2 * h + 1] = o.gx.y;
-                        if (MODE == MODE_BWD) {
-                            const float2 gg = make_float2(gs[2 * h], gs[2 * h + 1]);
-                            part_q2 = __ffma2_rn(gg, o.tq, part_q2);
-                            part_a2 = __ffma2_rn(gg, o.ta, part_a2);
-                        }
-                        packed = h == 0 ? __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040)
-                                        : __byte_perm(packed, __byte_perm((unsigned int)o.k0[0], (unsigned int)o.k0[1], 0x0040), 0x5410);
-                        if (MODE != MODE_BWD && do_hist) {
-                            hist_inc(hist_a, o.k0[0]);
-                            hist_inc(hist_a, o.k0[1]);
-                        }
-                    }
-                }
-                if (MODE == MODE_HARD) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        int k0, k1;
-                        hard_pair(P, make_float2(xs[2 * h], xs[2 * h + 1]), k0, k1);
-                        packed = h == 0 ? __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040)
-                                        : __byte_perm(packed, __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040), 0x5410);
-                        if (do_hist) {
-                            hist_inc(hist_a, k0);
-                            hist_inc(hist_a, k1);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int c = 0; c < (((kPairs && PATH != PATH_LATTICE) || MODE == MODE_HARD) ? 0 : 4); ++c) {
-                    if (kPairs && use_pairs) break;      // (only LATTICE decides this at run time; the bound stays constant)
-                    const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
-                    ys[c] = o.y;
-                    gxs[c] = o.gx;
-                    part_q += o.tq;
-                    part_a += o.ta;
-                    packed |= ((unsigned int)o.k0 & 0xffu) << (8 * c);
-                    if (MODE != MODE_BWD && do_hist) hist_inc(hist_a, o.k0);
-                }
-                if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) CDL_ST(y4 + i, make_float4(ys[0], ys[1], ys[2], ys[3]));
-                if (MODE == MODE_BWD && gx != nullptr) CDL_ST(gx4 + i, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
-                if (MODE != MODE_BWD && idx != nullptr) idx4[i] = packed;
             }
         }
+        if (MODE == MODE_HARD) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                int k0, k1;
+                hard_pair(P, make_float2(xs[2 * h], xs[2 * h + 1]), k0, k1);
+                packed = h == 0 ? __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040)
+                                : __byte_perm(packed, __byte_perm((unsigned int)k0, (unsigned int)k1, 0x0040), 0x5410);
+                if (do_hist) {
+                    hist_inc(hist_a, k0);
+                    hist_inc(hist_a, k1);
+                }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < (((kPairs && PATH != PATH_LATTICE) || MODE == MODE_HARD) ? 0 : 4); ++c) {
+            if (kPairs && use_pairs) break;      // (only LATTICE decides this at run time; the bound stays constant)
+            const ElemOut o = quant_elem<MODE, PATH, RATE>(P, Ltab, xs[c], gs[c], mp_s, lane);
+            ys[c] = o.y;
+            gxs[c] = o.gx;
+            part_q += o.tq;
+            part_a += o.ta;
+            packed |= ((unsigned int)o.k0 & 0xffu) << (8 * c);
+            if (MODE != MODE_BWD && do_hist) hist_inc(hist_a, o.k0);
+        }
+        if (MODE == MODE_SOFT || (MODE == MODE_SAMPLE && y != nullptr)) CDL_ST(yp, make_float4(ys[0], ys[1], ys[2], ys[3]));
+        if (MODE == MODE_BWD && gx != nullptr) CDL_ST(gxp, make_float4(gxs[0], gxs[1], gxs[2], gxs[3]));
+        if (MODE != MODE_BWD && idx != nullptr) *ip = packed;
+    };
+    auto flush_partials = [&]() {
         if (MODE == MODE_BWD) {
             acc_q += (double)(part_q + (part_q2.x + part_q2.y));
             acc_a += (double)(part_a + (part_a2.x + part_a2.y));
+            part_q = part_a = 0.0f;
+            part_q2 = part_a2 = make_float2(0.0f, 0.0f);
+        }
+    };
+
+    // Whole batches first (kBatch loads in flight, no bounds checks inside), then the at most kBatch - 1 groups left
+    // over; every stream is walked with a running pointer, so a step costs additions, not 64-bit address arithmetic.
+    {
+        int64_t i = tid;
+        const float4 *xp = x4 + i, *gp = g4 + i;
+        float4 *yp = y4 + i, *gxp = gx4 + i;
+        unsigned int *ip = idx4 + i;
+        const int64_t last_full = n4 - (kBatch - 1) * stride;       // a batch starting below this is whole
+        for (; i < last_full; i += kBatch * stride) {
+            float4 xv[kBatch], gv[kBatch];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                xv[b] = CDL_LD(xp + b * stride);
+                if (MODE == MODE_BWD) gv[b] = CDL_LD(gp + b * stride);
+            }
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b)
+                group(xv[b], MODE == MODE_BWD ? gv[b] : make_float4(0.f, 0.f, 0.f, 0.f), i + b * stride, yp + b * stride, gxp + b * stride, ip + b * stride);
+            flush_partials();
+            xp += kBatch * stride;
+            gp += kBatch * stride;
+            yp += kBatch * stride;
+            gxp += kBatch * stride;
+            ip += kBatch * stride;
+        }
+        for (; i < n4; i += stride) {
+            const float4 xq = CDL_LD(xp);
+            const float4 gq = MODE == MODE_BWD ? CDL_LD(gp) : make_float4(0.f, 0.f, 0.f, 0.f);
+            group(xq, gq, i, yp, gxp, ip);
+            flush_partials();
+            xp += stride;
+            gp += stride;
+            yp += stride;
+            gxp += stride;
+            ip += stride;
         }
     }
 
