@@ -827,7 +827,10 @@ quantize_kernel(const QuantDev P, const float *__restrict__ x, const float *__re
         const float4 *xp = x4 + i, *gp = g4 + i;
         float4 *yp = y4 + i, *gxp = gx4 + i;
         unsigned int *ip = idx4 + i;
-        const int64_t last_full = n4 - (kBatch - 1) * stride;       // a batch starting below this is whole
+        // (The level-loop paths have a long body that the arithmetic, not the loads, paces: they take the one-group
+        // loop below for everything, which keeps a single copy of that body in the instruction cache.)
+        constexpr bool kLongBody = MODE != MODE_HARD && (PATH == PATH_LOOP || PATH == PATH_LATTICE);
+        const int64_t last_full = kLongBody ? 0 : n4 - (kBatch - 1) * stride;       // a batch starting below this is whole
         for (; i < last_full; i += kBatch * stride) {
             float4 xv[kBatch], gv[kBatch];
 #pragma unroll
