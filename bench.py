@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--no-extras", action="store_true",
                     help="default line without its sweep / gemm / network blocks (e.g. for a profiler capture)")
     ap.add_argument("--no-network", action="store_true", help="default line without the whole-network block")
+    ap.add_argument("--call-steps", type=int, default=None,
+                    help="steps of the call-by-call pass that times each kernel (default: --steps, at least 50, at most 500)")
     ap.add_argument("--no-graph", action="store_true", help="launch the calls of a step one by one instead of replaying a CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="quantizer-only bandwidth sweep (sizes x levels x alpha), one JSON line, 1 GPU")
@@ -236,7 +238,7 @@ def kernel_table(calls, model, per_call_ms, hbm, tp):
     return kernels
 
 
-def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, peaks_hbm, tp):
+def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, peaks_hbm, tp, call_steps=None):
     """The same layer as a convolution computed straight from the NHWC index tensor (cdl_qconv_*): same w, x and
     dL/dY, the data gradient feeds the activation quantizer's backward pass directly.  Returns a dict of times."""
     n_img, H, W, C = case.a_shape
@@ -262,7 +264,7 @@ def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, p
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    k_steps = max(50, min(steps, 200))
+    k_steps = call_steps if call_steps else max(50, min(steps, 200))
     per = per_call_times(torch, cs, CALLS, k_steps, stream)
     model = conv_call_model(case, step.n_x)
     kern = kernel_table(CALLS, model, per, peaks_hbm, tp)
@@ -1006,7 +1008,7 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
 
     # ---- per-call times: a second pass over the same steps, launched call by call with an event between calls
-    k_steps = max(50, min(args.steps, 500))
+    k_steps = args.call_steps if args.call_steps else max(50, min(args.steps, 500))
     per_call_ms = per_call_times(torch, step, CALLS, k_steps, stream, **run_kw)
     status = cdl.cdl_workspace_status(step.ws, check=False)
 
@@ -1082,7 +1084,8 @@ def main():
                               "host kept ahead of the device"),
         }
         if world == 1 and args.workload == "resnet18_layer3_conv" and not args.no_implicit:
-            line["implicit_conv"] = run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, args.steps, hbm, tp)
+            line["implicit_conv"] = run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, args.steps, hbm, tp,
+                                                      args.call_steps)
         extras = world == 1 and args.workload == "resnet18_layer3_conv" and not args.no_extras
         if extras:
             del step, graph
