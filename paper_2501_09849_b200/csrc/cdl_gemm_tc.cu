@@ -260,29 +260,54 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
-__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
-}
-
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+// The four MMAs (K = 32 each) of one 128-byte stage in one go: descriptor k is (lo + k * step, hi); the first one
+// accumulates only when `accumulate` is set, the others always.
+template <bool PAIR>
+__device__ __forceinline__ void tc_mma4_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step, uint32_t b_lo,
+                                           uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
+    if (PAIR) {
+        asm volatile(
+            "{\n\t.reg .pred p, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+            "setp.ne.b32 p, %8, 0;\n\t"
+            "setp.eq.b32 t, 0, 0;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%4, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, p;\n\t"
+            "add.u32 al, %1, %3;\n\tadd.u32 bl, %4, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, t;\n\t"
+            "add.u32 al, al, %3;\n\tadd.u32 bl, bl, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, t;\n\t"
+            "add.u32 al, al, %3;\n\tadd.u32 bl, bl, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, t;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+            "setp.ne.b32 p, %8, 0;\n\t"
+            "setp.eq.b32 t, 0, 0;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%4, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, p;\n\t"
+            "add.u32 al, %1, %3;\n\tadd.u32 bl, %4, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, t;\n\t"
+            "add.u32 al, al, %3;\n\tadd.u32 bl, bl, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, t;\n\t"
+            "add.u32 al, al, %3;\n\tadd.u32 bl, bl, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, t;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
+    }
 }
 
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
@@ -416,98 +441,125 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const uint32_t stage_tx = (uint32_t)kABytes + b_bytes;
     bool failed = false;
 
+    // The three roles below are single threads, and what bounds a pipeline stage is the length of their own
+    // instruction streams (a poll of a barrier that is already complete costs some 40 cycles, every dependent
+    // instruction a handful): each stage loop therefore keeps running addresses and coordinates, has no division,
+    // no table look-up outside a tap change and no test of a launch parameter that could be taken outside.
+    const uint32_t bar0 = smem_u32(&bars[0]);                    // full barriers; the empty ones follow at + 8 * kStagesMax
+    constexpr uint32_t kEmptyOff = 8u * kStagesMax;
+    constexpr uint32_t kRingBytes = (uint32_t)kStages * (uint32_t)kStageBytes;
+
     if (warp == 0 || warp == 2 + kEpiWarps) {
         // ------------------------------------------------------------ TMA producer (one lane; with a second TMA
         // warp the first issues the X-operand loads and arms the barrier, the second issues the Y-operand loads)
         const bool do_a = warp == 0, do_b = !kSplitProducer || warp != 0;
         if (lane == 0) {
-            uint32_t it = 0;
+            const int conv = P.conv, a_mn = P.a_mn_major, b_mn = P.b_mn_major, TNv = P.TN, tiles_j = P.tiles_j;
+            const int cW = P.cW > 0 ? P.cW : 1, cH = P.cH > 0 ? P.cH : 1, cHW = cH * cW;
+            const int cpad = P.cpad, cC = P.cC, c_stride = P.c_stride, pad_w = P.pad_w, pad_h = P.pad_h;
+            const int last_tap = P.taps - 1, y_tap_rows = P.y_tap_rows;
+            const int pix_dh = BR / cW, pix_dw = BR % cW;        // 128 pixels further on
+            // pair: both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
+            const uint32_t arm_tx = PAIR ? 2u * stage_tx : stage_tx;
+            const bool arm = do_a && rank == 0;
+            uint32_t st_off = 0u, st_bar = bar0, st_par = 1u;    // ring position: byte offset, full barrier, parity of "empty"
             SlotWork sw = slot_work(P, slot);
             while (!failed) {
                 const WorkItem w = next_item(sw);
                 if (!w.valid) break;
                 const int tile = w.tile;
-                const int ti = tile / P.tiles_j, tj = tile % P.tiles_j;
-                const int rb0 = w.rb0, rb1 = w.rb1;
+                const int ti = tile / tiles_j, tj = tile - ti * tiles_j;
+                const int rb0 = w.rb0, nrb = w.rb1 - w.rb0;
                 const int arow = ti * TMU + (int)rank * TM;
-                // Patch gather: pixel block, channel block and filter tap of the first stage of this unit, kept up
-                // to date with additions only inside the loop (this one thread feeds the whole pipeline).
-                int g_cb = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, g_tap = 0, g_c0 = 0;
-                if (P.conv != 0) {
+                const int b_row0 = tj * TNv + brow;
+                // Patch gather: pixel block, channel offset and filter tap of the first stage of this unit
+                int g_c = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, g_tap = 0, b_tap_red = 0, b_tap_row = 0;
+                if (conv != 0) {
                     // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
                     const int i0 = arow < P.I ? arow : 0;
-                    g_tap = P.conv == 1 ? rb0 / P.cblocks : i0 / P.cpad;
-                    g_cb = P.conv == 1 ? rb0 % P.cblocks : 0;
-                    g_c0 = P.conv == 1 ? 0 : i0 % P.cpad;
-                    const int pix = P.conv == 1 ? i0 : rb0 * BR;
-                    g_n = pix / (P.cH * P.cW);
-                    const int rem = pix - g_n * (P.cH * P.cW);
-                    g_h = rem / P.cW;
-                    g_w = rem % P.cW;
+                    g_tap = conv == 1 ? rb0 / P.cblocks : i0 / cpad;
+                    g_c = conv == 1 ? (rb0 - g_tap * P.cblocks) * BR : i0 - g_tap * cpad;
+                    const int pix = conv == 1 ? i0 : rb0 * BR;
+                    g_n = pix / cHW;
+                    const int rem = pix - g_n * cHW;
+                    g_h = rem / cW;
+                    g_w = rem - g_h * cW;
                     g_oh = P.tap_oh[g_tap];
                     g_ow = P.tap_ow[g_tap];
+                    // Y coordinates of a tap: its own row block of a stacked matrix, or C (not the padded count)
+                    // reduced columns per tap of a plain one
+                    b_tap_row = y_tap_rows > 0 ? (int)P.tap_y[g_tap] * y_tap_rows : 0;
+                    b_tap_red = y_tap_rows > 0 || conv != 1 ? 0 : g_tap * cC;
                 }
-                const int pix_dh = BR / (P.cW > 0 ? P.cW : 1), pix_dw = BR % (P.cW > 0 ? P.cW : 1);   // 128 pixels further on
-                for (int rb = rb0; rb < rb1; ++rb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, P.wait_ns)) {
+                int c_red = rb0 * BR;                            // reduced coordinate of a stored operand
+                int c_w = g_w * c_stride - pad_w, c_h = g_h * c_stride - pad_h;
+                for (int i = 0; i < nrb; ++i) {
+                    if (!mbar_try_wait_now(st_bar + kEmptyOff, st_par) &&
+                        !mbar_wait(st_bar + kEmptyOff, st_par, abort_flag, P.wait_ns)) {
                         failed = true;
                         break;
                     }
-                    const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
-                    const uint32_t sb = sa + kABytes;
-                    int b_row = tj * P.TN + brow;
-                    if (P.y_tap_rows > 0) b_row += (int)P.tap_y[g_tap] * P.y_tap_rows;
-                    // Y coordinate along r: the stored matrix has C (not the padded count) rows per tap
-                    const int b_red = P.y_tap_rows > 0 ? g_cb * BR : (P.conv == 1 ? g_tap * P.cC + g_cb * BR : rb * BR);
-                    const int g_c = P.conv == 1 ? g_cb * BR : g_c0;
-                    const int c_w = g_w * P.c_stride - P.pad_w, c_h = g_h * P.c_stride - P.pad_h, c_n = g_n, c_ow = g_ow, c_oh = g_oh;
-                    if (P.conv == 1) {            // next stage: next channel block, then next tap
-                        if (++g_cb == P.cblocks) {
-                            g_cb = 0;
-                            g_tap = g_tap + 1 < P.taps ? g_tap + 1 : g_tap;      // (past the last tap nothing more is loaded)
-                            g_oh = P.tap_oh[g_tap];
-                            g_ow = P.tap_ow[g_tap];
-                        }
-                    } else if (P.conv == 2) {     // next stage: 128 pixels further on
-                        g_w += pix_dw;
-                        g_h += pix_dh;
-                        if (g_w >= P.cW) {
-                            g_w -= P.cW;
-                            ++g_h;
-                        }
-                        while (g_h >= P.cH) {
-                            g_h -= P.cH;
-                            ++g_n;
-                        }
+                    const uint32_t sa = smem_base + st_off, sb = sa + kABytes, fb = st_bar;
+                    st_off += (uint32_t)kStageBytes;
+                    st_bar += 8u;
+                    if (st_off == kRingBytes) {
+                        st_off = 0u;
+                        st_bar = bar0;
+                        st_par ^= 1u;
                     }
-                    if (PAIR) {
-                        // both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
-                        if (rank == 0 && do_a) mbar_expect_tx(full_bar(s), 2u * stage_tx);
+                    if (arm) mbar_expect_tx(fb, arm_tx);
+                    if (conv == 0) {
                         if (do_a) {
-                            if (P.conv != 0) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
-                            else if (P.a_mn_major) tma_load_2d_pair(sa, &map_a, arow, rb * BR, full_bar(s));
-                            else tma_load_2d_pair(sa, &map_a, rb * BR, arow, full_bar(s));
+                            const int x0 = a_mn ? arow : c_red, x1 = a_mn ? c_red : arow;    // {inner, outer}
+                            if (PAIR) tma_load_2d_pair(sa, &map_a, x0, x1, fb);
+                            else tma_load_2d(sa, &map_a, x0, x1, fb);
                         }
                         if (do_b) {
-                            if (P.b_mn_major) tma_load_2d_pair(sb, &map_b, b_row, b_red, full_bar(s));
-                            else tma_load_2d_pair(sb, &map_b, b_red, b_row, full_bar(s));
+                            const int y0 = b_mn ? b_row0 : c_red, y1 = b_mn ? c_red : b_row0;
+                            if (PAIR) tma_load_2d_pair(sb, &map_b, y0, y1, fb);
+                            else if (b_mn) {
+                                for (int bb = 0; bb < b_blocks; ++bb) tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, y0 + bb * 128, y1, fb);
+                            } else tma_load_2d(sb, &map_b, y0, y1, fb);
                         }
+                        c_red += BR;
                         continue;
                     }
                     if (do_a) {
-                        mbar_expect_tx(full_bar(s), stage_tx);
-                        if (P.conv != 0) tma_load_im2col(sa, &map_a, g_c, c_w, c_h, c_n, c_ow, c_oh, full_bar(s));
-                        else if (P.a_mn_major) tma_load_2d(sa, &map_a, arow, rb * BR, full_bar(s));   // {i (inner), r}
-                        else tma_load_2d(sa, &map_a, rb * BR, arow, full_bar(s));                 // {r (inner), i}
+                        if (PAIR) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
+                        else tma_load_im2col(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
                     }
-                    if (!do_b) continue;
-                    if (P.b_mn_major) {
-                        for (int bb = 0; bb < b_blocks; ++bb)
-                            tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, b_row + bb * 128, b_red, full_bar(s));
-                    } else {
-                        tma_load_2d(sb, &map_b, b_red, b_row, full_bar(s));
+                    if (do_b) {
+                        const int red = conv == 1 ? b_tap_red + g_c : c_red, row = b_row0 + b_tap_row;
+                        const int y0 = b_mn ? row : red, y1 = b_mn ? red : row;
+                        if (PAIR) tma_load_2d_pair(sb, &map_b, y0, y1, fb);
+                        else if (b_mn) {
+                            for (int bb = 0; bb < b_blocks; ++bb) tma_load_2d(sb + (uint32_t)bb * 128 * BR, &map_b, y0 + bb * 128, y1, fb);
+                        } else tma_load_2d(sb, &map_b, y0, y1, fb);
+                    }
+                    if (conv == 1) {              // next stage: next channel block, then next tap
+                        g_c += BR;
+                        if (g_c == cpad) {
+                            g_c = 0;
+                            g_tap = g_tap < last_tap ? g_tap + 1 : g_tap;      // (past the last tap nothing more is loaded)
+                            g_oh = P.tap_oh[g_tap];
+                            g_ow = P.tap_ow[g_tap];
+                            if (y_tap_rows > 0) b_tap_row = (int)P.tap_y[g_tap] * y_tap_rows;
+                            else b_tap_red = g_tap * cC;
+                        }
+                    } else {                      // next stage: 128 pixels further on
+                        c_red += BR;
+                        g_w += pix_dw;
+                        g_h += pix_dh;
+                        if (g_w >= cW) {
+                            g_w -= cW;
+                            ++g_h;
+                        }
+                        while (g_h >= cH) {
+                            g_h -= cH;
+                            ++g_n;
+                        }
+                        c_w = g_w * c_stride - pad_w;
+                        c_h = g_h * c_stride - pad_h;
                     }
                 }
             }
@@ -519,12 +571,25 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (one lane; CTA 0 in pair mode)
         if (lane == 0 && rank == 0) {
-            uint32_t it = 0, tcount = 0;
+            // Operand descriptors: the upper word is fixed per launch (stride between 8-row groups, version, swizzle),
+            // the lower word holds the start address and the leading offset and moves with the stage and with k.
+            // K-major: rows are 128-byte lines, 8-row groups 1024 bytes apart, 32 bytes per MMA along r.
+            // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of the
+            // non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
+            const uint64_t a_d0 = P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024);
+            const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + kABytes, 128 * BR, 1024) : make_desc(smem_base + kABytes, 16, 1024);
+            const uint32_t a_hi = (uint32_t)(a_d0 >> 32), b_hi = (uint32_t)(b_d0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)a_d0, b_lo0 = (uint32_t)b_d0;
+            const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
+            const uint32_t b_step = P.b_mn_major ? (4096u >> 4) : (32u >> 4);
+            const uint32_t idesc = P.idesc;
+            uint32_t tcount = 0;
+            uint32_t st_off16 = 0u, st_bar = bar0, st_par = 0u;     // ring position (offset in 16-byte units), parity of "full"
             SlotWork sw = slot_work(P, slot);
             for (; !failed; ++tcount) {
                 const WorkItem w = next_item(sw);
                 if (!w.valid) break;
-                const int rb0 = w.rb0, rb1 = w.rb1;
+                const int nrb = w.rb1 - w.rb0;
                 const int buf = tcount & 1;
                 const uint32_t tph = (tcount >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, P.wait_ns)) {
@@ -533,32 +598,27 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256u;
-                for (int rb = rb0; rb < rb1; ++rb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag, P.wait_ns)) {
+                uint32_t acc = 0u;                                   // the first MMA of a unit overwrites the accumulator
+                for (int i = 0; i < nrb; ++i) {
+                    if (!mbar_try_wait_now(st_bar, st_par) && !mbar_wait(st_bar, st_par, abort_flag, P.wait_ns)) {
                         failed = true;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sa = smem_base + (uint32_t)s * kStageBytes;
-                    const uint32_t sb = sa + kABytes;
-                    // K-major: rows are 128-byte lines, 8-row groups 1024 bytes apart, 32 bytes per MMA along r.
-                    // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of
-                    // the non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
-                    const uint64_t adesc = P.a_mn_major ? make_desc(sa, 128 * BR, 1024) : make_desc(sa, 16, 1024);
-                    const uint64_t bdesc = P.b_mn_major ? make_desc(sb, 128 * BR, 1024) : make_desc(sb, 16, 1024);
-                    const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
-                    const uint32_t b_step = P.b_mn_major ? (4096u >> 4) : (32u >> 4);
-#pragma unroll
-                    for (int k = 0; k < BR / 32; ++k) {
-                        const uint32_t acc = (rb > rb0 || k > 0) ? 1u : 0u;
-                        if (PAIR) tc_mma_i8_pair(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc, acc);
-                        else tc_mma_i8(d_tmem, adesc + (uint64_t)(k * a_step), bdesc + (uint64_t)(k * b_step), P.idesc, acc);
+                    const uint32_t a_lo = a_lo0 + st_off16, b_lo = b_lo0 + st_off16, eb = st_bar + kEmptyOff;
+                    st_off16 += (uint32_t)(kStageBytes >> 4);
+                    st_bar += 8u;
+                    if (st_off16 == (kRingBytes >> 4)) {
+                        st_off16 = 0u;
+                        st_bar = bar0;
+                        st_par ^= 1u;
                     }
+                    if (PAIR) tc_mma4_i8<true>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                    else tc_mma4_i8<false>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                    acc = 1u;
                     // frees the stage (in both CTAs of a pair) once these MMAs have read it
-                    if (PAIR) tc_commit_pair(empty_bar(s));
-                    else tc_commit(empty_bar(s));
+                    if (PAIR) tc_commit_pair(eb);
+                    else tc_commit(eb);
                 }
                 if (!failed) {                               // accumulator complete
                     if (PAIR) tc_commit_pair(tfull_bar(buf));

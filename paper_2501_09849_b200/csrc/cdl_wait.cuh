@@ -44,6 +44,21 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
+// The same poll without a suspend-time hint (the time it may stay suspended is then the implementation's own): it
+// costs about half of the hinted form when the phase is already complete, which is what the single threads that
+// drive a pipeline mostly find, so they try this once before they go into the bounded wait.
+__device__ __forceinline__ bool mbar_try_wait_now(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Records an expired wait in a status block: two tag words first, then the code itself, so that a reader takes
 // the block for a record only when all three words are there (stale memory of a recycled allocation is not).
 __device__ __forceinline__ void record_timeout(int *status)
