@@ -463,19 +463,53 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint32_t arm_tx = PAIR ? 2u * stage_tx : stage_tx;
             const bool arm = do_a && rank == 0;
             uint32_t st_off = 0u, st_bar = bar0, st_par = 1u;    // ring position: byte offset, full barrier, parity of "empty"
+            // Forward-type patch gathers with one tile column and an unsplit reduction visit tiles slot, slot + slots,
+            // ...: the pixel of a tile's first row then moves by a fixed step, kept as (image, row, column) with
+            // carries instead of being divided out of the row index for every tile (a short tile has few stages to
+            // hide that behind).
+            const bool walk = conv == 1 && tiles_j == 1 && P.splits == 1;
+            int wk_n = 0, wk_h = 0, wk_w = 0, wk_dn = 0, wk_dh = 0, wk_dw = 0;
+            if (walk) {
+                const int first = slot * TMU + (int)rank * TM, step = P.slots * TMU;
+                wk_n = first / cHW;
+                wk_h = (first - wk_n * cHW) / cW;
+                wk_w = first - wk_n * cHW - wk_h * cW;
+                wk_dn = step / cHW;
+                wk_dh = (step - wk_dn * cHW) / cW;
+                wk_dw = step - wk_dn * cHW - wk_dh * cW;
+            }
             SlotWork sw = slot_work(P, slot);
             while (!failed) {
                 const WorkItem w = next_item(sw);
                 if (!w.valid) break;
                 const int tile = w.tile;
-                const int ti = tile / tiles_j, tj = tile - ti * tiles_j;
+                const int ti = tiles_j == 1 ? tile : tile / tiles_j, tj = tile - ti * tiles_j;
                 const int rb0 = w.rb0, nrb = w.rb1 - w.rb0;
                 const int arow = ti * TMU + (int)rank * TM;
                 const int b_row0 = tj * TNv + brow;
                 // Patch gather: pixel block, channel offset and filter tap of the first stage of this unit
                 int g_c = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, g_tap = 0, b_tap_red = 0, b_tap_row = 0;
-                if (conv != 0) {
+                if (walk) {
                     // a block wholly outside the matrix (second CTA of a ragged pair) loads block 0: never stored
+                    const bool inside = arow < P.I;
+                    g_n = inside ? wk_n : 0;
+                    g_h = inside ? wk_h : 0;
+                    g_w = inside ? wk_w : 0;
+                    wk_w += wk_dw;
+                    wk_h += wk_dh;
+                    wk_n += wk_dn;
+                    if (wk_w >= cW) {
+                        wk_w -= cW;
+                        ++wk_h;
+                    }
+                    if (wk_h >= cH) {
+                        wk_h -= cH;
+                        ++wk_n;
+                    }
+                    g_oh = P.tap_oh[0];
+                    g_ow = P.tap_ow[0];
+                    b_tap_row = y_tap_rows > 0 ? (int)P.tap_y[0] * y_tap_rows : 0;
+                } else if (conv != 0) {
                     const int i0 = arow < P.I ? arow : 0;
                     g_tap = conv == 1 ? rb0 / P.cblocks : i0 / cpad;
                     g_c = conv == 1 ? (rb0 - g_tap * P.cblocks) * BR : i0 - g_tap * cpad;
