@@ -289,6 +289,8 @@ def run_implicit_conv(torch, cdl, CdlLayerStep, CALLS, case, step, q_g, steps, p
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e_steps,
                     "overlap": "two sets of device buffers: the copy of step i+1 overlaps the kernels of step i"},
             "gpu_launches": steps * cs.kernels_per_step(), "device_status": status, "kernels": kern,
+            "step_hbm": {"bytes": int(sum(m["bytes"] for m in model.values())),
+                         "frac_of_measured_per_gpu": round(sum(m["bytes"] for m in model.values()) / (ms * 1e-3) / 1e9 / peaks_hbm, 4)},
             "note": "same layer through cdl_qconv_fwd/bwd: no stored patch matrix, dX in the layout of x"}
 
 
@@ -1074,6 +1076,10 @@ def main():
             "layer_fwd_bwd_ms": ms_step, "gemm_ms": gemm_ms, "gemm_int8_tops": 6.0 * M * K * N / (gemm_ms * 1e-3) / 1e12,
             "quantizer_ms": quant_ms, "quantizer_Gelem_per_s": quant_elems / (quant_ms * 1e-3) / 1e9,
             "quantizer_hbm_frac_measured": sum(model[c]["bytes"] for c in CALLS if model[c]["elems"]) / (quant_ms * 1e-3) / 1e9 / hbm,
+            # every call's algorithmic bytes over the step time: what the step as a whole makes of the memory system
+            "step_hbm": {"bytes": int(sum(model[c]["bytes"] for c in CALLS)),
+                         "GBps": round(sum(model[c]["bytes"] for c in CALLS) / (ms_step * 1e-3) / 1e9 * world, 1),
+                         "frac_of_measured_per_gpu": round(sum(model[c]["bytes"] for c in CALLS) / (ms_step * 1e-3) / 1e9 / hbm, 4)},
             "kernels": kernels, "roofline": roof, "tensor_peaks": tp, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e_steps,
