@@ -11,8 +11,10 @@
 // In convolution form the X operand is not a stored matrix: its tiles are gathered from an NHWC index tensor by
 // TMA im2col loads (patch matrix of a stride-1 convolution, or its transpose for dW), see ConvGather.
 //
-// Tiling: 128 x TN output tile per work unit (TN in {16..256}), or a 256 x 256 tile shared by a pair of CTAs
-// (tcgen05 cta_group::2) when the output is wide and tall enough; 128 bytes of the reduced dimension per pipeline
+// Tiling: 128 x TN output tile per work unit (TN in {16..256}), a 256 x TN tile of one CTA when TN <= 128 and X is
+// K-major (one 256-row X box per stage, two accumulators: a narrow product gets twice the rows out of every
+// pipeline stage), or a 256 x 256 tile shared by a pair of CTAs (tcgen05 cta_group::2) when the output is wide and
+// tall enough; 128 bytes of the reduced dimension per pipeline
 // stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is [rows][128 bytes] with
 // the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or columns outside the matrix
 // are zero-filled by TMA, which makes ragged edges and R tails exact.
@@ -108,6 +110,7 @@ struct TcParams {
     int slab_rows;          // 0: splits add into one I x J buffer.  > 0: split s stores its partial tile into rows
                             // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
     int slots;              // work slots (CTA pairs, or CTAs) = the grid: slot p takes units p, p + slots, ...
+    int tall;               // 1: a CTA's tile is 256 rows x TN (TN <= 128): one 256-row X box per stage, two accumulators
 };
 
 // One piece of work of a slot: pipeline stages [rb0, rb1) of a tile (a unit of tiles * splits).
@@ -438,7 +441,15 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const uint32_t b_bytes = PAIR ? (uint32_t)(128 * BR)
                                   : (P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR));
     const int brow = PAIR ? (int)rank * 128 : 0;                          // this CTA's share of the Y tile
-    const uint32_t stage_tx = (uint32_t)kABytes + b_bytes;
+    // Tall tiles (one CTA per tile, TN <= 128, K-major X): a stage holds 256 rows of X, fetched by one TMA box, and the
+    // same Y block serves two MMA sets whose accumulators sit 128 TMEM columns apart.  A stage costs its three single
+    // threads about the same whatever it holds, so a narrow product, whose stages carry little, gets twice the rows
+    // out of each.
+    const int tall = PAIR ? 0 : P.tall;
+    const int tmu = TMU << tall;                    // rows of a work unit's tile
+    const int rows_cta = TM << tall;                // ... of which this CTA's
+    const uint32_t a_bytes = (uint32_t)kABytes << tall;
+    const uint32_t stage_tx = a_bytes + b_bytes;
     bool failed = false;
 
     // The three roles below are single threads, and what bounds a pipeline stage is the length of their own
@@ -470,7 +481,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const bool walk = conv == 1 && tiles_j == 1 && P.splits == 1;
             int wk_n = 0, wk_h = 0, wk_w = 0, wk_dn = 0, wk_dh = 0, wk_dw = 0;
             if (walk) {
-                const int first = slot * TMU + (int)rank * TM, step = P.slots * TMU;
+                const int first = slot * tmu + (int)rank * rows_cta, step = P.slots * tmu;
                 wk_n = first / cHW;
                 wk_h = (first - wk_n * cHW) / cW;
                 wk_w = first - wk_n * cHW - wk_h * cW;
@@ -485,7 +496,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const int tile = w.tile;
                 const int ti = tiles_j == 1 ? tile : tile / tiles_j, tj = tile - ti * tiles_j;
                 const int rb0 = w.rb0, nrb = w.rb1 - w.rb0;
-                const int arow = ti * TMU + (int)rank * TM;
+                const int arow = ti * tmu + (int)rank * rows_cta;
                 const int b_row0 = tj * TNv + brow;
                 // Patch gather: pixel block, channel offset and filter tap of the first stage of this unit
                 int g_c = 0, g_w = 0, g_h = 0, g_n = 0, g_ow = 0, g_oh = 0, g_tap = 0, b_tap_red = 0, b_tap_row = 0;
@@ -533,7 +544,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         failed = true;
                         break;
                     }
-                    const uint32_t sa = smem_base + st_off, sb = sa + kABytes, fb = st_bar;
+                    const uint32_t sa = smem_base + st_off, sb = sa + a_bytes, fb = st_bar;
                     st_off += (uint32_t)kStageBytes;
                     st_bar += 8u;
                     if (st_off == kRingBytes) {
@@ -611,7 +622,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of the
             // non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
             const uint64_t a_d0 = P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024);
-            const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + kABytes, 128 * BR, 1024) : make_desc(smem_base + kABytes, 16, 1024);
+            const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + a_bytes, 128 * BR, 1024) : make_desc(smem_base + a_bytes, 16, 1024);
             const uint32_t a_hi = (uint32_t)(a_d0 >> 32), b_hi = (uint32_t)(b_d0 >> 32);
             const uint32_t a_lo0 = (uint32_t)a_d0, b_lo0 = (uint32_t)b_d0;
             const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
@@ -648,7 +659,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         st_par ^= 1u;
                     }
                     if (PAIR) tc_mma4_i8<true>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
-                    else tc_mma4_i8<false>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                    else {
+                        tc_mma4_i8<false>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                        if (tall) tc_mma4_i8<false>(d_tmem + 128u, a_lo + (uint32_t)(kABytes >> 4), a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                    }
                     acc = 1u;
                     // frees the stage (in both CTAs of a pair) once these MMAs have read it
                     if (PAIR) tc_commit_pair(eb);
@@ -756,9 +770,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 break;
             }
             tc_fence_after();
+            for (int sub = 0; sub <= tall; ++sub) {          // the two 128-row halves of a tall tile in turn
             // first output row of this warp; a transposed patch matrix whose taps are padded to 128 channels has
             // rows that exist only in the tiling (never stored) and the others move up
-            int wrow0 = ti * TMU + (int)rank * TM + quarter * 32;
+            int wrow0 = ti * tmu + (int)rank * rows_cta + sub * TM + quarter * 32;
             if (P.conv == 2 && P.cpad != P.cC) {
                 const int tap = wrow0 / P.cpad, c = wrow0 - tap * P.cpad;
                 wrow0 = c < P.cC ? tap * P.cC + c : 0x7fffff00;
@@ -768,7 +783,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const int n = grow / per, rem = grow - n * per, pi = rem / P.sc_Q, qj = rem - pi * P.sc_Q;
                 my_orow = (n * P.sc_H + P.sc_s * pi + P.sc_a) * P.sc_W + P.sc_s * qj + P.sc_b;
             }
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256u + (uint32_t)sub * 128u;
             const int tile_cols = min(P.TN, P.J - tj * P.TN);
             const int nchunks = wrow0 < P.I_out ? (tile_cols + 31) / 32 : 0;   // uniform over the warp
 
@@ -850,6 +865,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         ch += kChunkStep;
                     }
                 }
+            }
             }
             tc_fence_before();
             __syncwarp();
@@ -960,7 +976,7 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 // [N,H,W,C] byte tensor read in im2col mode: one load fetches 128 consecutive base pixels x 128 channel bytes, the
 // base pixels running over the gather's grid (first at the lower corner, `stride` apart), the filter tap given per
 // load as an offset.
-bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g)
+bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g, uint32_t pixels)
 {
     static EncodeIm2colFn fn = nullptr;
     if (fn == nullptr) {
@@ -979,7 +995,7 @@ bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g)
     // last base pixel, relative to the far corner of the tensor
     const int upper[2] = {g.lower_w + (g.Q - 1) * g.stride - (g.W - 1), g.lower_h + (g.P - 1) * g.stride - (g.H - 1)};
     const cuuint32_t estr[4] = {1u, (cuuint32_t)g.stride, (cuuint32_t)g.stride, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, 128u, 128u,
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, 128u, pixels,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -993,16 +1009,18 @@ struct Plan {
     int TN;         // output columns per tile
     int splits;     // parts of the reduced dimension
     int pair;       // 1: CTA pairs on 256-row tiles
-    int tile_rows;  // output rows per work unit (128, or 256 for a pair)
+    int tall;       // 1: one CTA per 256-row tile (narrow outputs, K-major X)
+    int tile_rows;  // output rows per work unit (128, or 256 for a pair or a tall tile)
 };
 
-Plan plan(int I, int J, int R, int min_splits)
+Plan plan(int I, int J, int R, int min_splits, bool x_k_major)
 {
     Plan p;
     p.TN = 256;
     while (p.TN > 16 && p.TN / 2 >= J) p.TN /= 2;
     p.pair = (p.TN == 256 && I > TM) ? 1 : 0;
-    p.tile_rows = p.pair ? 2 * TM : TM;
+    p.tall = (!p.pair && x_k_major && p.TN >= 32 && p.TN <= 128 && I >= 4 * TM) ? 1 : 0;
+    p.tile_rows = (p.pair || p.tall) ? 2 * TM : TM;
     const int slots = p.pair ? kPlanSMs / 2 : kPlanSMs;      // work units that run at once
     const long long tiles = (long long)((I + p.tile_rows - 1) / p.tile_rows) * ((J + p.TN - 1) / p.TN);
     const int rblocks = (R + BR - 1) / BR;
@@ -1033,13 +1051,18 @@ int min_exact_splits(int R, long long xmax, long long ymax)
 // so long that its int32 total could overflow for byte operands of the widest range and it has to be cut).
 size_t tc_gemm_scratch_bytes(int I, int J, int R)
 {
-    Plan p = plan(I, J, R, 1);
     size_t need = 0;
-    if (p.splits > 1) need = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t) * p.splits;
-    if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
-        p = plan(I, J, R, min_exact_splits(R, 255, 128));
-        const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
-        if (slab * p.splits > need) need = slab * p.splits;
+    for (int xk = 0; xk < 2; ++xk) {             // the tiling depends on how the X operand is stored: cover both
+        Plan p = plan(I, J, R, 1, xk != 0);
+        if (p.splits > 1) {
+            const size_t all = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t) * p.splits;
+            if (all > need) need = all;
+        }
+        if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
+            p = plan(I, J, R, min_exact_splits(R, 255, 128), xk != 0);
+            const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
+            if (slab * p.splits > need) need = slab * p.splits;
+        }
     }
     return (need + 255u) & ~(size_t)255u;
 }
@@ -1071,7 +1094,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     // keeps its own slab, and the slabs are summed in int64 (float output only).
     const bool wide = (long long)Rt * X.absmax * Y.absmax >= ((long long)1 << 31);
     if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
-    const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1);
+    const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1, !a_mn);
     const bool want_next = next != nullptr && next->idx_out != nullptr;
     if (want_next && wide) return CDL_ERR_OVERFLOW_RISK;     // the index is taken from one finished accumulator
     const int TN = pl.TN;
@@ -1080,6 +1103,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const int splits = (want_next || scatter) ? 1 : pl.splits;
     const bool pair = pl.pair != 0;
     P.TN = TN;
+    P.tall = pl.tall;
     P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
     // A split reduction with only a float output keeps one slab per split (plain stores, no clear, no atomics in L2)
     // and sums the slabs in the conversion kernel; with compact_scratch (or an int32 output) the splits add into
@@ -1096,7 +1120,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.a_mn_major = a_mn ? 1 : 0;
     P.b_mn_major = b_mn ? 1 : 0;
     P.idesc = (2u << 4) | ((X.is_unsigned ? 0u : 1u) << 7) | ((Y.is_unsigned ? 0u : 1u) << 10) |
-              ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(pl.tile_rows >> 4) << 24);
+              ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)((pl.pair ? 2 * TM : TM) >> 4) << 24);
     P.nq_out = nullptr;
     P.nq_q = P.nq_rq = P.nq_flo = P.nq_fhi = 0.0f;
     P.nq_fast = P.nq_vec = 0;
@@ -1169,9 +1193,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     CUtensorMap map_a, map_b;
     bool ok;
     // K-major operand: stored [outer][r], r contiguous -> inner = r.  MN-major: stored [r][outer] -> inner = outer.
-    if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv);
+    if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv, (uint32_t)(TM << pl.tall));
     else if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
-    else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, TM);
+    else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, (uint32_t)(TM << pl.tall));
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
     else if (conv != nullptr && conv->y_tap_rows > 0)   // all taps' row blocks of the stored matrix, conv->C reduced columns each
         ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->y_rows,
@@ -1230,8 +1254,8 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const int dev_slots = pair ? pair_slots[dev] : sms;
     P.slots = (int)(units < dev_slots ? units : dev_slots);
     // bytes a CTA loads per work unit against the bytes it stores (4-byte outputs of a 128 x TN tile)
-    const long long unit_load = (long long)((P.rblocks + splits - 1) / splits) * (kABytes + (pair ? 128 : TN) * BR);
-    const bool store_heavy = unit_load <= 2ll * TM * TN * 4;
+    const long long unit_load = (long long)((P.rblocks + splits - 1) / splits) * ((kABytes << pl.tall) + (pair ? 128 : TN) * BR);
+    const bool store_heavy = unit_load <= 2ll * (TM << pl.tall) * TN * 4;
     if (pair) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
