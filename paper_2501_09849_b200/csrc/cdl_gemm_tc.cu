@@ -11,8 +11,8 @@
 // In convolution form the X operand is not a stored matrix: its tiles are gathered from an NHWC index tensor by
 // TMA im2col loads (patch matrix of a stride-1 convolution, or its transpose for dW), see ConvGather.
 //
-// Tiling: 128 x TN output tile per work unit (TN in {16..256}), a 256 x TN tile of one CTA when TN <= 128 and X is
-// K-major (one 256-row X box per stage, two accumulators: a narrow product gets twice the rows out of every
+// Tiling: 128 x TN output tile per work unit (TN in {16..256}), a 256 x TN tile of one CTA when TN <= 128
+// (256 rows of X per stage, two accumulators sharing the Y block: a narrow product gets twice the rows out of every
 // pipeline stage), or a 256 x 256 tile shared by a pair of CTAs (tcgen05 cta_group::2) when the output is wide and
 // tall enough; 128 bytes of the reduced dimension per pipeline
 // stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is [rows][128 bytes] with
@@ -473,6 +473,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // pair: both CTAs' bytes are counted on CTA 0's barrier, which CTA 0 arms for the two of them
             const uint32_t arm_tx = PAIR ? 2u * stage_tx : stage_tx;
             const bool arm = do_a && rank == 0;
+            const bool tall2 = tall != 0 && (conv == 2 || (conv == 0 && a_mn != 0));    // X fetched as two boxes per stage
             uint32_t st_off = 0u, st_bar = bar0, st_par = 1u;    // ring position: byte offset, full barrier, parity of "empty"
             // Forward-type patch gathers with one tile column and an unsplit reduction visit tiles slot, slot + slots,
             // ...: the pixel of a tile's first row then moves by a fixed step, kept as (image, row, column) with
@@ -536,6 +537,15 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     b_tap_row = y_tap_rows > 0 ? (int)P.tap_y[g_tap] * y_tap_rows : 0;
                     b_tap_red = y_tap_rows > 0 || conv != 1 ? 0 : g_tap * cC;
                 }
+                // second 128 rows of a tall transposed patch tile: their own tap and channel block
+                int g2_c = 0, g2_ow = 0, g2_oh = 0;
+                if (tall2 && conv == 2) {
+                    const int i1 = arow + TM < P.I ? arow + TM : 0;
+                    const int tap1 = i1 / cpad;
+                    g2_c = i1 - tap1 * cpad;
+                    g2_oh = P.tap_oh[tap1];
+                    g2_ow = P.tap_ow[tap1];
+                }
                 int c_red = rb0 * BR;                            // reduced coordinate of a stored operand
                 int c_w = g_w * c_stride - pad_w, c_h = g_h * c_stride - pad_h;
                 for (int i = 0; i < nrb; ++i) {
@@ -558,6 +568,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                             const int x0 = a_mn ? arow : c_red, x1 = a_mn ? c_red : arow;    // {inner, outer}
                             if (PAIR) tma_load_2d_pair(sa, &map_a, x0, x1, fb);
                             else tma_load_2d(sa, &map_a, x0, x1, fb);
+                            // (an MN-major box is 128 rows of the tile wide: a tall tile takes two)
+                            if (tall2) tma_load_2d(sa + kABytes, &map_a, x0 + TM, x1, fb);
                         }
                         if (do_b) {
                             const int y0 = b_mn ? b_row0 : c_red, y1 = b_mn ? c_red : b_row0;
@@ -572,6 +584,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     if (do_a) {
                         if (PAIR) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
                         else tma_load_im2col(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
+                        if (tall2) tma_load_im2col(sa + kABytes, &map_a, g2_c, c_w, c_h, g_n, g2_ow, g2_oh, fb);
                     }
                     if (do_b) {
                         const int red = conv == 1 ? b_tap_red + g_c : c_red, row = b_row0 + b_tap_row;
@@ -1013,13 +1026,13 @@ struct Plan {
     int tile_rows;  // output rows per work unit (128, or 256 for a pair or a tall tile)
 };
 
-Plan plan(int I, int J, int R, int min_splits, bool x_k_major)
+Plan plan(int I, int J, int R, int min_splits)
 {
     Plan p;
     p.TN = 256;
     while (p.TN > 16 && p.TN / 2 >= J) p.TN /= 2;
     p.pair = (p.TN == 256 && I > TM) ? 1 : 0;
-    p.tall = (!p.pair && x_k_major && p.TN >= 32 && p.TN <= 128 && I >= 4 * TM) ? 1 : 0;
+    p.tall = (!p.pair && p.TN >= 32 && p.TN <= 128 && I >= 4 * TM) ? 1 : 0;
     p.tile_rows = (p.pair || p.tall) ? 2 * TM : TM;
     const int slots = p.pair ? kPlanSMs / 2 : kPlanSMs;      // work units that run at once
     const long long tiles = (long long)((I + p.tile_rows - 1) / p.tile_rows) * ((J + p.TN - 1) / p.TN);
@@ -1051,18 +1064,13 @@ int min_exact_splits(int R, long long xmax, long long ymax)
 // so long that its int32 total could overflow for byte operands of the widest range and it has to be cut).
 size_t tc_gemm_scratch_bytes(int I, int J, int R)
 {
+    Plan p = plan(I, J, R, 1);
     size_t need = 0;
-    for (int xk = 0; xk < 2; ++xk) {             // the tiling depends on how the X operand is stored: cover both
-        Plan p = plan(I, J, R, 1, xk != 0);
-        if (p.splits > 1) {
-            const size_t all = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t) * p.splits;
-            if (all > need) need = all;
-        }
-        if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
-            p = plan(I, J, R, min_exact_splits(R, 255, 128), xk != 0);
-            const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
-            if (slab * p.splits > need) need = slab * p.splits;
-        }
+    if (p.splits > 1) need = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t) * p.splits;
+    if ((long long)R * 255 * 128 >= ((long long)1 << 31)) {
+        p = plan(I, J, R, min_exact_splits(R, 255, 128));
+        const size_t slab = (size_t)((I + p.tile_rows - 1) / p.tile_rows) * p.tile_rows * (size_t)J * sizeof(int32_t);
+        if (slab * p.splits > need) need = slab * p.splits;
     }
     return (need + 255u) & ~(size_t)255u;
 }
@@ -1094,7 +1102,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     // keeps its own slab, and the slabs are summed in int64 (float output only).
     const bool wide = (long long)Rt * X.absmax * Y.absmax >= ((long long)1 << 31);
     if (wide && acc_out != nullptr) return CDL_ERR_OVERFLOW_RISK;
-    const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1, !a_mn);
+    const Plan pl = plan(It, J, Rt, wide ? min_exact_splits(Rt, X.absmax, Y.absmax) : 1);
     const bool want_next = next != nullptr && next->idx_out != nullptr;
     if (want_next && wide) return CDL_ERR_OVERFLOW_RISK;     // the index is taken from one finished accumulator
     const int TN = pl.TN;
@@ -1193,9 +1201,9 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     CUtensorMap map_a, map_b;
     bool ok;
     // K-major operand: stored [outer][r], r contiguous -> inner = r.  MN-major: stored [r][outer] -> inner = outer.
-    if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv, (uint32_t)(TM << pl.tall));
+    if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv, conv->transposed ? (uint32_t)BR : (uint32_t)(TM << pl.tall));
     else if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
-    else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, (uint32_t)(TM << pl.tall));
+    else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, (uint32_t)(TM << pl.tall));     // K-major: one box of the tile's rows
     if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
     else if (conv != nullptr && conv->y_tap_rows > 0)   // all taps' row blocks of the stored matrix, conv->C reduced columns each
         ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->y_rows,
