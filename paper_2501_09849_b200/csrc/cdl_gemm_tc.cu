@@ -377,7 +377,9 @@ __device__ __forceinline__ int next_hard_index(float y, float q, float rq, float
 // what the shared-memory-capacity x latency product of one SM cannot otherwise sustain.  Hand-shake in pair mode:
 // the TMA loads of both CTAs count their bytes on CTA 0's "stage full" barrier; tcgen05.commit multicasts "stage
 // free" and "accumulator full" to both CTAs; the epilogues of both CTAs arrive on CTA 0's "accumulator free" barrier.
-template <bool PAIR, bool STORE_HEAVY>
+// CONV (0 stored X, 1 forward-type gather, 2 transposed gather) is a template argument for the sake of the TMA
+// producers' stage loop: every test of the mode taken out of it shows in the stage time.
+template <bool PAIR, bool STORE_HEAVY, int CONV>
 __global__ void __launch_bounds__(threads_tc(STORE_HEAVY), 1)
 index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_f, const __grid_constant__ CUtensorMap map_acc,
@@ -465,7 +467,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // warp the first issues the X-operand loads and arms the barrier, the second issues the Y-operand loads)
         const bool do_a = warp == 0, do_b = !kSplitProducer || warp != 0;
         if (lane == 0) {
-            const int conv = P.conv, a_mn = P.a_mn_major, b_mn = P.b_mn_major, TNv = P.TN, tiles_j = P.tiles_j;
+            constexpr int conv = CONV;
+            const int a_mn = P.a_mn_major, b_mn = P.b_mn_major, TNv = P.TN, tiles_j = P.tiles_j;
             const int cW = P.cW > 0 ? P.cW : 1, cH = P.cH > 0 ? P.cH : 1, cHW = cH * cW;
             const int cpad = P.cpad, cC = P.cC, c_stride = P.c_stride, pad_w = P.pad_w, pad_h = P.pad_h;
             const int last_tap = P.taps - 1, y_tap_rows = P.y_tap_rows;
@@ -1016,6 +1019,22 @@ bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g, 
 }  // namespace
 
 namespace {
+// The template instance for a launch: CTA pair or single CTA, 16 or 8 epilogue warps, kind of X operand.
+template <bool PAIR, bool STORE_HEAVY>
+const void *kernel_variant_conv(int conv)
+{
+    if (conv == 1) return reinterpret_cast<const void *>(&index_gemm_tc_kernel<PAIR, STORE_HEAVY, 1>);
+    if (conv == 2) return reinterpret_cast<const void *>(&index_gemm_tc_kernel<PAIR, STORE_HEAVY, 2>);
+    return reinterpret_cast<const void *>(&index_gemm_tc_kernel<PAIR, STORE_HEAVY, 0>);
+}
+const void *kernel_variant(bool pair, bool store_heavy, int conv)
+{
+    if (pair) return store_heavy ? kernel_variant_conv<true, true>(conv) : kernel_variant_conv<true, false>(conv);
+    return store_heavy ? kernel_variant_conv<false, true>(conv) : kernel_variant_conv<false, false>(conv);
+}
+}  // namespace
+
+namespace {
 // Split of the reduced dimension: when the tiles alone cannot occupy half of the device, and always into at
 // least min_splits parts (the caller's bound that keeps every part's int32 partial sums exact).
 struct Plan {
@@ -1232,12 +1251,11 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return CDL_ERR_LAUNCH;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(index_gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(index_gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(index_gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(index_gemm_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return CDL_ERR_LAUNCH;
+        for (int v = 0; v < 12; ++v) {
+            if (cudaFuncSetAttribute(kernel_variant((v & 1) != 0, (v & 2) != 0, v >> 2), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return CDL_ERR_LAUNCH;
+            }
         }
         cudaLaunchConfig_t qc = {};
         cudaLaunchAttribute qa[1];
@@ -1251,7 +1269,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         qc.attrs = qa;
         qc.numAttrs = 1;
         int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, index_gemm_tc_kernel<true, false>, &qc) != cudaSuccess || nclusters < 1) {
+        if (cudaOccupancyMaxActiveClusters(&nclusters, kernel_variant(true, false, 0), &qc) != cudaSuccess || nclusters < 1) {
             (void)cudaGetLastError();
             nclusters = sms / 2;
         }
@@ -1264,28 +1282,24 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     // bytes a CTA loads per work unit against the bytes it stores (4-byte outputs of a 128 x TN tile)
     const long long unit_load = (long long)((P.rblocks + splits - 1) / splits) * ((kABytes << pl.tall) + (pair ? 128 : TN) * BR);
     const bool store_heavy = unit_load <= 2ll * (TM << pl.tall) * TN * 4;
-    if (pair) {
+    {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2;
         at[0].val.clusterDim.y = 1;
         at[0].val.clusterDim.z = 1;
-        cfg.gridDim = dim3(2u * (unsigned)P.slots);
+        cfg.gridDim = dim3(pair ? 2u * (unsigned)P.slots : (unsigned)P.slots);
         cfg.blockDim = dim3(threads_tc(store_heavy));
         cfg.dynamicSmemBytes = kSmemBytes;
         cfg.stream = stream;
         cfg.attrs = at;
-        cfg.numAttrs = 1;
-        const cudaError_t le = store_heavy ? cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true, true>, map_a, map_b, map_f, map_acc, P)
-                                           : cudaLaunchKernelEx(&cfg, index_gemm_tc_kernel<true, false>, map_a, map_b, map_f, map_acc, P);
-        if (le != cudaSuccess) {
+        cfg.numAttrs = pair ? 1 : 0;
+        void *args[5] = {&map_a, &map_b, &map_f, &map_acc, &P};
+        if (cudaLaunchKernelExC(&cfg, kernel_variant(pair, store_heavy, P.conv), args) != cudaSuccess) {
             (void)cudaGetLastError();
             return CDL_ERR_LAUNCH;
         }
-    } else {
-        if (store_heavy) index_gemm_tc_kernel<false, true><<<P.slots, threads_tc(true), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
-        else index_gemm_tc_kernel<false, false><<<P.slots, threads_tc(false), kSmemBytes, stream>>>(map_a, map_b, map_f, map_acc, P);
     }
     if (cudaGetLastError() != cudaSuccess) return CDL_ERR_LAUNCH;
     if (f_out != nullptr && (splits > 1 || slabs)) {
