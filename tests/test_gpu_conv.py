@@ -130,6 +130,8 @@ def test_resnet_layer1_geometry_sampled(torch):
     (2, 10, 10, 64, 128, 4, 4, 2, 1, 1),
     (2, 13, 13, 128, 128, 3, 3, 3, 1, 1),     # stride 3: nine pixel classes
     (1, 17, 9, 64, 64, 5, 3, 4, 2, 0),        # stride 4, unequal padding
+    (8, 24, 24, 64, 128, 3, 3, 2, 1, 1),      # large enough for 256-row tiles: scattered rows of the four classes, dW
+    (9, 23, 25, 128, 64, 1, 1, 2, 0, 0),      # the same for the shortcut, ragged in every dimension
 ])
 def test_strided_convolutions(torch, N, H, W, C, CO, R, S, stride, ph, pw):
     X, Wt, G = make(40 + H + R + stride, N, H, W, C, CO, R, S, stride=stride, ph=ph, pw=pw)

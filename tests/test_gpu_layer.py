@@ -121,7 +121,11 @@ def test_tiny_layer_products_from_quantized_tensors(torch):
 
 
 @pytest.mark.parametrize("M,K,N", [(1, 16, 16), (5, 20, 7), (130, 147, 64), (257, 144, 16), (300, 520, 130),
-                                   (64, 2304, 256), (1000, 64, 1000)])
+                                   (64, 2304, 256), (1000, 64, 1000),
+                                   # 256-row tiles of one CTA (at most 128 output columns, at least 512 rows), ragged
+                                   # in every dimension: forward and dW of the first, forward of the other two, and
+                                   # dX / dW of the last (640 and 1152 rows of the transposed operand)
+                                   (1000, 640, 64), (2048 + 77, 200, 128), (700, 1152, 96)])
 def test_ragged_shapes_and_signedness(torch, M, K, N):
     for a_lo, a_hi in ((0, 255), (-128, 127), (0, 15)):
         A = inputs.uniform_indices((M, K), a_lo, a_hi, seed=M + K)

@@ -30,7 +30,8 @@ def ref_index(acc, qa, qw, bias, nq, lo, hi):
 
 
 @pytest.mark.parametrize("M,K,N,lo,hi", [(300, 520, 256, 0, 15), (130, 144, 48, -7, 7), (64, 256, 128, 0, 255),
-                                         (257, 160, 20, 0, 15)])
+                                         (257, 160, 20, 0, 15),
+                                         (900, 320, 64, 0, 15), (1300, 144, 112, -7, 7)])    # 256-row tiles of one CTA
 def test_linear_forward_emits_the_next_layers_index(torch, M, K, N, lo, hi):
     rng = np.random.default_rng(M + N)
     A = rng.integers(0, 16, (M, K)).astype(np.uint8)
