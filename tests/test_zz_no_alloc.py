@@ -21,8 +21,9 @@ def test_noalloc_dw_matches_regular_entry_point_twice_in_a_row():
     import torch
     cdl.load_library()
     a, g = cdl.IndexDesc(0.25, 0, 15), cdl.IndexDesc(1e-3, -127, 127)
-    # (M, K, N): a split reduction (few output tiles, long M), a ragged one, and a single-split one
-    for call, (M, K, N) in enumerate([(4096, 256, 128), (3000, 144, 16), (300, 640, 256)]):
+    # (M, K, N): a split reduction (few output tiles, long M), a ragged one, a single-split one, and one whose
+    # output is tiled in 256-row blocks of one CTA (at most 128 columns, 640 rows)
+    for call, (M, K, N) in enumerate([(4096, 256, 128), (3000, 144, 16), (300, 640, 256), (2000, 640, 64)]):
         A = torch.from_numpy(inputs.uniform_indices((M, K), 0, 15, seed=40 + call)).cuda()
         G = torch.from_numpy(inputs.uniform_indices((M, N), -127, 127, seed=50 + call)).cuda()
         nb = cdl.cdl_workspace_bytes(cdl.CDL_OP_QLINEAR_BWD, M, N, K)
