@@ -111,6 +111,7 @@ struct TcParams {
                             // [s * slab_rows, ...) of a (splits * slab_rows) x J buffer, summed in int64 afterwards
     int slots;              // work slots (CTA pairs, or CTAs) = the grid: slot p takes units p, p + slots, ...
     int tall;               // 1: a CTA's tile is 256 rows x TN (TN <= 128): one 256-row X box per stage, two accumulators
+    int k64;                // 1: forward-type gather of 64 channels per tap: X rows are 64 bytes (64-byte swizzle), two MMAs per stage
 };
 
 // One piece of work of a slot: pipeline stages [rb0, rb1) of a tile (a unit of tiles * splits).
@@ -313,6 +314,38 @@ __device__ __forceinline__ void tc_mma4_i8(uint32_t d_tmem, uint32_t a_lo, uint3
     }
 }
 
+// Two MMAs (K = 32 each) of a stage that holds 64 bytes of r.
+template <bool PAIR>
+__device__ __forceinline__ void tc_mma2_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t a_step, uint32_t b_lo,
+                                           uint32_t b_hi, uint32_t b_step, uint32_t idesc, uint32_t accumulate)
+{
+    if (PAIR) {
+        asm volatile(
+            "{\n\t.reg .pred p, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+            "setp.ne.b32 p, %8, 0;\n\t"
+            "setp.eq.b32 t, 0, 0;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%4, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, p;\n\t"
+            "add.u32 al, %1, %3;\n\tadd.u32 bl, %4, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9, %9, %9, %9, %9}, t;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+            "setp.ne.b32 p, %8, 0;\n\t"
+            "setp.eq.b32 t, 0, 0;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%4, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, p;\n\t"
+            "add.u32 al, %1, %3;\n\tadd.u32 bl, %4, %6;\n\t"
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %7, {%9, %9, %9, %9}, t;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(a_step), "r"(b_lo), "r"(b_hi), "r"(b_step), "r"(idesc), "r"(accumulate), "r"(0u)
+            : "memory");
+    }
+}
+
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
 {
     asm volatile(
@@ -352,6 +385,18 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
     d |= (uint64_t)1 << 46;   // descriptor version for sm_100
     d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+// The same for a K-major block whose rows are 64 bytes (64-byte swizzle): 8-row groups sbo_bytes = 512 apart.
+__device__ __forceinline__ uint64_t make_desc64(uint32_t saddr, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;       // leading offset: not used by a swizzled K-major block narrower than the swizzle span
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version for sm_100
+    d |= (uint64_t)4 << 61;   // SWIZZLE_64B
     return d;
 }
 
@@ -451,7 +496,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const int tmu = TMU << tall;                    // rows of a work unit's tile
     const int rows_cta = TM << tall;                // ... of which this CTA's
     const uint32_t a_bytes = (uint32_t)kABytes << tall;
-    const uint32_t stage_tx = a_bytes + b_bytes;
+    // a 64-channel tap fills half of the X block: rows of 64 bytes, 8 KB per 128 rows (the Y block keeps its place)
+    const uint32_t stage_tx = (P.k64 ? a_bytes >> 1 : a_bytes) + b_bytes;
     bool failed = false;
 
     // The three roles below are single threads, and what bounds a pipeline stage is the length of their own
@@ -637,7 +683,9 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // K-major: rows are 128-byte lines, 8-row groups 1024 bytes apart, 32 bytes per MMA along r.
             // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of the
             // non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
-            const uint64_t a_d0 = P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024);
+            const uint64_t a_d0 = P.k64 ? make_desc64(smem_base, 512) : (P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024));
+            const int k64 = P.k64;
+            const uint32_t a_sub16 = (uint32_t)((k64 ? kABytes / 2 : kABytes) >> 4);      // 128 rows further on, in 16-byte units
             const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + a_bytes, 128 * BR, 1024) : make_desc(smem_base + a_bytes, 16, 1024);
             const uint32_t a_hi = (uint32_t)(a_d0 >> 32), b_hi = (uint32_t)(b_d0 >> 32);
             const uint32_t a_lo0 = (uint32_t)a_d0, b_lo0 = (uint32_t)b_d0;
@@ -674,10 +722,16 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                         st_bar = bar0;
                         st_par ^= 1u;
                     }
-                    if (PAIR) tc_mma4_i8<true>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                    if (k64) {          // 64 bytes of r per stage: two MMAs per 128-row block
+                        if (PAIR) tc_mma2_i8<true>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                        else {
+                            tc_mma2_i8<false>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                            if (tall) tc_mma2_i8<false>(d_tmem + 128u, a_lo + a_sub16, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                        }
+                    } else if (PAIR) tc_mma4_i8<true>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
                     else {
                         tc_mma4_i8<false>(d_tmem, a_lo, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
-                        if (tall) tc_mma4_i8<false>(d_tmem + 128u, a_lo + (uint32_t)(kABytes >> 4), a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
+                        if (tall) tc_mma4_i8<false>(d_tmem + 128u, a_lo + a_sub16, a_hi, a_step, b_lo, b_hi, b_step, idesc, acc);
                     }
                     acc = 1u;
                     // frees the stage (in both CTAs of a pair) once these MMAs have read it
@@ -994,6 +1048,7 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 // load as an offset.
 bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g, uint32_t pixels)
 {
+    const bool k64 = !g.transposed && g.C == 64;      // 64-channel taps: rows of 64 bytes, 64-byte swizzle
     static EncodeIm2colFn fn = nullptr;
     if (fn == nullptr) {
         void *p = nullptr;
@@ -1011,8 +1066,8 @@ bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g, 
     // last base pixel, relative to the far corner of the tensor
     const int upper[2] = {g.lower_w + (g.Q - 1) * g.stride - (g.W - 1), g.lower_h + (g.P - 1) * g.stride - (g.H - 1)};
     const cuuint32_t estr[4] = {1u, (cuuint32_t)g.stride, (cuuint32_t)g.stride, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, 128u, pixels,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper, k64 ? 64u : 128u, pixels,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, k64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1131,6 +1186,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     const bool pair = pl.pair != 0;
     P.TN = TN;
     P.tall = pl.tall;
+    P.k64 = (conv != nullptr && !conv->transposed && conv->C == 64) ? 1 : 0;
     P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
     // A split reduction with only a float output keeps one slab per split (plain stores, no clear, no atomics in L2)
     // and sums the slabs in the conversion kernel; with compact_scratch (or an int32 output) the splits add into

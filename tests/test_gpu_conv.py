@@ -106,7 +106,8 @@ def test_resnet_layer_geometry_14x14(torch):
     run_all(torch, X, Wt, G, 3, 3)
 
 
-@pytest.mark.parametrize("C,CO", [(64, 64), (64, 128), (192, 64), (128, 192), (320, 256)])
+@pytest.mark.parametrize("C,CO", [(64, 64), (64, 128), (192, 64), (128, 192), (320, 256),
+                                  (64, 256), (256, 64)])     # 64-byte rows of X under a CTA pair: forward, and dX
 def test_channel_counts_that_are_not_multiples_of_128(torch, C, CO):
     # a tap then fills its last 128-channel block only partly: the missing channels read as zero
     X, Wt, G = make(20 + C + CO, 3, 9, 10, C, CO, 3, 3)
