@@ -485,8 +485,10 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const uint32_t tmem_base = tmem_base_s;
 
     const int b_blocks = PAIR ? 1 : (P.TN + 127) / 128;                   // 128-wide blocks of an MN-major B tile
-    const uint32_t b_bytes = PAIR ? (uint32_t)(128 * BR)
-                                  : (P.b_mn_major ? (uint32_t)(b_blocks * 128 * BR) : (uint32_t)(P.TN * BR));
+    // (an MN-major Y block of a 64-channel tap holds the tap's 64 r-rows only)
+    const uint32_t b_rrows = (P.k64 && P.b_mn_major) ? 64u : (uint32_t)BR;
+    const uint32_t b_bytes = P.b_mn_major ? (uint32_t)b_blocks * 128u * b_rrows
+                                          : (uint32_t)(PAIR ? 128 : P.TN) * (P.k64 ? 64u : (uint32_t)BR);     // (K-major: 64-byte rows as well)
     const int brow = PAIR ? (int)rank * 128 : 0;                          // this CTA's share of the Y tile
     // Tall tiles (one CTA per tile, TN <= 128, K-major X): a stage holds 256 rows of X, fetched by one TMA box, and the
     // same Y block serves two MMA sets whose accumulators sit 128 TMEM columns apart.  A stage costs its three single
@@ -686,7 +688,8 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint64_t a_d0 = P.k64 ? make_desc64(smem_base, 512) : (P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024));
             const int k64 = P.k64;
             const uint32_t a_sub16 = (uint32_t)((k64 ? kABytes / 2 : kABytes) >> 4);      // 128 rows further on, in 16-byte units
-            const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + a_bytes, 128 * BR, 1024) : make_desc(smem_base + a_bytes, 16, 1024);
+            const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + a_bytes, 128 * BR, 1024)
+                                               : (P.k64 ? make_desc64(smem_base + a_bytes, 512) : make_desc(smem_base + a_bytes, 16, 1024));
             const uint32_t a_hi = (uint32_t)(a_d0 >> 32), b_hi = (uint32_t)(b_d0 >> 32);
             const uint32_t a_lo0 = (uint32_t)a_d0, b_lo0 = (uint32_t)b_d0;
             const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
@@ -1025,16 +1028,17 @@ bool encode_out_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t 
 }
 
 // 2D byte tensor [outer][inner] with row pitch `pitch` bytes; box = {128 bytes, box_rows}, 128-byte swizzle.
-bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t pitch, uint32_t box_rows)
+bool encode_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t pitch, uint32_t box_rows,
+                bool rows64 = false)      // rows64: boxes of 64-byte rows under the 64-byte swizzle
 {
     EncodeTiledFn fn = get_encode();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {inner, outer};
     const cuuint64_t strides[1] = {pitch};
-    const cuuint32_t box[2] = {128u, box_rows};
+    const cuuint32_t box[2] = {rows64 ? 64u : 128u, box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1279,11 +1283,11 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     if (conv != nullptr) ok = encode_im2col_map(&map_a, X.ptr, *conv, conv->transposed ? (uint32_t)BR : (uint32_t)(TM << pl.tall));
     else if (a_mn) ok = encode_map(&map_a, X.ptr, (uint64_t)I, (uint64_t)R, (uint64_t)X.stride_red, BR);
     else ok = encode_map(&map_a, X.ptr, (uint64_t)R, (uint64_t)I, (uint64_t)X.stride_outer, (uint32_t)(TM << pl.tall));     // K-major: one box of the tile's rows
-    if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, BR);
+    if (b_mn) ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)J, (uint64_t)R, (uint64_t)Y.stride_red, P.k64 ? 64u : (uint32_t)BR);
     else if (conv != nullptr && conv->y_tap_rows > 0)   // all taps' row blocks of the stored matrix, conv->C reduced columns each
         ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)conv->C, (uint64_t)conv->y_rows,
-                              (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
-    else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN);
+                              (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN, P.k64 != 0);
+    else ok = ok && encode_map(&map_b, Y.ptr, (uint64_t)R, (uint64_t)J, (uint64_t)Y.stride_outer, pair ? 128u : (uint32_t)TN, P.k64 != 0);
     // outputs through shared memory + TMA when their pitch and base allow it and the tile is at least one box wide
     CUtensorMap map_f = map_a, map_acc = map_a;      // placeholders when unused
     const bool out_ok = TN >= 32 && (J & 3) == 0 && !scatter;      // scattered rows are copied out by the warps
