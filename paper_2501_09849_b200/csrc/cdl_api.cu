@@ -532,7 +532,7 @@ size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
     const int cp = (shape->C + 127) / 128 * 128, cop = (C_out + 127) / 128 * 128;
     const size_t f = tc_gemm_scratch_bytes((int)g.M_out, C_out, g.taps * cp);
     const size_t dx = g.stride == 1 ? tc_gemm_scratch_bytes((int)g.M_in, shape->C, g.taps * cop) : 0;   // (strided: no split)
-    const size_t dw = tc_gemm_scratch_bytes(g.taps * cp, C_out, (int)g.M_out);
+    const size_t dw = tc_gemm_scratch_bytes(g.taps * (shape->C == 64 ? 64 : cp), C_out, (int)g.M_out);     // (64-channel taps: no padding)
     size_t m = f > dx ? f : dx;
     if (dw > m) m = dw;
     return kStatusBytes + m;

@@ -112,6 +112,8 @@ struct TcParams {
     int slots;              // work slots (CTA pairs, or CTAs) = the grid: slot p takes units p, p + slots, ...
     int tall;               // 1: a CTA's tile is 256 rows x TN (TN <= 128): one 256-row X box per stage, two accumulators
     int k64;                // 1: forward-type gather of 64 channels per tap: X rows are 64 bytes (64-byte swizzle), two MMAs per stage
+    int k64t;               // 1: transposed gather of 64 channels per tap: 64 tile rows per tap (no padding to 128), X boxes of
+                            //    64 channels x 128 pixels under the 64-byte swizzle, two per 128 tile rows
 };
 
 // One piece of work of a slot: pipeline stages [rb0, rb1) of a tile (a unit of tiles * splits).
@@ -400,6 +402,19 @@ __device__ __forceinline__ uint64_t make_desc64(uint32_t saddr, uint32_t sbo_byt
     return d;
 }
 
+// MN-major block of 64-byte lines (64-byte swizzle): r-rows are 64-byte lines, 8-row groups sbo_bytes = 512 apart,
+// 64-wide blocks of the non-reduced dimension lbo_bytes apart.
+__device__ __forceinline__ uint64_t make_desc64_mn(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fffu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version for sm_100
+    d |= (uint64_t)4 << 61;   // SWIZZLE_64B
+    return d;
+}
+
 // clamp(rint(y / q), lo, hi) exactly as the quantizer kernels compute it: reciprocal product, rounding by adding
 // 1.5 * 2^23, and the IEEE quotient itself whenever the product lies within 2^-12 of a half-integer (the product
 // is within 3 ulp of the quotient and indices are at most 255).  A NaN clamps to lo.
@@ -499,6 +514,7 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const int rows_cta = TM << tall;                // ... of which this CTA's
     const uint32_t a_bytes = (uint32_t)kABytes << tall;
     // a 64-channel tap fills half of the X block: rows of 64 bytes, 8 KB per 128 rows (the Y block keeps its place)
+    // (a transposed 64-channel gather fills its block: two boxes of 64 channels x 128 pixels per 128 tile rows)
     const uint32_t stage_tx = (P.k64 ? a_bytes >> 1 : a_bytes) + b_bytes;
     bool failed = false;
 
@@ -525,6 +541,9 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint32_t arm_tx = PAIR ? 2u * stage_tx : stage_tx;
             const bool arm = do_a && rank == 0;
             const bool tall2 = tall != 0 && (conv == 2 || (conv == 0 && a_mn != 0));    // X fetched as two boxes per stage
+            // boxes of a transposed patch tile
+            const int t_box_rows = P.k64t ? 64 : TM, t_nbox = rows_cta / t_box_rows;
+            const uint32_t t_box_bytes = (uint32_t)t_box_rows * BR;
             uint32_t st_off = 0u, st_bar = bar0, st_par = 1u;    // ring position: byte offset, full barrier, parity of "empty"
             // Forward-type patch gathers with one tile column and an unsplit reduction visit tiles slot, slot + slots,
             // ...: the pixel of a tile's first row then moves by a fixed step, kept as (image, row, column) with
@@ -588,14 +607,20 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     b_tap_row = y_tap_rows > 0 ? (int)P.tap_y[g_tap] * y_tap_rows : 0;
                     b_tap_red = y_tap_rows > 0 || conv != 1 ? 0 : g_tap * cC;
                 }
-                // second 128 rows of a tall transposed patch tile: their own tap and channel block
-                int g2_c = 0, g2_ow = 0, g2_oh = 0;
-                if (tall2 && conv == 2) {
-                    const int i1 = arow + TM < P.I ? arow + TM : 0;
-                    const int tap1 = i1 / cpad;
-                    g2_c = i1 - tap1 * cpad;
-                    g2_oh = P.tap_oh[tap1];
-                    g2_ow = P.tap_ow[tap1];
+                // further boxes of a transposed patch tile (128 tile rows each, or 64 for 64-channel taps): their own tap
+                // and channel block
+                int gx_c[3] = {0, 0, 0}, gx_ow[3] = {0, 0, 0}, gx_oh[3] = {0, 0, 0};
+                if (conv == 2) {
+#pragma unroll
+                    for (int b = 1; b < 4; ++b) {           // (constant indices: the arrays stay in registers)
+                        if (b < t_nbox) {
+                            const int i1 = arow + b * t_box_rows < P.I ? arow + b * t_box_rows : 0;
+                            const int tap1 = i1 / cpad;
+                            gx_c[b - 1] = i1 - tap1 * cpad;
+                            gx_oh[b - 1] = P.tap_oh[tap1];
+                            gx_ow[b - 1] = P.tap_ow[tap1];
+                        }
+                    }
                 }
                 int c_red = rb0 * BR;                            // reduced coordinate of a stored operand
                 int c_w = g_w * c_stride - pad_w, c_h = g_h * c_stride - pad_h;
@@ -635,7 +660,14 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     if (do_a) {
                         if (PAIR) tma_load_im2col_pair(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
                         else tma_load_im2col(sa, &map_a, g_c, c_w, c_h, g_n, g_ow, g_oh, fb);
-                        if (tall2) tma_load_im2col(sa + kABytes, &map_a, g2_c, c_w, c_h, g_n, g2_ow, g2_oh, fb);
+                        if (conv == 2) {
+#pragma unroll
+                            for (int b = 1; b < 4; ++b)
+                                if (b < t_nbox) {
+                                    if (PAIR) tma_load_im2col_pair(sa + (uint32_t)b * t_box_bytes, &map_a, gx_c[b - 1], c_w, c_h, g_n, gx_ow[b - 1], gx_oh[b - 1], fb);
+                                    else tma_load_im2col(sa + (uint32_t)b * t_box_bytes, &map_a, gx_c[b - 1], c_w, c_h, g_n, gx_ow[b - 1], gx_oh[b - 1], fb);
+                                }
+                        }
                     }
                     if (do_b) {
                         const int red = conv == 1 ? b_tap_red + g_c : c_red, row = b_row0 + b_tap_row;
@@ -685,14 +717,16 @@ index_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // K-major: rows are 128-byte lines, 8-row groups 1024 bytes apart, 32 bytes per MMA along r.
             // MN-major: r-rows are 128-byte lines, 8-row groups 1024 bytes apart (SBO), 128-wide blocks of the
             // non-reduced dimension BR * 128 bytes apart (LBO), 32 r-rows = 4096 bytes per MMA.
-            const uint64_t a_d0 = P.k64 ? make_desc64(smem_base, 512) : (P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024));
+            const uint64_t a_d0 = P.k64 ? make_desc64(smem_base, 512)
+                                        : (P.k64t ? make_desc64_mn(smem_base, 64 * BR, 512)
+                                                  : (P.a_mn_major ? make_desc(smem_base, 128 * BR, 1024) : make_desc(smem_base, 16, 1024)));
             const int k64 = P.k64;
             const uint32_t a_sub16 = (uint32_t)((k64 ? kABytes / 2 : kABytes) >> 4);      // 128 rows further on, in 16-byte units
             const uint64_t b_d0 = P.b_mn_major ? make_desc(smem_base + a_bytes, 128 * BR, 1024)
                                                : (P.k64 ? make_desc64(smem_base + a_bytes, 512) : make_desc(smem_base + a_bytes, 16, 1024));
             const uint32_t a_hi = (uint32_t)(a_d0 >> 32), b_hi = (uint32_t)(b_d0 >> 32);
             const uint32_t a_lo0 = (uint32_t)a_d0, b_lo0 = (uint32_t)b_d0;
-            const uint32_t a_step = P.a_mn_major ? (4096u >> 4) : (32u >> 4);
+            const uint32_t a_step = P.k64t ? (2048u >> 4) : (P.a_mn_major ? (4096u >> 4) : (32u >> 4));      // 32 r-rows, or 32 bytes of r
             const uint32_t b_step = P.b_mn_major ? (4096u >> 4) : (32u >> 4);
             const uint32_t idesc = P.idesc;
             uint32_t tcount = 0;
@@ -1052,7 +1086,7 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 // load as an offset.
 bool encode_im2col_map(CUtensorMap *map, const void *base, const ConvGather &g, uint32_t pixels)
 {
-    const bool k64 = !g.transposed && g.C == 64;      // 64-channel taps: rows of 64 bytes, 64-byte swizzle
+    const bool k64 = g.C == 64;      // 64-channel taps: boxes 64 channels wide, 64-byte swizzle
     static EncodeIm2colFn fn = nullptr;
     if (fn == nullptr) {
         void *p = nullptr;
@@ -1167,7 +1201,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     int It = I, Rt = R;
     if (conv != nullptr) {
         const int cpad = (conv->C + BR - 1) / BR * BR;
-        if (conv->transposed) It = conv->taps * cpad;
+        if (conv->transposed) It = conv->taps * (conv->C == 64 ? 64 : cpad);     // (64-channel taps are not padded)
         else Rt = conv->taps * cpad;
     }
     TcParams P;
@@ -1191,6 +1225,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
     P.TN = TN;
     P.tall = pl.tall;
     P.k64 = (conv != nullptr && !conv->transposed && conv->C == 64) ? 1 : 0;
+    P.k64t = (conv != nullptr && conv->transposed && conv->C == 64) ? 1 : 0;
     P.tiles_i = (It + pl.tile_rows - 1) / pl.tile_rows;
     // A split reduction with only a float output keeps one slab per split (plain stores, no clear, no atomics in L2)
     // and sums the slabs in the conversion kernel; with compact_scratch (or an int32 output) the splits add into
@@ -1234,7 +1269,7 @@ int launch_index_gemm_tc(const GemmOperand &X, const GemmOperand &Y, int I, int 
         P.cW = conv->Q;
         P.cC = conv->C;
         P.cblocks = (conv->C + BR - 1) / BR;
-        P.cpad = P.cblocks * BR;
+        P.cpad = P.k64t ? 64 : P.cblocks * BR;
         P.pad_h = -conv->lower_h;
         P.pad_w = -conv->lower_w;
         P.c_stride = conv->stride;
