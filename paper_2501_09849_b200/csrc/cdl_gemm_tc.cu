@@ -9,15 +9,18 @@
 //   dW       dW = A^T G    X = A [M,K] (i = k contiguous: MN-major)  Y-op = G [M,N] (j contiguous: MN-major)
 //
 // In convolution form the X operand is not a stored matrix: its tiles are gathered from an NHWC index tensor by
-// TMA im2col loads (patch matrix of a stride-1 convolution, or its transpose for dW), see ConvGather.
+// TMA im2col loads (patch matrix of a convolution, or its transpose for dW), see ConvGather.  The kind of X operand
+// is a template argument (the producers' stage loop tests nothing about it).
 //
 // Tiling: 128 x TN output tile per work unit (TN in {16..256}), a 256 x TN tile of one CTA when TN <= 128
 // (256 rows of X per stage, two accumulators sharing the Y block: a narrow product gets twice the rows out of every
 // pipeline stage), or a 256 x 256 tile shared by a pair of CTAs (tcgen05 cta_group::2) when the output is wide and
-// tall enough; 128 bytes of the reduced dimension per pipeline
-// stage, four tcgen05.mma (K = 32 each) per stage.  Every shared-memory operand block is [rows][128 bytes] with
-// the 128-byte swizzle, written by TMA boxes whose inner extent is 128 bytes; rows or columns outside the matrix
-// are zero-filled by TMA, which makes ragged edges and R tails exact.
+// tall enough; 128 bytes of the reduced dimension per pipeline stage, four tcgen05.mma (K = 32 each) per stage.
+// Every shared-memory operand block is [rows][128 bytes] with the 128-byte swizzle, written by TMA boxes whose inner
+// extent is 128 bytes; rows or columns outside the matrix are zero-filled by TMA, which makes ragged edges and R
+// tails exact.  A convolution with 64 channels per filter tap would fill only half of such rows: its gathered
+// blocks are 64 bytes wide under the 64-byte swizzle instead (K-major rows of 64 bytes and two MMAs per stage for
+// forward and dX; MN-major boxes of 64 channels, two per 128 tile rows, for dW).
 // Warp roles: warp 0 and the last warp issue TMA (X and Y operand), warp 1 owns TMEM and issues the MMAs, the
 // 8 (or, for products that store more than they load, 16) warps between them run the epilogue; two TMEM
 // accumulators let the epilogue of one tile overlap the MMAs of the next.
