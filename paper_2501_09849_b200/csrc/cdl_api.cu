@@ -528,7 +528,7 @@ size_t cdl_qconv_workspace_bytes(const cdl_conv_shape *shape, int32_t C_out)
 {
     ConvGeo g;
     if (!conv_geo(shape, C_out, &g)) return 0;
-    // the tiling pads every tap to whole 128-channel blocks
+    // the tiling pads every tap to whole 128-channel blocks (except the transposed gather of 64-channel taps)
     const int cp = (shape->C + 127) / 128 * 128, cop = (C_out + 127) / 128 * 128;
     const size_t f = tc_gemm_scratch_bytes((int)g.M_out, C_out, g.taps * cp);
     const size_t dx = g.stride == 1 ? tc_gemm_scratch_bytes((int)g.M_in, shape->C, g.taps * cop) : 0;   // (strided: no split)
