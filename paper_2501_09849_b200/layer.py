@@ -120,12 +120,19 @@ class CdlLayerStep:
 
     def run_forked(self):
         """The same ten calls as run(), issued on the current stream and two helper streams along the step's data
-        dependencies:
-            current:  quantize w -> forward -> dA -> dW -> quantizer backward on w
+        dependencies.  Stored-matrix form:
+            current:  dW -> forward -> dA                       (the three products, back to back)
             second:   quantize x -> entropy of x -> quantizer backward on x
+            third:    quantize dL/dY -> quantize w -> entropy of w -> quantizer backward on w
+        dW needs G_idx but not W_idx, so it goes first and the weight passes leave the chain of the products (the
+        forward product needs W_idx, dA needs G_idx and W_idx, the backward pass on w needs dW and the level
+        probabilities of w and runs beside the other two products).  Convolution form, where the forward product
+        and dW read X_idx and the activation quantizer's backward pass reads dA:
+            current:  quantize w -> forward -> dA -> dW -> quantizer backward on w
+            second:   quantize x -> entropy of x -> (after dA) quantizer backward on x
             third:    quantize dL/dY ;  entropy of w
-        The forward product needs W_idx; dA needs G_idx and W_idx; dW needs G_idx; the backward pass on w needs dW
-        and the level probabilities of w.  All helper work is joined back into the current stream at the end."""
+        Both orders were measured against the alternatives on the benchmark layer; all helper work is joined back
+        into the current stream at the end."""
         t = self.torch
         if not hasattr(self, "_helpers"):
             self._helpers = (t.cuda.Stream(), t.cuda.Stream())
@@ -142,34 +149,47 @@ class CdlLayerStep:
         fork = after(s0)
         s1.wait_event(fork)
         s2.wait_event(fork)
-        # second stream: everything on the activation tensor (in the convolution form its backward pass waits
-        # for the data gradient, see below)
+        # second stream: everything on the activation tensor
         cdl.cdl_quantize_soft(self.x, self.n_x, self.Px, self.x_soft, self.X_idx, self.hist_x, s1)
         x_ready = after(s1)
         cdl.cdl_index_entropy(self.hist_x, nlx, sc[1:2], self.prob_x, None, s1)
         if self.conv is None:
             cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
-        # third stream: gradient indices
-        cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, s2)
-        g_ready = after(s2)
-        # current stream: weights, then the three products
-        cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, s0)
-        w_ready = after(s0)
-        s2.wait_event(w_ready)
-        cdl.cdl_index_entropy(self.hist_w, nlw, sc[0:1], self.prob_w, None, s2)
-        pw_ready = after(s2)
-        if self.conv is not None:
+            # third stream: gradient indices first (dW waits for them), then the weights
+            cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, s2)
+            g_ready = after(s2)
+            cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, s2)
+            w_ready = after(s2)
+            cdl.cdl_index_entropy(self.hist_w, nlw, sc[0:1], self.prob_w, None, s2)
+            # current stream: the three products
+            s0.wait_event(g_ready)
+            self._bwd_dw(s0)
+            dw_ready = after(s0)
+            s0.wait_event(w_ready)
+            self._fwd(s0)
+            self._bwd_dx(s0)
+            s2.wait_event(dw_ready)
+            cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, sc[2:3], sc[3:4], s2)
+        else:
+            # third stream: gradient indices
+            cdl.cdl_quantize_hard(self.dY, M * N, self.Pg, self.G_idx, None, s2)
+            g_ready = after(s2)
+            # current stream: weights, then the three products
+            cdl.cdl_quantize_soft(self.w, self.n_w, self.Pw, self.w_soft, self.W_idx, self.hist_w, s0)
+            w_ready = after(s0)
+            s2.wait_event(w_ready)
+            cdl.cdl_index_entropy(self.hist_w, nlw, sc[0:1], self.prob_w, None, s2)
             s0.wait_event(x_ready)
-        self._fwd(s0)
-        s0.wait_event(g_ready)
-        self._bwd_dx(s0)
-        if self.conv is not None:
+            self._fwd(s0)
+            s0.wait_event(g_ready)
+            self._bwd_dx(s0)
             s1.wait_event(after(s0))
             cdl.cdl_quantize_backward(self.x, self.gx_in, self.n_x, self.Px_b, self.dx, sc[4:5], sc[5:6], s1)
-        self._bwd_dw(s0)
-        s0.wait_event(pw_ready)
-        cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, sc[2:3], sc[3:4], s0)
+            self._bwd_dw(s0)
+            s0.wait_event(after(s2))
+            cdl.cdl_quantize_backward(self.w, self.dW, self.n_w, self.Pw_b, self.dw, sc[2:3], sc[3:4], s0)
         s0.wait_event(after(s1))
+        s0.wait_event(after(s2))
 
     def input_tensors(self):
         if self.conv is not None:
